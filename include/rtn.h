@@ -1,0 +1,147 @@
+/*
+ * rtn.h -- C ABI of librtn_b200: the forward ternary-by-ternary contraction of the
+ * Reparameterized Ternary Network (RTN, arXiv 1912.02057) on NVIDIA B200 (sm_100a).
+ *
+ * Path: ternarize + pack (Eq. 1-3, Table 1)  ->  packed ternary GEMM / implicit-GEMM conv2d
+ * (Eq. 9)  ->  affine scale/offset epilogue (Eq. 10, generalised to a weight offset).
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer unless its comment says "host".  The caller owns
+ *     every buffer; the library allocates no memory and keeps no state besides one device
+ *     status word (see rtn_last_device_status).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work and return without synchronising, except rtn_pack_weights and
+ *     rtn_last_device_status, which synchronise the stream.
+ *   - Errors are return codes; argument errors are found on the host before any launch and
+ *     leave every buffer untouched.  Nothing throws, aborts or traps.
+ *   - Codes: x (activation) and w (weight) in {-1, 0, +1}.  S_xw = sum_k x*w, S_x = sum_k x,
+ *     S_w = sum_k w (exact int32; |S| <= K <= 2^24).
+ *
+ * Packed operand format (Table 1 and the bit-plane vectors W1, W2, A1, A2 of Eq. 9)
+ *   A row of K codes occupies ceil(K/128) blocks of 32 bytes (2 bits per code):
+ *     block j, bytes  0..15 : plane 1 ("non-zero" bit) of codes 128j .. 128j+127
+ *     block j, bytes 16..31 : plane 2 ("sign" bit, 1 = positive) of the same codes
+ *   Code 128j+i sits in bit (i mod 8) of byte (i div 8) of its plane (little-endian words:
+ *   bit (i mod 32) of 32-bit word (i div 32)).  Table 1: 00 -> 0, 01 -> 0, 10 -> -1, 11 -> +1.
+ *   The packers emit the canonical zero 00 and zero-fill positions past K; every consumer also
+ *   accepts 01 as zero.  Rows are contiguous: row stride = rtn_packed_row_bytes(K).  Packed
+ *   buffers must be 16-byte aligned.
+ *   Convolution filters [N][C][kh][kw] are packed as rows of length rtn_conv_packed_k(C,kh,kw)
+ *   = kh*kw*Cw, Cw = C rounded up to 32, in (kh, kw, c) order with zero codes in the channel
+ *   padding (the im2col patch of the paper's "Methodology" section, channel innermost).
+ */
+#ifndef RTN_H_
+#define RTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RTN_OK = 0,
+    RTN_ERR_NULL = 1,           /* a required pointer is NULL                                  */
+    RTN_ERR_SHAPE = 2,          /* a size is <= 0, too large, or inconsistent                  */
+    RTN_ERR_ALIGN = 3,          /* a buffer misses its alignment                               */
+    RTN_ERR_VALUE = 4,          /* a weight code outside {-1,0,+1}, or a bad enum value        */
+    RTN_ERR_UNSUPPORTED = 5,    /* the requested variant cannot run this shape                 */
+    RTN_ERR_CUDA = 6,           /* a CUDA runtime call failed (launch, attribute, copy)        */
+    RTN_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait gave up (see last_device_status) */
+} rtn_status;
+
+/* Treatment of filter taps that fall outside the image.  The paper never mentions padding; it
+ * calls the Eq. 10 constant C "a constant which can be pre-stored", which holds only for
+ * RTN_PAD_CODE_ZERO: an outside tap has CODE 0, i.e. real value a_offset, and S_w and K cover
+ * all C*kh*kw taps.  RTN_PAD_VALUE_ZERO makes an outside tap contribute nothing (what a
+ * floating-point conv2d on the de-quantised tensor does): S_w and K then cover inside taps only. */
+typedef enum { RTN_PAD_CODE_ZERO = 0, RTN_PAD_VALUE_ZERO = 1 } rtn_pad_mode;
+
+/* Kernel family.  POPC: Eq. 9 evaluated with AND/XOR/popcount on the packed planes.
+ * I8: planes expanded to int8 in shared memory and contracted on the tensor cores
+ * (tcgen05 kind::i8).  AUTO picks per shape.  Both give identical integers. */
+typedef enum { RTN_VARIANT_AUTO = 0, RTN_VARIANT_POPC = 1, RTN_VARIANT_I8 = 2 } rtn_variant;
+
+/* Bytes of one packed row of K codes: ceil(K/128)*32.  0 if K <= 0. */
+size_t rtn_packed_row_bytes(int64_t K);
+/* Bytes of a packed operand of `rows` rows. */
+size_t rtn_packed_bytes(int64_t rows, int64_t K);
+/* Length of a packed convolution filter row: kh*kw*roundup(C,32).  0 on bad arguments. */
+int64_t rtn_conv_packed_k(int64_t C, int64_t kh, int64_t kw);
+/* Output extent of a convolution: (in + 2*pad - k)/stride + 1 (0 if not positive). */
+int64_t rtn_conv_out_dim(int64_t in, int64_t k, int64_t stride, int64_t pad);
+
+/* Weight ternary codes -> packed planes and code sums (Table 1; W1, W2 of Eq. 9; the
+ * pre-stored 1 (x) W^t of Eq. 10).  Offline step.
+ *   w_codes  int8 [N][C][kh][kw] in {-1,0,+1} (a GEMM weight [N][K] is C=K, kh=kw=1)
+ *   w_packed out, N rows of rtn_conv_packed_k(C,kh,kw) codes, 16-byte aligned
+ *   w_sum    out, int32 [1 + kh*kw][N]: row 0 = S_w over all taps and channels, row 1+t = sum
+ *            over the channels of tap t = i*kw + j (used by RTN_PAD_VALUE_ZERO at borders)
+ * Synchronises `stream`.  Returns RTN_ERR_VALUE if any code is outside {-1,0,+1} (outputs are
+ * then unspecified). */
+rtn_status rtn_pack_weights(const int8_t* w_codes, int64_t N, int64_t C, int64_t kh, int64_t kw,
+                            void* w_packed, int32_t* w_sum, void* stream);
+
+/* fp32 activations -> ternary codes (Eq. 3) -> packed planes (Table 1), plus S_x per row.
+ *   a        fp32 [M][K] row-major
+ *   t_lo,t_hi  n_thr thresholds (n_thr == 1: per layer; n_thr == K: per input feature k).
+ *            code = +1 if a > t_hi, else -1 if a < t_lo, else 0; comparisons are strict and
+ *            done in fp32, so a value equal to a threshold, and a NaN, code to 0.  With the BN
+ *            transform k*a+b of Eq. 2 (k > 0): t_hi = (0.5-b)/k, t_lo = -(0.5+b)/k.
+ *   a_packed out, M packed rows of K codes, 16-byte aligned
+ *   a_sum    out, int32 [M] = S_x (may be NULL) */
+rtn_status rtn_ternarize_pack_act(const float* a, int64_t M, int64_t K,
+                                  const float* t_lo, const float* t_hi, int64_t n_thr,
+                                  void* a_packed, int32_t* a_sum, void* stream);
+
+/* Packed ternary GEMM with the affine epilogue (Eq. 9 then Eq. 10 with a weight offset):
+ *   out[m][n] = a_s*w_s*S_xw + a_s*w_o*S_x[m] + a_o*w_s*S_w[n] + K*a_o*w_o
+ *             = sum_k (a_s*x[m][k] + a_o) * (w_s*w[n][k] + w_o)
+ *   a_packed M rows, w_packed N rows of K codes (w_packed from rtn_pack_weights with C=K)
+ *   a_sum    int32 [M] (S_x), w_sum int32 [N] (row 0 of rtn_pack_weights' w_sum)
+ *   a_scale,a_offset  n_aparam floats: 1 (per layer: gamma, beta of Eq. 4) or M (per row)
+ *   w_scale,w_offset  n_wparam floats: 1 or N (per output channel: alpha of Eq. 5; the paper
+ *                     has w_offset = 0)
+ *   out      fp32 [M][N] row-major
+ *   dbg_acc  NULL, or int32 [M][N] that receives the raw S_xw */
+rtn_status rtn_ternary_gemm(const void* a_packed, const int32_t* a_sum,
+                            const void* w_packed, const int32_t* w_sum,
+                            int64_t M, int64_t N, int64_t K,
+                            const float* a_scale, const float* a_offset, int64_t n_aparam,
+                            const float* w_scale, const float* w_offset, int64_t n_wparam,
+                            float* out, int32_t* dbg_acc, rtn_variant variant, void* stream);
+
+/* Ternary conv2d as an implicit GEMM (im2col never materialised), input ternarized in-kernel:
+ *   x        fp32 [B][C][H][W]; code per Eq. 3 with thresholds per layer (n_thr == 1) or per
+ *            input channel (n_thr == C)
+ *   w_packed,w_sum  from rtn_pack_weights(w_codes, N, C, kh, kw)
+ *   a_scale,a_offset  per-layer gamma, beta (by value); w_scale,w_offset as in the GEMM
+ *   out      fp32 [B][N][Ho][Wo], Ho = rtn_conv_out_dim(H,kh,stride,pad), same for Wo
+ *   dbg_acc  NULL, or int32 of out's shape that receives the raw S_xw
+ * out[b][n][ho][wo] = sum over taps of (a_s*x + a_o)*(w_s*w + w_o) under pad_mode's rule. */
+rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
+                              const float* t_lo, const float* t_hi, int64_t n_thr,
+                              const void* w_packed, const int32_t* w_sum,
+                              int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                              rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                              const float* w_scale, const float* w_offset, int64_t n_wparam,
+                              float* out, int32_t* dbg_acc, rtn_variant variant, void* stream);
+
+/* The variant RTN_VARIANT_AUTO resolves to for a shape (never AUTO). */
+rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
+rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
+                                    int64_t kh, int64_t kw, int64_t stride, int64_t pad);
+
+/* Synchronises `stream`, then reads and clears the device status word of the current device.
+ * RTN_OK, or RTN_ERR_DEVICE_TIMEOUT if a kernel's bounded wait (on an mbarrier of the
+ * tensor-core pipeline) ran out since the last call; that kernel's output is then invalid. */
+rtn_status rtn_last_device_status(void* stream);
+
+/* Static text for a status code. */
+const char* rtn_status_string(rtn_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RTN_H_ */

@@ -1,0 +1,14 @@
+"""B200-native forward ternary-by-ternary contraction of the Reparameterized Ternary Network
+(arXiv 1912.02057): ternarize + pack, packed ternary GEMM / conv2d, affine epilogue.
+
+The compute lives in the CUDA shared library ``librtn_b200.so`` (C ABI declared in
+``include/rtn.h``); :mod:`.binding` marshals torch tensors into it and fails loudly when the
+library is missing.  :mod:`.inputs` draws the seeded synthetic workloads.
+"""
+from .binding import (  # noqa: F401
+    RtnError, lib, lib_path,
+    rtn_packed_row_bytes, rtn_packed_bytes, rtn_conv_packed_k, rtn_conv_out_dim,
+    rtn_pack_weights, rtn_ternarize_pack_act, rtn_ternary_gemm, rtn_ternary_conv2d,
+    rtn_last_device_status, rtn_choose_gemm_variant, rtn_choose_conv_variant,
+    PAD_CODE_ZERO, PAD_VALUE_ZERO, VARIANT_AUTO, VARIANT_POPC, VARIANT_I8,
+)

@@ -1,0 +1,192 @@
+"""Seeded synthetic inputs shaped like the paper's ResNet-18 / ImageNet layers.
+
+This module only draws random numbers (numpy ``default_rng``, PCG64) and names shapes.  It
+holds none of the method's arithmetic: no thresholding, no packing, no sums.  Both the CUDA
+library's callers and the CPU checker's callers take their inputs from here, so both sides see
+the same bytes.
+
+The paper (arXiv 1912.02057, section "Experiments") evaluates on ImageNet and CIFAR-10 with
+trained weights; neither is needed for the forward contraction, and these tensors stand in:
+post-ReLU activations are max(0, N(0,1)), weight codes are i.i.d. with a chosen zero fraction
+and symmetric signs, scales are U(0.5, 1.5) and offsets U(-0.1, 0.1) (the learned values the
+paper lists in its appendix table of scales and offsets have the same order of magnitude).
+"""
+from dataclasses import dataclass, field
+
+import numpy as np
+
+
+def rng(seed):
+    return np.random.default_rng(seed)
+
+
+def weight_codes(g, shape, p_zero):
+    """i.i.d. codes: P(0) = p_zero, P(+1) = P(-1) = (1 - p_zero) / 2."""
+    u = g.random(shape, dtype=np.float32)
+    half = (1.0 - p_zero) / 2.0
+    codes = np.zeros(shape, np.int8)
+    codes[u < half] = -1
+    codes[u >= 1.0 - half] = 1
+    return codes
+
+
+def relu_normal(g, shape):
+    """fp32 max(0, N(0,1)): what a ReLU layer hands to the next layer's BN + ternarizer."""
+    a = g.standard_normal(shape, dtype=np.float32)
+    np.maximum(a, 0.0, out=a)
+    return a
+
+
+def uniform(g, lo, hi, shape=()):
+    return (lo + (hi - lo) * g.random(shape, dtype=np.float64)).astype(np.float32)
+
+
+@dataclass
+class GemmCase:
+    """One ternary GEMM problem: fp32 activations [M,K], weight codes [N,K], parameters."""
+    name: str
+    a: np.ndarray          # fp32 [M,K]
+    w_codes: np.ndarray    # int8 [N,K]
+    t_lo: np.ndarray       # fp32 [1] or [K]
+    t_hi: np.ndarray
+    a_scale: np.ndarray    # fp32 [1] or [M]
+    a_offset: np.ndarray
+    w_scale: np.ndarray    # fp32 [1] or [N]
+    w_offset: np.ndarray
+
+    @property
+    def M(self): return self.a.shape[0]
+    @property
+    def N(self): return self.w_codes.shape[0]
+    @property
+    def K(self): return self.a.shape[1]
+
+
+@dataclass
+class ConvCase:
+    """One ternary conv2d problem: fp32 NCHW input, weight codes [N,C,kh,kw], parameters."""
+    name: str
+    x: np.ndarray          # fp32 [B,C,H,W]
+    w_codes: np.ndarray    # int8 [N,C,kh,kw]
+    stride: int
+    pad: int
+    t_lo: np.ndarray       # fp32 [1] or [C]
+    t_hi: np.ndarray
+    a_scale: float
+    a_offset: float
+    w_scale: np.ndarray    # fp32 [1] or [N]
+    w_offset: np.ndarray
+    notes: dict = field(default_factory=dict)
+
+    @property
+    def B(self): return self.x.shape[0]
+    @property
+    def C(self): return self.x.shape[1]
+    @property
+    def H(self): return self.x.shape[2]
+    @property
+    def W(self): return self.x.shape[3]
+    @property
+    def N(self): return self.w_codes.shape[0]
+    @property
+    def kh(self): return self.w_codes.shape[2]
+    @property
+    def kw(self): return self.w_codes.shape[3]
+    @property
+    def Ho(self): return (self.H + 2 * self.pad - self.kh) // self.stride + 1
+    @property
+    def Wo(self): return (self.W + 2 * self.pad - self.kw) // self.stride + 1
+    @property
+    def gemm_mnk(self):
+        return (self.B * self.Ho * self.Wo, self.N, self.C * self.kh * self.kw)
+
+
+def gemm_case(name, M, N, K, seed, p_zero, act="relu", thresholds=(0.3, 1.0),
+              per_row_act_params=False, a_scale=None, a_offset=None, per_k_thresholds=False):
+    g = rng(seed)
+    w = weight_codes(g, (N, K), p_zero)
+    if act == "relu":
+        a = relu_normal(g, (M, K))
+    elif act == "uniform3":          # U(-1.5, 1.5): thresholds -0.5/+0.5 split it in thirds
+        a = (3.0 * g.random((M, K), dtype=np.float32) - 1.5).astype(np.float32)
+    else:
+        raise ValueError(act)
+    if per_k_thresholds:
+        lo = uniform(g, thresholds[0] - 0.1, thresholds[0] + 0.1, (K,))
+        hi = uniform(g, thresholds[1] - 0.1, thresholds[1] + 0.1, (K,))
+    else:
+        lo = np.array([thresholds[0]], np.float32)
+        hi = np.array([thresholds[1]], np.float32)
+    w_s, w_o = uniform(g, 0.5, 1.5, (N,)), uniform(g, -0.1, 0.1, (N,))
+    if per_row_act_params:
+        a_s, a_o = uniform(g, 0.5, 1.5, (M,)), uniform(g, -0.1, 0.1, (M,))
+    else:
+        a_s = np.array([1.0 if a_scale is None else a_scale], np.float32)
+        a_o = np.array([0.05 if a_offset is None else a_offset], np.float32)
+    return GemmCase(name, a, w, lo, hi, a_s, a_o, w_s, w_o)
+
+
+def conv_case(name, B, C, H, W, N, k, stride, pad, seed, p_zero, thresholds="around_offset",
+              per_channel_thresholds=False):
+    g = rng(seed)
+    w = weight_codes(g, (N, C, k, k), p_zero)
+    x = relu_normal(g, (B, C, H, W))
+    w_s, w_o = uniform(g, 0.5, 1.5, (N,)), uniform(g, -0.1, 0.1, (N,))
+    a_s, a_o = float(uniform(g, 0.5, 1.5)), float(uniform(g, -0.1, 0.1))
+    if thresholds == "around_offset":      # +-0.5 around the activation offset
+        lo, hi = a_o - 0.5, a_o + 0.5
+    else:
+        lo, hi = thresholds
+    if per_channel_thresholds:
+        t_lo = uniform(g, lo - 0.1, lo + 0.1, (C,))
+        t_hi = uniform(g, hi - 0.1, hi + 0.1, (C,))
+    else:
+        t_lo, t_hi = np.array([lo], np.float32), np.array([hi], np.float32)
+    return ConvCase(name, x, w, stride, pad, t_lo, t_hi, a_s, a_o, w_s, w_o)
+
+
+# ------------------------------------------------------------------ the five named workloads
+def config1():
+    """GEMM 64x64x576 (a 3x3x64 conv unrolled), P(0)=0.4, thresholds 0.3 / 1.0, seed 0."""
+    return gemm_case("cfg1_gemm_64x64x576", 64, 64, 576, seed=0, p_zero=0.4,
+                     thresholds=(0.3, 1.0), a_scale=1.0, a_offset=0.05)
+
+
+def config2(batch=32, thresholds="around_offset"):
+    """conv 3x3 s1 p1, 64->64, 56x56, batch 32; thresholds +-0.5 around the activation offset."""
+    return conv_case(f"cfg2_conv3x3_c64_56x56_b{batch}", batch, 64, 56, 56, 64, 3, 1, 1,
+                     seed=2, p_zero=0.4, thresholds=thresholds)
+
+
+def config3a(p_zero=0.5, batch=128):
+    """conv 3x3 s1 p1, 256->256, 14x14, batch 128; weight-zero fraction swept."""
+    return conv_case(f"cfg3a_conv3x3_c256_14x14_b{batch}_z{p_zero}", batch, 256, 14, 14, 256, 3,
+                     1, 1, seed=3, p_zero=p_zero)
+
+
+def config3b(p_zero=0.5, batch=128):
+    """1x1 stride-2 downsample conv 128->256 at 28x28, batch 128."""
+    return conv_case(f"cfg3b_conv1x1s2_c128_28x28_b{batch}_z{p_zero}", batch, 128, 28, 28, 256, 1,
+                     2, 0, seed=31, p_zero=p_zero)
+
+
+def config5(n):
+    """Square GEMM M=N=K=n, codes 1/3 each, per-row activation and per-column weight params."""
+    return gemm_case(f"cfg5_gemm_{n}", n, n, n, seed=5, p_zero=1.0 / 3.0, act="uniform3",
+                     thresholds=(-0.5, 0.5), per_row_act_params=True)
+
+
+def resnet18_ternary_layers():
+    """The 19 ternary conv layers of ResNet-18 (stages 1-4; stem and FC stay full precision),
+    in the order of the paper's appendix table of learned scales and offsets.
+    Tuples: (name, C_in, C_out, k, stride, pad, H_in)."""
+    L = []
+    L += [(f"layer1.{b}.conv{c}", 64, 64, 3, 1, 1, 56) for b in (0, 1) for c in (1, 2)]
+    for s, (cin, cout, hin) in enumerate([(64, 128, 56), (128, 256, 28), (256, 512, 14)], start=2):
+        hout = hin // 2
+        L += [(f"layer{s}.0.conv1", cin, cout, 3, 2, 1, hin),
+              (f"layer{s}.0.conv2", cout, cout, 3, 1, 1, hout),
+              (f"layer{s}.0.downsample.0", cin, cout, 1, 2, 0, hin),
+              (f"layer{s}.1.conv1", cout, cout, 3, 1, 1, hout),
+              (f"layer{s}.1.conv2", cout, cout, 3, 1, 1, hout)]
+    return L
