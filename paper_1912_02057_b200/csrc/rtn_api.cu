@@ -1,0 +1,258 @@
+// C ABI of librtn_b200 (declared in rtn.h): argument checks, variant choice, launches.
+#include "rtn_internal.cuh"
+
+#include <limits.h>
+
+namespace {
+
+// One status word per device, living in device memory for the life of the library.
+__device__ unsigned g_status_word;
+
+constexpr int kMaxDevices = 64;
+unsigned* g_status_ptr[kMaxDevices];
+
+// Device address of the status word of the current device (NULL on failure).
+unsigned* status_word()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    if (g_status_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        if (cudaMemset(p, 0, sizeof(unsigned)) != cudaSuccess) return nullptr;
+        g_status_ptr[dev] = static_cast<unsigned*>(p);
+    }
+    return g_status_ptr[dev];
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+constexpr int64_t kMaxK = int64_t(1) << 24;       // |S| <= K must stay exact in fp32 and int32
+constexpr int64_t kMaxDim = int64_t(1) << 31;
+
+rtn_status check_params(const float* s, const float* o, int64_t n, int64_t full)
+{
+    if (s == nullptr || o == nullptr) return RTN_ERR_NULL;
+    if (n != 1 && n != full) return RTN_ERR_SHAPE;
+    if (!aligned4(s) || !aligned4(o)) return RTN_ERR_ALIGN;
+    return RTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rtn_packed_row_bytes(int64_t K)
+{
+    if (K <= 0) return 0;
+    return (size_t)rtn::blocks_of(K) * rtn::kBlockBytes;
+}
+
+size_t rtn_packed_bytes(int64_t rows, int64_t K)
+{
+    if (rows <= 0 || K <= 0) return 0;
+    return (size_t)rows * rtn_packed_row_bytes(K);
+}
+
+int64_t rtn_conv_packed_k(int64_t C, int64_t kh, int64_t kw)
+{
+    if (C <= 0 || kh <= 0 || kw <= 0) return 0;
+    return kh * kw * ((C + 31) / 32 * 32);
+}
+
+int64_t rtn_conv_out_dim(int64_t in, int64_t k, int64_t stride, int64_t pad)
+{
+    if (in <= 0 || k <= 0 || stride <= 0 || pad < 0) return 0;
+    const int64_t span = in + 2 * pad - k;
+    if (span < 0) return 0;
+    return span / stride + 1;
+}
+
+const char* rtn_status_string(rtn_status s)
+{
+    switch (s) {
+        case RTN_OK: return "RTN_OK";
+        case RTN_ERR_NULL: return "RTN_ERR_NULL: a required pointer is NULL";
+        case RTN_ERR_SHAPE: return "RTN_ERR_SHAPE: bad or inconsistent size";
+        case RTN_ERR_ALIGN: return "RTN_ERR_ALIGN: buffer alignment";
+        case RTN_ERR_VALUE: return "RTN_ERR_VALUE: weight code outside {-1,0,+1} or bad enum";
+        case RTN_ERR_UNSUPPORTED: return "RTN_ERR_UNSUPPORTED: variant cannot run this shape";
+        case RTN_ERR_CUDA: return "RTN_ERR_CUDA: CUDA runtime call failed";
+        case RTN_ERR_DEVICE_TIMEOUT: return "RTN_ERR_DEVICE_TIMEOUT: bounded device wait gave up";
+    }
+    return "unknown rtn_status";
+}
+
+rtn_status rtn_pack_weights(const int8_t* w_codes, int64_t N, int64_t C, int64_t kh, int64_t kw,
+                            void* w_packed, int32_t* w_sum, void* stream)
+{
+    if (w_codes == nullptr || w_packed == nullptr || w_sum == nullptr) return RTN_ERR_NULL;
+    if (N <= 0 || C <= 0 || kh <= 0 || kw <= 0 || kh > 64 || kw > 64 || N >= kMaxDim) return RTN_ERR_SHAPE;
+    if (C > kMaxK || rtn_conv_packed_k(C, kh, kw) > kMaxK) return RTN_ERR_SHAPE;
+    if (!aligned16(w_packed) || !aligned4(w_sum)) return RTN_ERR_ALIGN;
+    unsigned* st = status_word();
+    if (st == nullptr) return RTN_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (rtn::launch_pack_weights(w_codes, N, C, (int)kh, (int)kw, static_cast<uint8_t*>(w_packed),
+                                 w_sum, st, s) != cudaSuccess) return RTN_ERR_CUDA;
+    unsigned h = 0;
+    if (cudaMemcpyAsync(&h, st, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return RTN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return RTN_ERR_CUDA;
+    if (h & rtn::kStatusBadWeightCode) {
+        const unsigned keep = h & ~rtn::kStatusBadWeightCode;
+        cudaMemcpyAsync(st, &keep, sizeof(keep), cudaMemcpyHostToDevice, s);
+        cudaStreamSynchronize(s);
+        return RTN_ERR_VALUE;
+    }
+    return RTN_OK;
+}
+
+rtn_status rtn_ternarize_pack_act(const float* a, int64_t M, int64_t K,
+                                  const float* t_lo, const float* t_hi, int64_t n_thr,
+                                  void* a_packed, int32_t* a_sum, void* stream)
+{
+    if (a == nullptr || t_lo == nullptr || t_hi == nullptr || a_packed == nullptr) return RTN_ERR_NULL;
+    if (M <= 0 || K <= 0 || M >= kMaxDim || K > kMaxK) return RTN_ERR_SHAPE;
+    if (n_thr != 1 && n_thr != K) return RTN_ERR_SHAPE;
+    if (!aligned16(a_packed) || !aligned4(a) || !aligned4(t_lo) || !aligned4(t_hi) ||
+        (a_sum != nullptr && !aligned4(a_sum))) return RTN_ERR_ALIGN;
+    if (rtn::launch_ternarize_pack(a, M, K, t_lo, t_hi, n_thr, static_cast<uint8_t*>(a_packed), a_sum,
+                                   static_cast<cudaStream_t>(stream)) != cudaSuccess) return RTN_ERR_CUDA;
+    return RTN_OK;
+}
+
+rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K)
+{
+    if (!rtn::gemm_i8_supported(M, N, K)) return RTN_VARIANT_POPC;
+    // Tiny problems finish inside one wave of the bit-plane kernel before the tensor-core
+    // pipeline has filled; everything else is far faster on the tensor cores.
+    if (M * N <= 128 * 128 && K <= 1024) return RTN_VARIANT_POPC;
+    return RTN_VARIANT_I8;
+}
+
+rtn_status rtn_ternary_gemm(const void* a_packed, const int32_t* a_sum,
+                            const void* w_packed, const int32_t* w_sum,
+                            int64_t M, int64_t N, int64_t K,
+                            const float* a_scale, const float* a_offset, int64_t n_aparam,
+                            const float* w_scale, const float* w_offset, int64_t n_wparam,
+                            float* out, int32_t* dbg_acc, rtn_variant variant, void* stream)
+{
+    if (a_packed == nullptr || a_sum == nullptr || w_packed == nullptr || w_sum == nullptr ||
+        out == nullptr) return RTN_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || M >= kMaxDim || N >= kMaxDim || K > kMaxK) return RTN_ERR_SHAPE;
+    rtn_status st = check_params(a_scale, a_offset, n_aparam, M);
+    if (st != RTN_OK) return st;
+    st = check_params(w_scale, w_offset, n_wparam, N);
+    if (st != RTN_OK) return st;
+    if (!aligned16(a_packed) || !aligned16(w_packed) || !aligned4(a_sum) || !aligned4(w_sum) ||
+        !aligned4(out) || (dbg_acc != nullptr && !aligned4(dbg_acc))) return RTN_ERR_ALIGN;
+    if (variant != RTN_VARIANT_AUTO && variant != RTN_VARIANT_POPC && variant != RTN_VARIANT_I8)
+        return RTN_ERR_VALUE;
+    if (variant == RTN_VARIANT_AUTO) variant = rtn_choose_gemm_variant(M, N, K);
+    if (variant == RTN_VARIANT_I8 && !rtn::gemm_i8_supported(M, N, K)) return RTN_ERR_UNSUPPORTED;
+    if (variant == RTN_VARIANT_POPC && ((M + 15) / 16 > INT_MAX || (N + 63) / 64 > 65535))
+        return RTN_ERR_UNSUPPORTED;
+
+    rtn::GemmArgs g;
+    g.a_packed = static_cast<const uint8_t*>(a_packed);
+    g.a_sum = a_sum;
+    g.w_packed = static_cast<const uint8_t*>(w_packed);
+    g.w_sum = w_sum;
+    g.M = M; g.N = N; g.K = K;
+    g.ep = rtn::EpilogueParams{a_scale, a_offset, n_aparam, 0.f, 0.f, w_scale, w_offset, n_wparam};
+    g.out = out;
+    g.dbg_acc = dbg_acc;
+    g.status = status_word();
+    if (g.status == nullptr) return RTN_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const cudaError_t e = (variant == RTN_VARIANT_I8) ? rtn::launch_gemm_i8(g, s)
+                                                      : rtn::launch_gemm_popc(g, s);
+    return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
+static rtn_status fill_conv_args(rtn::ConvArgs& c, const float* x, int64_t B, int64_t C, int64_t H,
+                                 int64_t W, const float* t_lo, const float* t_hi, int64_t n_thr,
+                                 const void* w_packed, const int32_t* w_sum, int64_t N, int64_t kh,
+                                 int64_t kw, int64_t stride, int64_t pad, rtn_pad_mode pad_mode,
+                                 float a_scale, float a_offset, const float* w_scale,
+                                 const float* w_offset, int64_t n_wparam, float* out, int32_t* dbg_acc)
+{
+    if (x == nullptr || t_lo == nullptr || t_hi == nullptr || w_packed == nullptr ||
+        w_sum == nullptr || out == nullptr) return RTN_ERR_NULL;
+    const int64_t lim = 1 << 20;
+    if (B <= 0 || C <= 0 || H <= 0 || W <= 0 || N <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0 ||
+        B > lim || C > lim || H > lim || W > lim || N > lim || kh > 64 || kw > 64 || stride > 64 ||
+        pad > 64) return RTN_ERR_SHAPE;
+    if (n_thr != 1 && n_thr != C) return RTN_ERR_SHAPE;
+    const int64_t Ho = rtn_conv_out_dim(H, kh, stride, pad), Wo = rtn_conv_out_dim(W, kw, stride, pad);
+    if (Ho <= 0 || Wo <= 0) return RTN_ERR_SHAPE;
+    if (rtn_conv_packed_k(C, kh, kw) > kMaxK) return RTN_ERR_SHAPE;
+    if (B * C * H * W >= (int64_t(1) << 40) || B * N * Ho * Wo >= (int64_t(1) << 40)) return RTN_ERR_SHAPE;
+    if (pad_mode != RTN_PAD_CODE_ZERO && pad_mode != RTN_PAD_VALUE_ZERO) return RTN_ERR_VALUE;
+    rtn_status st = check_params(w_scale, w_offset, n_wparam, N);
+    if (st != RTN_OK) return st;
+    if (!aligned16(w_packed) || !aligned4(x) || !aligned4(out) || !aligned4(w_sum) || !aligned4(t_lo) ||
+        !aligned4(t_hi) || (dbg_acc != nullptr && !aligned4(dbg_acc))) return RTN_ERR_ALIGN;
+    c.x = x; c.B = (int)B; c.C = (int)C; c.H = (int)H; c.W = (int)W;
+    c.t_lo = t_lo; c.t_hi = t_hi; c.n_thr = (int)n_thr;
+    c.w_packed = static_cast<const uint8_t*>(w_packed); c.w_sum = w_sum;
+    c.N = (int)N; c.kh = (int)kh; c.kw = (int)kw; c.stride = (int)stride; c.pad = (int)pad;
+    c.Ho = (int)Ho; c.Wo = (int)Wo; c.pad_mode = (int)pad_mode;
+    c.ep = rtn::EpilogueParams{nullptr, nullptr, 1, a_scale, a_offset, w_scale, w_offset, n_wparam};
+    c.out = out; c.dbg_acc = dbg_acc; c.status = nullptr;
+    return RTN_OK;
+}
+
+rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
+                                    int64_t kh, int64_t kw, int64_t stride, int64_t pad)
+{
+    rtn::ConvArgs c{};
+    c.B = (int)B; c.C = (int)C; c.H = (int)H; c.W = (int)W; c.N = (int)N; c.kh = (int)kh; c.kw = (int)kw;
+    c.stride = (int)stride; c.pad = (int)pad;
+    c.Ho = (int)rtn_conv_out_dim(H, kh, stride, pad); c.Wo = (int)rtn_conv_out_dim(W, kw, stride, pad);
+    return rtn::conv_i8_supported(c) ? RTN_VARIANT_I8 : RTN_VARIANT_POPC;
+}
+
+rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
+                              const float* t_lo, const float* t_hi, int64_t n_thr,
+                              const void* w_packed, const int32_t* w_sum,
+                              int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                              rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                              const float* w_scale, const float* w_offset, int64_t n_wparam,
+                              float* out, int32_t* dbg_acc, rtn_variant variant, void* stream)
+{
+    rtn::ConvArgs c{};
+    rtn_status st = fill_conv_args(c, x, B, C, H, W, t_lo, t_hi, n_thr, w_packed, w_sum, N, kh, kw,
+                                   stride, pad, pad_mode, a_scale, a_offset, w_scale, w_offset,
+                                   n_wparam, out, dbg_acc);
+    if (st != RTN_OK) return st;
+    if (variant != RTN_VARIANT_AUTO && variant != RTN_VARIANT_POPC && variant != RTN_VARIANT_I8)
+        return RTN_ERR_VALUE;
+    if (variant == RTN_VARIANT_AUTO) variant = rtn::conv_i8_supported(c) ? RTN_VARIANT_I8 : RTN_VARIANT_POPC;
+    if (variant == RTN_VARIANT_I8 && !rtn::conv_i8_supported(c)) return RTN_ERR_UNSUPPORTED;
+    if (variant == RTN_VARIANT_POPC && !rtn::conv_popc_supported(c)) return RTN_ERR_UNSUPPORTED;
+    c.status = status_word();
+    if (c.status == nullptr) return RTN_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const cudaError_t e = (variant == RTN_VARIANT_I8) ? rtn::launch_conv_i8(c, s)
+                                                      : rtn::launch_conv_popc(c, s);
+    return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
+rtn_status rtn_last_device_status(void* stream)
+{
+    unsigned* st = status_word();
+    if (st == nullptr) return RTN_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned h = 0;
+    if (cudaMemcpyAsync(&h, st, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return RTN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return RTN_ERR_CUDA;
+    if (h != 0) {
+        if (cudaMemsetAsync(st, 0, sizeof(unsigned), s) != cudaSuccess) return RTN_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return RTN_ERR_CUDA;
+    }
+    return (h & rtn::kStatusWaitTimeout) ? RTN_ERR_DEVICE_TIMEOUT : RTN_OK;
+}
+
+}  // extern "C"

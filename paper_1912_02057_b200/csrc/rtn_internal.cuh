@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of librtn_b200 (not installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "rtn.h"
+
+namespace rtn {
+
+// Bits of the device status word.
+constexpr unsigned kStatusBadWeightCode = 1u;   // rtn_pack_weights met a code outside {-1,0,+1}
+constexpr unsigned kStatusWaitTimeout   = 2u;   // a bounded mbarrier wait gave up
+
+// Packed format: 128 codes per 32-byte block (16 B plane 1 "non-zero", 16 B plane 2 "sign").
+constexpr int kBlockCodes = 128;
+constexpr int kBlockBytes = 32;
+
+inline int64_t blocks_of(int64_t K) { return (K + kBlockCodes - 1) / kBlockCodes; }
+
+// Arguments of the affine epilogue, common to GEMM and conv.
+//   out = a_s*w_s*S_xw + a_s*w_o*S_x + a_o*w_s*S_w + K*a_o*w_o      (Eq. 10 plus a weight offset)
+struct EpilogueParams {
+    const float* a_scale;   // device, n_aparam entries (GEMM) -- or NULL when by value (conv)
+    const float* a_offset;
+    int64_t n_aparam;
+    float a_scale_val;      // used when a_scale == NULL
+    float a_offset_val;
+    const float* w_scale;   // device, n_wparam entries
+    const float* w_offset;
+    int64_t n_wparam;
+};
+
+struct GemmArgs {
+    const uint8_t* a_packed;
+    const int32_t* a_sum;
+    const uint8_t* w_packed;
+    const int32_t* w_sum;
+    int64_t M, N, K;
+    EpilogueParams ep;
+    float* out;
+    int32_t* dbg_acc;
+    unsigned* status;       // device status word
+};
+
+struct ConvArgs {
+    const float* x;
+    int B, C, H, W;
+    const float* t_lo;
+    const float* t_hi;
+    int n_thr;
+    const uint8_t* w_packed;
+    const int32_t* w_sum;   // [1 + kh*kw][N]
+    int N, kh, kw, stride, pad, Ho, Wo;
+    int pad_mode;
+    EpilogueParams ep;
+    float* out;
+    int32_t* dbg_acc;
+    unsigned* status;
+};
+
+// Launchers (each returns the cudaError_t of its launch).
+cudaError_t launch_pack_weights(const int8_t* w, int64_t N, int64_t C, int kh, int kw,
+                                uint8_t* packed, int32_t* w_sum, unsigned* status, cudaStream_t s);
+cudaError_t launch_ternarize_pack(const float* a, int64_t M, int64_t K, const float* t_lo,
+                                  const float* t_hi, int64_t n_thr, uint8_t* packed, int32_t* a_sum,
+                                  cudaStream_t s);
+cudaError_t launch_gemm_popc(const GemmArgs& g, cudaStream_t s);
+bool conv_popc_supported(const ConvArgs& c);
+cudaError_t launch_conv_popc(const ConvArgs& c, cudaStream_t s);
+
+// Tensor-core (tcgen05 kind::i8) variants; *_supported say whether a shape can run there.
+bool gemm_i8_supported(int64_t M, int64_t N, int64_t K);
+cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s);
+bool conv_i8_supported(const ConvArgs& c);
+cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s);
+
+// ----------------------------------------------------------------------------------------------
+// Device helpers
+// ----------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+// Eq. 3, strict comparisons in fp32; the +1 case is tested first.  Returns (nz, positive).
+__device__ __forceinline__ void ternarize(float v, float lo, float hi, bool& nz, bool& pos)
+{
+    pos = v > hi;
+    nz = pos || (v < lo);
+}
+
+// Epilogue in double, rounded once to fp32 (used by the POPC kernels).
+__device__ __forceinline__ float epilogue_f64(int s_xw, int s_x, int s_w, double k_eff,
+                                              double a_s, double a_o, double w_s, double w_o)
+{
+    const double r = a_s * w_s * (double)s_xw + a_s * w_o * (double)s_x
+                   + a_o * w_s * (double)s_w + k_eff * a_o * w_o;
+    return (float)r;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace rtn

@@ -1,0 +1,71 @@
+"""The shared library loads without a GPU and exports every entry point rtn.h declares; argument
+errors are reported on the host before anything is launched."""
+import ctypes
+import os
+import re
+
+import paper_1912_02057_b200 as rtn
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "rtn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rtn_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert {"rtn_pack_weights", "rtn_ternarize_pack_act", "rtn_ternary_gemm",
+            "rtn_ternary_conv2d"} <= set(names)
+    L = ctypes.CDLL(rtn.lib_path())
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_size_helpers():
+    assert rtn.rtn_packed_row_bytes(1) == 32
+    assert rtn.rtn_packed_row_bytes(128) == 32
+    assert rtn.rtn_packed_row_bytes(129) == 64
+    assert rtn.rtn_packed_row_bytes(576) == 160
+    assert rtn.rtn_packed_row_bytes(0) == 0
+    assert rtn.rtn_packed_bytes(64, 576) == 64 * 160
+    assert rtn.rtn_conv_packed_k(64, 3, 3) == 576
+    assert rtn.rtn_conv_packed_k(3, 7, 7) == 49 * 32
+    assert rtn.rtn_conv_packed_k(0, 3, 3) == 0
+    assert rtn.rtn_conv_out_dim(56, 3, 1, 1) == 56
+    assert rtn.rtn_conv_out_dim(56, 3, 2, 1) == 28
+    assert rtn.rtn_conv_out_dim(28, 1, 2, 0) == 14
+    assert rtn.rtn_conv_out_dim(2, 3, 1, 0) == 0
+
+
+def test_argument_errors_come_back_as_codes_without_a_gpu():
+    L = rtn.lib()
+    vp = ctypes.c_void_p
+    # NULL pointers
+    assert L.rtn_pack_weights(None, 4, 4, 1, 1, None, None, None) == 1
+    assert L.rtn_ternarize_pack_act(None, 4, 4, None, None, 1, None, None, None) == 1
+    fake = vp(0x1000)          # never dereferenced: the checks below fail before any launch
+    odd = vp(0x1004)
+    assert L.rtn_pack_weights(fake, 0, 4, 1, 1, fake, fake, None) == 2
+    assert L.rtn_pack_weights(fake, 4, 4, 1, 1, odd, fake, None) == 3
+    assert L.rtn_ternarize_pack_act(fake, 4, 4, fake, fake, 3, fake, None, None) == 2
+    assert L.rtn_ternarize_pack_act(fake, 4, 4, fake, fake, 1, odd, None, None) == 3
+    gemm = lambda M, N, K, na, nw, variant, a=fake: L.rtn_ternary_gemm(
+        a, fake, fake, fake, M, N, K, fake, fake, na, fake, fake, nw, fake, None, variant, None)
+    assert gemm(0, 4, 4, 1, 1, 0) == 2
+    assert gemm(4, 4, 1 << 25, 1, 1, 0) == 2
+    assert gemm(4, 4, 4, 3, 1, 0) == 2
+    assert gemm(4, 4, 4, 1, 5, 0) == 2
+    assert gemm(4, 4, 4, 1, 1, 0, a=odd) == 3
+    assert gemm(4, 4, 4, 1, 1, 9) == 4
+    conv = lambda C, k, stride, pad, mode, nthr=1: L.rtn_ternary_conv2d(
+        fake, 1, C, 8, 8, fake, fake, nthr, fake, fake, 4, k, k, stride, pad, mode,
+        ctypes.c_float(1.0), ctypes.c_float(0.0), fake, fake, 1, fake, None, 0, None)
+    assert conv(0, 3, 1, 1, 0) == 2
+    assert conv(4, 3, 0, 1, 0) == 2
+    assert conv(4, 11, 1, 0, 0) == 2          # filter larger than the image
+    assert conv(4, 3, 1, 1, 0, nthr=3) == 2
+    assert conv(4, 3, 1, 1, 7) == 4
+    assert rtn.lib().rtn_status_string(2).startswith(b"RTN_ERR_SHAPE")
