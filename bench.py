@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the ternary hot path: effective ternary TOPS (2*M*N*K / s).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step = one pass of the whole hot path over one batch of seeded synthetic input: for a conv
+workload a single rtn_ternary_conv2d call (ternarize in-kernel -> implicit-GEMM contraction ->
+affine epilogue); for a GEMM workload rtn_ternarize_pack_act followed by rtn_ternary_gemm.  Weight
+packing is the offline step and happens before the timed region.
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an independent replica on
+its own GPU -- the path has no exchange step -- and `value` is the work of all ranks divided by
+the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1912_02057_b200 import inputs  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+WORKLOADS = {
+    "cfg2_conv3x3_c64_56x56_b32": lambda: inputs.config2(batch=32),
+    "cfg3a_conv3x3_c256_14x14_b128": lambda: inputs.config3a(0.5, batch=128),
+    "cfg3b_conv1x1s2_c128_28x28_b128": lambda: inputs.config3b(0.5, batch=128),
+    "cfg1_gemm_64x64x576": inputs.config1,
+    "cfg5_gemm_2048": lambda: inputs.config5(2048),
+    "cfg5_gemm_4096": lambda: inputs.config5(4096),
+    "cfg5_gemm_8192": lambda: inputs.config5(8192),
+}
+DEFAULT_WORKLOAD = "cfg2_conv3x3_c64_56x56_b32"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(case):
+    """Bytes the method must move per step: fp32 input once, fp32 output once, packed weights once."""
+    if isinstance(case, inputs.ConvCase):
+        M, N, K = case.gemm_mnk
+        kc = case.kh * case.kw * ((case.C + 31) // 32 * 32)
+        return case.x.nbytes + 4 * M * N + N * ((kc + 127) // 128) * 32
+    M, N, K = case.M, case.N, case.K
+    packed = lambda r: r * ((K + 127) // 128) * 32
+    # ternarize+pack: read fp32, write planes; GEMM: read both packed operands, write fp32
+    return case.a.nbytes + packed(M) + packed(M) + packed(N) + 4 * M * N
+
+
+def ops_of(case):
+    M, N, K = case.gemm_mnk if isinstance(case, inputs.ConvCase) else (case.M, case.N, case.K)
+    return 2.0 * M * N * K
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg (reference arm and cpu_baseline)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(case, budget_s=12.0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload.
+    Returns (ops per second, seconds, description)."""
+    import oracle
+    if isinstance(case, inputs.ConvCase):
+        def run(nb):
+            x = case.x[:nb]
+            t0 = time.perf_counter()
+            codes = oracle.ternarize(x, case.t_lo, case.t_hi, channel_axis=1)
+            oracle.conv2d(codes, case.w_codes, case.stride, case.pad, oracle.PAD_CODE_ZERO,
+                          case.a_scale, case.a_offset, case.w_scale, case.w_offset)
+            dt = time.perf_counter() - t0
+            M, N, K = case.gemm_mnk
+            return 2.0 * (M // case.B * nb) * N * K, dt
+        ops, dt = run(1)
+        nb = int(max(1, min(case.B, budget_s / max(dt, 1e-6))))
+        if nb > 1:
+            ops, dt = run(nb)
+        return ops / dt, dt, f"first {nb} of {case.B} images, all output channels (ternarize + conv2d + epilogue)"
+
+    def run(rows):
+        a = case.a[:rows]
+        t0 = time.perf_counter()
+        codes = oracle.ternarize(a, case.t_lo, case.t_hi, channel_axis=1)
+        n_ap = case.a_scale.size
+        oracle.gemm(codes, case.w_codes, case.a_scale[:rows] if n_ap > 1 else case.a_scale,
+                    case.a_offset[:rows] if n_ap > 1 else case.a_offset, case.w_scale, case.w_offset)
+        dt = time.perf_counter() - t0
+        return 2.0 * rows * case.N * case.K, dt
+    rows = min(case.M, 16)
+    ops, dt = run(rows)
+    rows2 = int(max(rows, min(case.M, rows * budget_s / max(dt, 1e-6))))
+    if rows2 > rows:
+        ops, dt = run(rows2)
+        rows = rows2
+    return ops / dt, dt, f"first {rows} of {case.M} rows, all columns (ternarize + gemm + epilogue)"
+
+
+def run_reference(args, case, name):
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step_budget = max(0.2, min(12.0, 60.0 / max(1, args.steps + args.warmup)))
+    sample = ""
+    for _ in range(args.warmup):
+        _, _, sample = oracle_sample(case, per_step_budget)
+    rates, secs = [], []
+    for _ in range(args.steps):
+        r, dt, sample = oracle_sample(case, per_step_budget)
+        rates.append(r)
+        secs.append(dt)
+    value = float(np.mean(rates)) / 1e12
+    line = {
+        "impl": "reference", "metric": "effective ternary TOPS (2MNK/s)", "value": value,
+        "unit": "TOPS", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * float(np.mean(secs)), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": name, "note": "CPU oracle on a bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": "TOPS", "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU leg
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, case, name):
+    import torch
+    import torch.distributed as dist
+    import paper_1912_02057_b200 as rtn
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    is_conv = isinstance(case, inputs.ConvCase)
+
+    # resident inputs: enough rotating copies that consecutive steps never find their data in L2
+    step_bytes = algorithmic_bytes(case)
+    n_sets = max(2, int(np.ceil(2.5 * L2_BYTES / step_bytes)))
+    n_sets = min(n_sets, 64)
+    w_packed, w_sum = rtn.rtn_pack_weights(dev(case.w_codes))
+    w_s, w_o = dev(case.w_scale), dev(case.w_offset)
+    t_lo, t_hi = dev(case.t_lo), dev(case.t_hi)
+    if is_conv:
+        xs = [dev(case.x) for _ in range(n_sets)]
+        outs = [torch.empty((case.B, case.N, case.Ho, case.Wo), dtype=torch.float32, device="cuda")
+                for _ in range(n_sets)]
+        variant = rtn.rtn_choose_conv_variant(case.B, case.C, case.H, case.W, case.N, case.kh,
+                                              case.kw, case.stride, case.pad)
+        launches_per_step = 1
+
+        def step(i):
+            j = i % n_sets
+            rtn.rtn_ternary_conv2d(xs[j], t_lo, t_hi, w_packed, w_sum, case.N, case.kh, case.kw,
+                                   case.stride, case.pad, rtn.PAD_CODE_ZERO, case.a_scale,
+                                   case.a_offset, w_s, w_o, out=outs[j])
+            return outs[j]
+        host_in = torch.from_numpy(case.x).pin_memory()
+    else:
+        M, N, K = case.M, case.N, case.K
+        xs = [dev(case.a) for _ in range(n_sets)]
+        a_s, a_o = dev(case.a_scale), dev(case.a_offset)
+        packs = [torch.empty((M, rtn.rtn_packed_row_bytes(K)), dtype=torch.uint8, device="cuda")
+                 for _ in range(n_sets)]
+        sums = [torch.empty((M,), dtype=torch.int32, device="cuda") for _ in range(n_sets)]
+        outs = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _ in range(n_sets)]
+        variant = rtn.rtn_choose_gemm_variant(M, N, K)
+        launches_per_step = 2
+
+        def step(i):
+            j = i % n_sets
+            rtn.rtn_ternarize_pack_act(xs[j], t_lo, t_hi, out=packs[j], out_sum=sums[j])
+            rtn.rtn_ternary_gemm(packs[j], sums[j], w_packed, w_sum[0], M, N, K, a_s, a_o, w_s, w_o,
+                                 out=outs[j])
+            return outs[j]
+        host_in = torch.from_numpy(case.a).pin_memory()
+    host_out = torch.empty(outs[0].shape, dtype=torch.float32).pin_memory()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        step(args.warmup + i)
+        ev[i][1].record()
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    status = rtn.rtn_last_device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} after the timed region")
+
+    # ---- end to end: pinned host input -> device, the C-ABI call(s), result -> pinned host
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(2):
+        xs[0].copy_(host_in, non_blocking=True)
+        host_out.copy_(step(0), non_blocking=True)
+    barrier()
+    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_begin.record()
+    for i in range(e2e_steps):
+        j = i % n_sets
+        xs[j].copy_(host_in, non_blocking=True)
+        host_out.copy_(step(j), non_blocking=True)
+    e_end.record()
+    barrier()
+    e2e_ms = e_begin.elapsed_time(e_end) / e2e_steps
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+    ops = ops_of(case)
+    value = world * ops / (ms_per_step * 1e-3) / 1e12
+    e2e_value = world * ops / (e2e_ms * 1e-3) / 1e12
+
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        kernel_ms = float(np.mean(step_ms))
+        achieved = step_bytes / (kernel_ms * 1e-3) / 1e9
+        line = {
+            "metric": "effective ternary TOPS (2MNK/s)", "value": value, "unit": "TOPS",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32 accumulate (int8 / 1-bit-plane operands), fp32 epilogue",
+            "data": "synthetic",
+            "config": {"workload": name, "variant": {1: "popc", 2: "i8"}[variant],
+                       "l2": f"{n_sets} rotating input/output sets ({n_sets * step_bytes >> 20} MiB) > L2",
+                       "thresholds": "t_lo = a_offset - 0.5, t_hi = a_offset + 0.5" if is_conv else
+                                     "per layer, as the workload names them",
+                       "weights": "packed before the timed region (offline step)",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": int(host_in.numel() * 4),
+                    "d2h_bytes_per_step": int(host_out.numel() * 4)},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                         "bytes_per_launch": int(step_bytes), "kernel_ms": kernel_ms},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            import oracle
+            rate, dt, sample = oracle_sample(case, 12.0)
+            line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TOPS", "cores": oracle.threads(),
+                                    "kind": "oracle", "sample": sample, "seconds": dt}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    case = WORKLOADS[args.workload]()
+    if args.impl == "reference":
+        run_reference(args, case, args.workload)
+    else:
+        run_ours(args, case, args.workload)
+
+
+if __name__ == "__main__":
+    main()
