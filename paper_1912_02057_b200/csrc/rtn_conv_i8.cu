@@ -1,28 +1,60 @@
 // Ternary conv2d (stride 1), tensor-core variant: fp32 NCHW input ternarized in-kernel (Eq. 3)
-// straight to int8 {-1,0,+1} in shared memory, filters expanded from their bit planes to int8 in
-// shared memory, tcgen05.mma kind::i8 into int32 accumulators in tensor memory, affine epilogue.
+// straight to int8 {-1,0,+1} in shared memory, filters expanded once per CTA from their bit
+// planes to int8 in shared memory, tcgen05.mma kind::i8 into int32 accumulators in tensor memory,
+// affine epilogue (Eq. 10 with a weight offset) fused.
 //
-// Implicit GEMM without im2col, by a shift: lay the zero-padded images of the batch out as one
-// long sequence of padded pixels, Q = (b*PH + r)*PW + c with PH = H + 2 pad, PW = W + 2 pad.  The
-// output whose top-left tap sits at padded pixel Q reads, for tap (i, j), padded pixel
-// Q + i*PW + j.  So for a tile of 128 consecutive Q the A operand of tap (i, j) is the SAME
-// shared-memory code array, read from a start address shifted by (i*PW + j) pixels.  Outputs whose
-// Q falls in the padding columns/rows (c >= Wo or r >= Ho) are computed and dropped.
+// Implicit GEMM without im2col, by a shift.  Lay the zero-padded images of the batch out as one
+// long sequence of padded rows G = b*PH + r (PH = H + 2 pad) of PW = W + 2 pad pixels each.  The
+// output whose top-left tap sits at padded pixel Q = G*PW + c reads, for tap (i, j), padded pixel
+// Q + i*PW + j.  For a run of consecutive Q the A operand of tap (i, j) is therefore the SAME
+// shared-memory code array read from a start address shifted by (i*PW + j) pixels.  Outputs whose
+// Q falls in the padding (c >= Wo or r >= Ho) are computed and dropped.
 //
-// Shared-memory code array: [channel chunk of 16][padded pixel][16 bytes] -- K-major without
-// swizzle, a core matrix (8 pixels x 16 channels) is 128 contiguous bytes wherever the window
-// starts.  Filters: [tap][channel chunk][n][16 bytes].  Within a group of 32 channels both
-// operands use the byte order of tc::unpack32.
+// Shared-memory code array: [channel chunk of 16][padded pixel][16 bytes] -- K-major, no swizzle:
+// an 8-pixel x 16-channel core matrix is 128 contiguous bytes wherever the window starts.
+// Filters: [tap][channel chunk][n][16 bytes].  Within a group of 32 channels both operands use
+// the byte order of tc::unpack32.  One extra filter row of all +1 makes the tensor core produce
+// the activation code sum S_x of every output pixel in accumulator column N.
+//
+// Work split: each CTA (one per SM, persistent) owns a contiguous strip of padded rows and walks
+// it in tiles of RT rows (RT*PW <= TM*128 accumulator lanes).  A tile needs RT + kh - 1 rows of
+// codes; the kh - 1 rows it shares with the previous tile are copied inside shared memory, so
+// every input value is fetched and ternarized once per strip.
+//
+// Warp roles, pipelined through mbarriers (two code buffers, two accumulator buffers, a ring of
+// input stages):
+//   warp  0       one thread issues the MMAs of tile i and commits them
+//   warp  1       producer: one thread streams the new fp32 rows of tile i+1.. into the stage ring
+//                 with TMA (one box = 16 channels x one image row), ahead of the converters
+//   warps 4..11   epilogue: tcgen05.ld the accumulators of tile i-1, affine form, store fp32
+//   warps 12..23  converters: read a stage, ternarize, write the code array of tile i
+// When the input cannot be described to TMA (W not a multiple of 4, unaligned base) the converters
+// load the fp32 values themselves.
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
+
+#include <cuda.h>
+#include <string.h>
 
 namespace rtn {
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kTileM = 128;                       // pixels per MMA (TMEM lanes)
-constexpr size_t kSmemLimit = 200 * 1024;
+constexpr int kMmaWarp = 0;
+constexpr int kProdWarp = 1;
+constexpr int kEpiWarp0 = 4;                           // first epilogue warp (multiple of 4)
+constexpr int kEpiWarps = 8;                           // two per TMEM lane quarter
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kConvWarp0 = kEpiWarp0 + kEpiWarps;
+constexpr int kConvWarps = 12;
+constexpr int kConvThreads = kConvWarps * 32;
+constexpr int kThreads = (kConvWarp0 + kConvWarps) * 32;
+constexpr int kMaxStages = 4;
+constexpr int kMaxMma = 160;                           // MMAs per sub-tile the descriptor table holds
+constexpr int kMaxSlots = 32;                          // row slots of a tile (rows + halo rows)
+constexpr int kTileM = 128;                            // pixels per MMA (TMEM lanes)
+constexpr size_t kSmemLimit = 220 * 1024;
+constexpr int kConvBarrier = 1;                        // named barrier of the converter warps
 
 // channel (within a group of 16) held by byte e of a 16-byte chunk: tc::unpack32's order
 // (0,4,8,12, 2,6,10,14, 1,5,9,13, 3,7,11,15)
@@ -31,87 +63,203 @@ __host__ __device__ constexpr int perm16(int e)
     return 4 * (e & 3) + ((e >> 2) == 0 ? 0 : (e >> 2) == 1 ? 2 : (e >> 2) == 2 ? 1 : 3);
 }
 
+// x / d for x*d < 2^32 (d >= 1): floor(x * ceil(2^32 / d) / 2^32)
+struct FastDiv {
+    uint32_t d, m;
+};
+inline FastDiv make_fastdiv(uint32_t d)
+{
+    FastDiv f;
+    f.d = d;
+    f.m = d <= 1 ? 0u : (uint32_t)(((uint64_t(1) << 32) + d - 1) / d);
+    return f;
+}
+__device__ __forceinline__ uint32_t fdiv(uint32_t x, FastDiv f) { return f.d <= 1 ? x : __umulhi(x, f.m); }
+
 struct ConvI8Plan {
     int PW, PH;            // padded image extent
-    int Cp, Np;            // channels rounded up to 32, output channels rounded up to 16
+    int Cp;                // channels rounded up to 32
+    int Np;                // accumulator columns: N outputs + the all-ones row, rounded up to 16
     int T;                 // taps
-    int TM;                // 128-pixel sub-tiles per CTA
-    int ppix;              // padded pixels held in shared memory per CTA
-    int64_t total_q;       // B*PH*PW
+    int TM;                // 128-pixel sub-tiles per tile
+    int RT;                // padded rows per tile
+    int halo;              // kh - 1 rows shared with the next tile
+    int ppix;              // pixels allocated per code buffer
+    int total_rows;        // B*PH
+    int grid;              // CTAs = strips
     uint32_t tmem_cols;
-    // byte offsets into dynamic shared memory
-    uint32_t off_a, off_w, off_psum, off_lo, off_hi, off_c1, off_c2, off_c3, off_bar, off_slot;
+    FastDiv div_pw, div_ph;
+    int n_mma;             // MMAs per sub-tile: taps * groups of 32 channels
+    int use_tma;           // input rows staged by TMA (else loaded by the converters)
+    int stages;            // depth of the staging ring
+    uint32_t box_bytes;    // one TMA box: 16 channels x one image row of fp32
+    uint32_t stage_bytes;
+    uint32_t off_stage;
+    uint32_t off_a[2], off_w, off_lo, off_hi, off_c, off_rows, off_bar, off_misc;
     size_t smem_bytes;
+    // Per MMA of a sub-tile (tap t, channel group h), in 16-byte units: start of the A window
+    // relative to the code buffer, start of the filter slice relative to the filter array.
+    uint32_t tab_a[kMaxMma], tab_b[kMaxMma];
 };
 
-inline uint32_t align_up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
-
-bool make_plan(const ConvArgs& c, ConvI8Plan& p)
+bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
 {
     if (c.stride != 1) return false;
     if (c.Ho <= 0 || c.Wo <= 0) return false;
     p.PW = c.W + 2 * c.pad;
     p.PH = c.H + 2 * c.pad;
+    if (p.PW > 256 || p.PH > 2048) return false;
     p.Cp = (c.C + 31) / 32 * 32;
-    p.Np = (c.N + 15) / 16 * 16;
+    p.Np = (c.N + 1 + 15) / 16 * 16;
     p.T = c.kh * c.kw;
+    p.halo = c.kh - 1;
     if (p.Np > 256) return false;
-    p.total_q = (int64_t)c.B * p.PH * p.PW;
-    const int64_t tiles1 = (p.total_q + kTileM - 1) / kTileM;
-    p.TM = (tiles1 >= 4 * 148 && 2 * p.Np <= 512) ? 2 : 1;
-    const int halo = (c.kh - 1) * p.PW + (c.kw - 1);
-    p.ppix = (p.TM * kTileM + halo + 7) / 8 * 8;
+    if ((int64_t)c.B * p.PH > (1 << 20)) return false;                // fast division ranges
+    p.total_rows = c.B * p.PH;
+    // two sub-tiles when the accumulators fit twice (double buffered) and there is enough work
+    p.TM = (4 * p.Np <= 512 && (int64_t)p.total_rows * p.PW >= (int64_t)4 * 148 * kTileM) ? 2 : 1;
+    if (2 * p.TM * p.Np > 512) return false;
+    p.RT = p.TM * kTileM / p.PW;
+    if (p.RT > kMaxSlots - p.halo) p.RT = kMaxSlots - p.halo;
+    if (p.RT < 1) return false;
+    p.ppix = (p.TM * kTileM + p.halo * p.PW + (c.kw - 1) + 7) / 8 * 8;
+    const int tiles = (p.total_rows + p.RT - 1) / p.RT;
+    p.grid = tiles < sms ? tiles : sms;
     uint32_t cols = 32;
-    while (cols < (uint32_t)(p.TM * p.Np)) cols *= 2;
+    while (cols < (uint32_t)(2 * p.TM * p.Np)) cols *= 2;
     p.tmem_cols = cols;
+    p.div_pw = make_fastdiv((uint32_t)p.PW);
+    p.div_ph = make_fastdiv((uint32_t)p.PH);
+    p.n_mma = p.T * (p.Cp / 32);
+    if (p.n_mma > kMaxMma) return false;
+    for (int i = 0; i < p.n_mma; ++i) {
+        const int t = i / (p.Cp / 32), h = i % (p.Cp / 32);
+        p.tab_a[i] = (uint32_t)(2 * h) * p.ppix + (uint32_t)((t / c.kw) * p.PW + (t % c.kw));
+        p.tab_b[i] = (uint32_t)((t * (p.Cp / 16) + 2 * h) * p.Np);
+    }
     uint32_t o = 0;
-    p.off_a = o;    o += (uint32_t)(p.Cp / 16) * p.ppix * 16;
+    const uint32_t a_bytes = (uint32_t)(p.Cp / 16) * p.ppix * 16;
+    p.off_a[0] = o; o += a_bytes;
+    p.off_a[1] = o; o += a_bytes;
     p.off_w = o;    o += (uint32_t)p.T * (p.Cp / 16) * p.Np * 16;
-    p.off_psum = o; o += (uint32_t)p.ppix * 4;
     p.off_lo = o;   o += (uint32_t)p.Cp * 4;
     p.off_hi = o;   o += (uint32_t)p.Cp * 4;
-    p.off_c1 = o;   o += (uint32_t)p.Np * 4;
-    p.off_c2 = o;   o += (uint32_t)p.Np * 4;
-    p.off_c3 = o;   o += (uint32_t)p.Np * 4;
-    o = align_up(o, 8);
-    p.off_bar = o;  o += 8;
-    p.off_slot = o; o += 8;
+    o = (o + 15) / 16 * 16;
+    p.off_c = o;    o += (uint32_t)p.Np * 16;           // float4 {c1, c2, c3, 0} per column
+    p.off_rows = o; o += kMaxSlots * 4;                 // producer's row table
+    p.off_bar = o;  o += (8 + 2 * kMaxStages) * 8;      // a_full[2] a_empty[2] acc_full[2] acc_empty[2] st_full[] st_empty[]
+    p.off_misc = o; o += 16;                            // tmem slot, dead flag
+    if (o > kSmemLimit) return false;
+    // staging ring for TMA: as many stages (2..4) as fit
+    p.use_tma = 0; p.stages = 0; p.off_stage = o;
+    p.box_bytes = 16u * (uint32_t)c.W * 4u;
+    p.stage_bytes = (uint32_t)(p.RT + p.halo) * p.box_bytes;
+    const bool tma_ok = (c.W % 4 == 0) && (reinterpret_cast<uintptr_t>(c.x) % 16 == 0);
+    if (tma_ok) {
+        const uint32_t base = (o + 127) / 128 * 128;
+        int ns = (int)((kSmemLimit - base) / p.stage_bytes);
+        if (ns > kMaxStages) ns = kMaxStages;
+        if (ns >= 2) {
+            p.use_tma = 1; p.stages = ns; p.off_stage = base;
+            o = base + (uint32_t)ns * p.stage_bytes;
+        }
+    }
     p.smem_bytes = o;
-    if (p.smem_bytes > kSmemLimit) return false;
-    // descriptor fields are 14 bits of 16-byte units
-    if ((uint32_t)p.ppix * 16 >= (1u << 18) || (uint32_t)p.Np * 16 >= (1u << 18)) return false;
-    const int64_t grid = (p.total_q + (int64_t)p.TM * kTileM - 1) / ((int64_t)p.TM * kTileM);
-    if (grid > 0x7fffffff) return false;
     return true;
 }
 
-__global__ void __launch_bounds__(kThreads)
-conv_i8_kernel(const ConvArgs a, const ConvI8Plan p)
+// Bounded wait that also gives up at once when another thread of the CTA has already timed out.
+__device__ __forceinline__ bool wait_or_die(uint64_t* bar, uint32_t parity, unsigned* status,
+                                            volatile int* dead)
+{
+    if (tc::mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < tc::kWaitPolls; ++i) {
+        if (tc::mbar_try_wait(bar, parity)) return true;
+        if (*dead) return false;
+        if (i > 32) __nanosleep(64);
+    }
+    *dead = 1;
+    atomicOr(status, kStatusWaitTimeout);
+    return false;
+}
+
+// TMA: one box {W, 1, 16, 1} of the fp32 tensor viewed as (W, H, C, B) -> shared memory
+// [16 channels][W]; completion is counted in bytes on `bar`.  Channels outside the tensor read as
+// zero.  No multicast.
+__device__ __forceinline__ void tma_load_row(uint32_t dst, const CUtensorMap* map, int r, int c0, int b,
+                                             uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(r), "r"(c0), "r"(b), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                 ::"r"(tc::smem_addr(bar)), "r"(bytes) : "memory");
+}
+
+// Issues NB MMAs whose descriptor low words are first gathered into registers: nothing but the
+// tcgen05.mma instructions then sits in the issue stream (loads left between MMAs would be
+// ordered after them by the asm's memory clobber and stall the single issuing thread).
+template <int NB>
+__device__ __forceinline__ void issue_mmas(const ConvI8Plan& p, int i0, uint32_t d, uint32_t a_tm,
+                                           uint32_t w16, uint64_t desc_hi, uint32_t idesc)
+{
+    uint32_t la[NB], lb[NB];
+    #pragma unroll
+    for (int j = 0; j < NB; ++j) { la[j] = a_tm + p.tab_a[i0 + j]; lb[j] = w16 + p.tab_b[i0 + j]; }
+    tc::mma_i8_ss(d, desc_hi | la[0], desc_hi | lb[0], idesc, i0 > 0);
+    #pragma unroll
+    for (int j = 1; j < NB; ++j) tc::mma_i8_ss_acc(d, desc_hi | la[j], desc_hi | lb[j], idesc);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __grid_constant__ CUtensorMap tmap)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    uint4* sA = reinterpret_cast<uint4*>(smem + p.off_a);        // [Cp/16][ppix]
     uint4* sW = reinterpret_cast<uint4*>(smem + p.off_w);        // [T][Cp/16][Np]
-    int* sPsum = reinterpret_cast<int*>(smem + p.off_psum);
     float* sLo = reinterpret_cast<float*>(smem + p.off_lo);
     float* sHi = reinterpret_cast<float*>(smem + p.off_hi);
-    float* sC1 = reinterpret_cast<float*>(smem + p.off_c1);
-    float* sC2 = reinterpret_cast<float*>(smem + p.off_c2);
-    float* sC3 = reinterpret_cast<float*>(smem + p.off_c3);
-    uint64_t* bar = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-    uint32_t* slot = reinterpret_cast<uint32_t*>(smem + p.off_slot);
+    float4* sC = reinterpret_cast<float4*>(smem + p.off_c);     // {c1, c2, c3, 0} per column
+    uint32_t* sRows = reinterpret_cast<uint32_t*>(smem + p.off_rows);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
+    uint64_t* a_full = bars;            // [2] converters -> MMA: code buffer written
+    uint64_t* a_empty = bars + 2;       // [2] MMA -> converters: MMAs that read the buffer are done
+    uint64_t* acc_full = bars + 4;      // [2] MMA -> epilogue: accumulators complete
+    uint64_t* acc_empty = bars + 6;     // [2] epilogue -> MMA: accumulators read out
+    uint64_t* st_full = bars + 8;                   // [stages] TMA -> converters: stage landed
+    uint64_t* st_empty = bars + 8 + kMaxStages;     // [stages] converters -> producer: stage read
+    uint32_t* slot = reinterpret_cast<uint32_t*>(smem + p.off_misc);
+    volatile int* dead = reinterpret_cast<volatile int*>(smem + p.off_misc + 8);
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t q0 = (int64_t)blockIdx.x * p.TM * kTileM;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nchunk = p.Cp / 16;
-    const int img = p.PH * p.PW;
+    // this CTA's strip of padded rows
+    const int s0 = (int)((int64_t)blockIdx.x * p.total_rows / p.grid);
+    const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
 
+    // ---------------------------------------------------------------- set-up (all threads)
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
-    if (tid == 0) {
-        tc::mbar_init(bar, 1);
+    if (threadIdx.x == 32) {
+        tc::mbar_init(&a_full[0], kConvThreads);
+        tc::mbar_init(&a_full[1], kConvThreads);
+        tc::mbar_init(&a_empty[0], 1);
+        tc::mbar_init(&a_empty[1], 1);
+        tc::mbar_init(&acc_full[0], 1);
+        tc::mbar_init(&acc_full[1], 1);
+        tc::mbar_init(&acc_empty[0], kEpiThreads);
+        tc::mbar_init(&acc_empty[1], kEpiThreads);
+        for (int i = 0; i < kMaxStages; ++i) {
+            tc::mbar_init(&st_full[i], 1);
+            tc::mbar_init(&st_empty[i], kConvThreads);
+        }
         tc::mbar_init_fence();
+        *dead = 0;
     }
-    for (int i = tid; i < p.ppix; i += kThreads) sPsum[i] = 0;
-    for (int c = tid; c < p.Cp; c += kThreads) {
+    for (int c = threadIdx.x; c < p.Cp; c += kThreads) {
         // channel padding: thresholds that code everything to 0
         sLo[c] = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
         sHi[c] = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
@@ -119,7 +267,7 @@ conv_i8_kernel(const ConvArgs a, const ConvI8Plan p)
     {   // per-output-channel constants in double, rounded once:
         //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
         const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
-        for (int n = tid; n < p.Np; n += kThreads) {
+        for (int n = threadIdx.x; n < p.Np; n += kThreads) {
             float c1 = 0.f, c2 = 0.f, c3 = 0.f;
             if (n < a.N) {
                 const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
@@ -128,51 +276,14 @@ conv_i8_kernel(const ConvArgs a, const ConvI8Plan p)
                 c2 = (float)(a_s * wo);
                 c3 = (float)(a_o * (ws * (double)a.w_sum[n] + (double)a.C * p.T * wo));
             }
-            sC1[n] = c1; sC2[n] = c2; sC3[n] = c3;
+            sC[n] = make_float4(c1, c2, c3, 0.f);
         }
     }
-    __syncthreads();
-
-    // ---- 1. ternarize the padded pixels this tile touches: item = (chunk of 16 channels, pixel)
-    for (int it = tid; it < nchunk * p.ppix; it += kThreads) {
-        const int ch = it / p.ppix, pp = it % p.ppix;
-        const int64_t Q = q0 + pp;
-        uint32_t w[4] = {0, 0, 0, 0};
-        if (Q < p.total_q) {
-            const int b = (int)(Q / img);
-            const int rem = (int)(Q % img);
-            const int r = rem / p.PW - a.pad, c = rem % p.PW - a.pad;
-            if (r >= 0 && r < a.H && c >= 0 && c < a.W) {
-                const float* src = a.x + (((int64_t)b * a.C) * a.H + r) * a.W + c;
-                const int64_t cs = (int64_t)a.H * a.W;
-                float v[16];
-                #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int cc = ch * 16 + perm16(e);
-                    v[e] = cc < a.C ? __ldg(src + cc * cs) : 0.0f;
-                }
-                #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int cc = ch * 16 + perm16(e);
-                    bool nz, pos;
-                    ternarize(v[e], sLo[cc], sHi[cc], nz, pos);
-                    const uint32_t byte = pos ? 0x01u : (nz ? 0xFFu : 0x00u);
-                    w[e >> 2] |= byte << (8 * (e & 3));
-                }
-                const int s = __dp4a((int)w[0], 0x01010101, __dp4a((int)w[1], 0x01010101,
-                              __dp4a((int)w[2], 0x01010101, __dp4a((int)w[3], 0x01010101, 0))));
-                if (s != 0) atomicAdd(&sPsum[pp], s);
-            }
-        }
-        sA[ch * p.ppix + pp] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-
-    // ---- 2. filters: bit planes -> int8, [tap][chunk][n]
-    {
+    {   // filters: bit planes -> int8, [tap][chunk][n]; row N is all +1, rows above it are 0
         const int cwords = p.Cp / 32;
         const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
         const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
-        for (int it = tid; it < p.T * cwords * p.Np; it += kThreads) {
+        for (int it = threadIdx.x; it < p.T * cwords * p.Np; it += kThreads) {
             const int n = it % p.Np;
             const int wd = it / p.Np;                    // word index in the row: t*cwords + cw
             uint32_t nz = 0, sg = 0;
@@ -180,6 +291,8 @@ conv_i8_kernel(const ConvArgs a, const ConvI8Plan p)
                 const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
                 nz = __ldg(blk + (wd & 3));
                 sg = __ldg(blk + 4 + (wd & 3));
+            } else if (n == a.N) {
+                nz = 0xFFFFFFFFu; sg = 0xFFFFFFFFu;
             }
             uint32_t o[8];
             tc::unpack32(nz, sg, o);
@@ -195,82 +308,268 @@ conv_i8_kernel(const ConvArgs a, const ConvI8Plan p)
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
 
-    // ---- 3. MMAs: for every sub-tile, tap and group of 32 channels
-    if (tid == 0) {
-        const uint32_t idesc = tc::idesc_i8(kTileM, (uint32_t)p.Np);
-        const uint32_t a_base = tc::smem_addr(sA), w_base = tc::smem_addr(sW);
-        const uint32_t a_lbo = (uint32_t)p.ppix * 16, w_lbo = (uint32_t)p.Np * 16;
-        for (int tm = 0; tm < p.TM; ++tm) {
-            bool acc = false;
-            for (int t = 0; t < p.T; ++t) {
-                const int shift = (t / a.kw) * p.PW + (t % a.kw);
-                for (int h = 0; h < p.Cp / 32; ++h) {
-                    const uint64_t ad = tc::smem_desc_kmajor(
-                        a_base + (uint32_t)(2 * h) * a_lbo + (uint32_t)(tm * kTileM + shift) * 16, a_lbo, 128);
-                    const uint64_t bd = tc::smem_desc_kmajor(
-                        w_base + (uint32_t)((t * nchunk + 2 * h) * p.Np) * 16, w_lbo, 128);
-                    tc::mma_i8_ss(tmem + (uint32_t)(tm * p.Np), ad, bd, idesc, acc);
-                    acc = true;
+    if (warp >= kConvWarp0) {
+        // ------------------------------------------------------------ converters
+        // consecutive lanes take consecutive padded pixels: conflict-free reads of a staged row,
+        // coalesced global loads on the direct path, conflict-free 16-byte stores of the codes
+        const int tid = threadIdx.x - kConvWarp0 * 32;
+        const int64_t cs = (int64_t)a.H * a.W;
+        uint32_t st_count = 0;                                 // stages consumed so far
+        int it = 0;
+        for (int g = s0; g < s1; g += p.RT, ++it) {
+            const int buf = it & 1;
+            uint4* sA = reinterpret_cast<uint4*>(smem + (buf ? p.off_a[1] : p.off_a[0]));      // [Cp/16][ppix]
+            const int nrows = min(p.RT, s1 - g);
+            const int slot0 = it == 0 ? 0 : p.halo;            // first row slot that is new
+            const int pp0 = slot0 * p.PW, pp1 = (nrows + p.halo) * p.PW;
+            wait_or_die(&a_empty[buf], ((it >> 1) & 1) ^ 1, a.status, dead);
+            if (it > 0) {
+                // the kh-1 rows shared with the previous tile: copy their codes (all converter
+                // threads must have finished writing the previous buffer first)
+                asm volatile("bar.sync %0, %1;" ::"r"(kConvBarrier), "r"(kConvThreads) : "memory");
+                const uint4* prev = reinterpret_cast<const uint4*>(smem + (buf ? p.off_a[0] : p.off_a[1]));
+                const int ncopy = p.halo * p.PW;
+                for (int i = tid; i < nchunk * ncopy; i += kConvThreads) {
+                    const int ch = i / ncopy, x = i - ch * ncopy;
+                    sA[ch * p.ppix + x] = prev[ch * p.ppix + p.RT * p.PW + x];
+                }
+            }
+            if (p.use_tma) {
+                for (int ch = 0; ch < nchunk; ++ch, ++st_count) {
+                    const uint32_t s = st_count % (uint32_t)p.stages;
+                    wait_or_die(&st_full[s], (st_count / (uint32_t)p.stages) & 1, a.status, dead);
+                    const float* stage = reinterpret_cast<const float*>(smem + p.off_stage + s * p.stage_bytes);
+                    for (int pp = pp0 + tid; pp < pp1; pp += kConvThreads) {
+                        // padded pixel -> (row slot, column) -> (image, row)
+                        const uint32_t sl = fdiv((uint32_t)pp, p.div_pw);
+                        const int c = (int)((uint32_t)pp - sl * (uint32_t)p.PW) - a.pad;
+                        const uint32_t G = (uint32_t)g + sl;
+                        const uint32_t b = fdiv(G, p.div_ph);
+                        const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
+                        uint32_t w[4] = {0, 0, 0, 0};
+                        if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
+                            const float* src = stage + ((sl - (uint32_t)slot0) * 16u) * (uint32_t)a.W + (uint32_t)c;
+                            float v[16];
+                            #pragma unroll
+                            for (int e = 0; e < 16; ++e) v[e] = src[perm16(e) * a.W];
+                            #pragma unroll
+                            for (int e = 0; e < 16; ++e) {
+                                const int cc = ch * 16 + perm16(e);
+                                bool nz, pos;
+                                ternarize(v[e], sLo[cc], sHi[cc], nz, pos);
+                                const uint32_t byte = pos ? 0x01u : (nz ? 0xFFu : 0x00u);
+                                w[e >> 2] |= byte << (8 * (e & 3));
+                            }
+                        }
+                        sA[ch * p.ppix + pp] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    tc::mbar_arrive(&st_empty[s]);
+                }
+            } else {
+                // direct path: item = (padded pixel, group of 32 channels), 32 loads in flight
+                const int ngroup = p.Cp / 32, npix = pp1 - pp0;
+                for (int i = tid; i < ngroup * npix; i += kConvThreads) {
+                    const int grp = i / npix, pp = pp0 + (i - grp * npix);
+                    const uint32_t sl = fdiv((uint32_t)pp, p.div_pw);
+                    const int c = (int)((uint32_t)pp - sl * (uint32_t)p.PW) - a.pad;
+                    const uint32_t G = (uint32_t)g + sl;
+                    const uint32_t b = fdiv(G, p.div_ph);
+                    const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
+                    uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                    if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
+                        const float* src = a.x + (((int64_t)b * a.C + grp * 32) * a.H + r) * a.W + c;
+                        float v[32];
+                        #pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            const int cc = (e >> 4) * 16 + perm16(e & 15);       // channel within the group
+                            v[e] = (grp * 32 + cc < a.C) ? __ldg(src + cc * cs) : 0.0f;
+                        }
+                        #pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            const int cc = grp * 32 + (e >> 4) * 16 + perm16(e & 15);
+                            bool nz, pos;
+                            ternarize(v[e], sLo[cc], sHi[cc], nz, pos);
+                            const uint32_t byte = pos ? 0x01u : (nz ? 0xFFu : 0x00u);
+                            w[e >> 2] |= byte << (8 * (e & 3));
+                        }
+                    }
+                    sA[(2 * grp) * p.ppix + pp] = make_uint4(w[0], w[1], w[2], w[3]);
+                    sA[(2 * grp + 1) * p.ppix + pp] = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+            }
+            tc::fence_smem_to_async_proxy();
+            tc::mbar_arrive(&a_full[buf]);
+        }
+    } else if (warp == kProdWarp) {
+        // ------------------------------------------------------------ producer
+        if (p.use_tma) {
+            uint32_t st_count = 0;
+            bool alive = true;
+            int it = 0;
+            for (int g = s0; g < s1 && alive; g += p.RT, ++it) {
+                const int nrows = min(p.RT, s1 - g);
+                const int slot0 = it == 0 ? 0 : p.halo;
+                const int nnew = nrows + p.halo - slot0;           // new row slots (<= 32)
+                // lane j looks at new slot j: which image row is it, if any
+                uint32_t info = 0xFFFFFFFFu;
+                if (lane < nnew) {
+                    const uint32_t G = (uint32_t)(g + slot0 + lane);
+                    const uint32_t b = fdiv(G, p.div_ph);
+                    const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
+                    if (b < (uint32_t)a.B && r >= 0 && r < a.H) info = (b << 11) | (uint32_t)r;
+                }
+                const uint32_t mask = __ballot_sync(0xffffffffu, info != 0xFFFFFFFFu);
+                __syncwarp();
+                sRows[lane] = info;
+                __syncwarp();
+                for (int ch = 0; ch < nchunk; ++ch, ++st_count) {
+                    const uint32_t s = st_count % (uint32_t)p.stages;
+                    const bool ok = wait_or_die(&st_empty[s], ((st_count / (uint32_t)p.stages) & 1) ^ 1, a.status, dead);
+                    if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+                    if (lane == 0) {
+                        if (mask == 0) {
+                            tc::mbar_arrive(&st_full[s]);
+                        } else {
+                            mbar_expect_tx(&st_full[s], (uint32_t)__popc(mask) * p.box_bytes);
+                            const uint32_t stage = tc::smem_addr(smem + p.off_stage + s * p.stage_bytes);
+                            const uint32_t bar = tc::smem_addr(&st_full[s]);
+                            uint32_t m = mask;
+                            while (m) {
+                                const int j = __ffs(m) - 1;
+                                m &= m - 1;
+                                const uint32_t inf = sRows[j];
+                                tma_load_row(stage + (uint32_t)j * p.box_bytes, &tmap, (int)(inf & 0x7FFu), ch * 16,
+                                             (int)(inf >> 11), bar);
+                            }
+                        }
+                    }
+                    __syncwarp();
                 }
             }
         }
-        tc::mma_commit(bar);
-    }
-    const bool alive = tc::mbar_wait(bar, 0, a.status);
-    tc::tc_fence_after_sync();
-
-    // ---- 4. epilogue: out = c1*S_xw + c2*S_x + c3
-    {
-        const int q = warp & 3, part = warp >> 2;
-        for (int tm = 0; tm < p.TM; ++tm) {
-            const int pl = tm * kTileM + q * 32 + lane;          // local padded pixel
-            const int64_t Q = q0 + pl;
-            const int b = (int)(Q / img);
-            const int rem = (int)(Q % img);
-            const int ho = rem / p.PW, wo = rem % p.PW;
-            const bool ok = alive && Q < p.total_q && ho < a.Ho && wo < a.Wo;
-            int s_x = 0;
-            int n_inside = p.T;
-            if (ok) {
-                for (int t = 0; t < p.T; ++t) s_x += sPsum[pl + (t / a.kw) * p.PW + (t % a.kw)];
-                if (a.pad_mode == RTN_PAD_VALUE_ZERO) {
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------ MMA issue (one thread)
+        if (lane == 0) {
+            const uint32_t idesc = tc::idesc_i8(kTileM, (uint32_t)p.Np);
+            // descriptor high word: 8-row group stride 128 bytes, sm_100 descriptor version, no swizzle
+            const uint64_t desc_hi = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
+            const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
+            const uint32_t w16 = (tc::smem_addr(sW) >> 4) + ((((uint32_t)p.Np * 16) >> 4) << 16);
+            int it = 0;
+            for (int g = s0; g < s1; g += p.RT, ++it) {
+                const int buf = it & 1;
+                const uint32_t ph = (it >> 1) & 1;
+                const int nrows = min(p.RT, s1 - g);
+                const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;          // sub-tiles with any row
+                const bool ok1 = wait_or_die(&a_full[buf], ph, a.status, dead);
+                const bool ok2 = wait_or_die(&acc_empty[buf], ph ^ 1, a.status, dead);
+                if (!(ok1 && ok2)) break;
+                tc::tc_fence_after_sync();
+                const uint32_t a16 = tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4;
+                for (int tm = 0; tm < ntm; ++tm) {
+                    const uint32_t d = tmem + (uint32_t)((buf * p.TM + tm) * p.Np);
+                    const uint32_t a_tm = a16 + (uint32_t)(tm * kTileM) + a_lbo_field;
+                    int i = 0;
+                    for (; i + 18 <= p.n_mma; i += 18) issue_mmas<18>(p, i, d, a_tm, w16, desc_hi, idesc);
+                    if (i + 8 <= p.n_mma) { issue_mmas<8>(p, i, d, a_tm, w16, desc_hi, idesc); i += 8; }
+                    if (i + 8 <= p.n_mma) { issue_mmas<8>(p, i, d, a_tm, w16, desc_hi, idesc); i += 8; }
+                    if (i + 4 <= p.n_mma) { issue_mmas<4>(p, i, d, a_tm, w16, desc_hi, idesc); i += 4; }
+                    if (i + 2 <= p.n_mma) { issue_mmas<2>(p, i, d, a_tm, w16, desc_hi, idesc); i += 2; }
+                    if (i + 1 <= p.n_mma) { issue_mmas<1>(p, i, d, a_tm, w16, desc_hi, idesc); i += 1; }
+                }
+                tc::mma_commit(&a_empty[buf]);
+                tc::mma_commit(&acc_full[buf]);
+            }
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ------------------------------------------------------------ epilogue (8 warps)
+        //   out = c1*S_xw + c2*S_x + c3.  Warp w reads TMEM lanes 32 (w mod 4)..+31 (pixels); the two
+        //   warps of a lane quarter split the 16-column blocks of the accumulator between them.
+        const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;      // kEpiWarp0 is a multiple of 4
+        const int64_t ostride = (int64_t)a.Ho * a.Wo;
+        const int nblk16 = (a.N + 15) / 16;
+        const int blk_begin = half == 0 ? 0 : (nblk16 + 1) / 2;
+        const int blk_end = half == 0 ? (nblk16 + 1) / 2 : nblk16;
+        int it = 0;
+        for (int g = s0; g < s1; g += p.RT, ++it) {
+            const int buf = it & 1;
+            const int nrows = min(p.RT, s1 - g);
+            const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
+            const bool alive = wait_or_die(&acc_full[buf], (it >> 1) & 1, a.status, dead);
+            tc::tc_fence_after_sync();
+            for (int tm = 0; tm < ntm; ++tm) {
+                const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);     // pixel within the tile
+                const uint32_t row = fdiv(pl, p.div_pw);
+                const int wo = (int)(pl - row * (uint32_t)p.PW);
+                const uint32_t G = (uint32_t)g + row;
+                const uint32_t b = fdiv(G, p.div_ph);
+                const int ho = (int)(G - b * (uint32_t)p.PH);
+                const bool ok = alive && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
+                int n_inside = p.T;
+                if (ok && a.pad_mode == RTN_PAD_VALUE_ZERO) {
                     n_inside = 0;
                     for (int t = 0; t < p.T; ++t) {
                         const int h = ho - a.pad + t / a.kw, v = wo - a.pad + t % a.kw;
                         n_inside += (h >= 0 && h < a.H && v >= 0 && v < a.W);
                     }
                 }
-            }
-            const bool border = n_inside < p.T;
-            const float fsx = (float)s_x;
-            const int64_t obase = (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
-            const int64_t ostride = (int64_t)a.Ho * a.Wo;
-            for (int c0 = part * 16; c0 < p.Np; c0 += 32) {
+                const bool border = n_inside < p.T;
+                const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + tm) * p.Np);
+                float* optr = a.out + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
+                int32_t* dptr = a.dbg_acc ? a.dbg_acc + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo : nullptr;
+                // S_x of this pixel: accumulator column N (the all-ones filter row)
+                uint32_t sx_raw;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
+                             : "=r"(sx_raw) : "r"(trow + (uint32_t)a.N) : "memory");
                 uint32_t v[16];
-                tc::tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(tm * p.Np + c0), v);
+                if (blk_begin < blk_end) tc::tmem_ld16(trow + (uint32_t)(blk_begin * 16), v);
                 tc::tmem_ld_wait();
-                if (!ok) continue;
-                #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int n = c0 + j;
-                    if (n >= a.N) break;
-                    const int s_xw = (int)v[j];
-                    float c3 = sC3[n];
-                    if (border) {
-                        // value-zero padding at an image border: S_w and K over inside taps only
-                        int s_w = 0;
-                        for (int t = 0; t < p.T; ++t) {
-                            const int h = ho - a.pad + t / a.kw, vv = wo - a.pad + t % a.kw;
-                            if (h >= 0 && h < a.H && vv >= 0 && vv < a.W) s_w += a.w_sum[(1 + t) * a.N + n];
+                const float fsx = (float)(int)sx_raw;
+                for (int blk = blk_begin; blk < blk_end; ++blk) {
+                    // take the block's values, then start the next block's load before the stores
+                    uint32_t u[16];
+                    #pragma unroll
+                    for (int j = 0; j < 16; ++j) u[j] = v[j];
+                    if (blk + 1 < blk_end) tc::tmem_ld16(trow + (uint32_t)((blk + 1) * 16), v);
+                    const int n0 = blk * 16;
+                    if (ok) {
+                        if (!border && dptr == nullptr && n0 + 16 <= a.N) {
+                            // fast path: a whole block, code-zero padding (or an interior pixel)
+                            #pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float4 c = sC[n0 + j];
+                                optr[(int64_t)(n0 + j) * ostride] = fmaf(c.x, (float)(int)u[j], fmaf(c.y, fsx, c.z));
+                            }
+                        } else {
+                            #pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const int n = n0 + j;
+                                if (n >= a.N) continue;
+                                const int s_xw = (int)u[j];
+                                const float4 c = sC[n];
+                                float c3 = c.z;
+                                if (border) {
+                                    // value-zero padding at an image border: S_w and K over inside taps only
+                                    int s_w = 0;
+                                    for (int t = 0; t < p.T; ++t) {
+                                        const int h = ho - a.pad + t / a.kw, vv = wo - a.pad + t % a.kw;
+                                        if (h >= 0 && h < a.H && vv >= 0 && vv < a.W) s_w += a.w_sum[(1 + t) * a.N + n];
+                                    }
+                                    const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
+                                    const double wo_ = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
+                                    c3 = (float)((double)a.ep.a_offset_val *
+                                                 (ws * (double)s_w + (double)a.C * n_inside * wo_));
+                                }
+                                optr[(int64_t)n * ostride] = fmaf(c.x, (float)s_xw, fmaf(c.y, fsx, c3));
+                                if (dptr != nullptr) dptr[(int64_t)n * ostride] = s_xw;
+                            }
                         }
-                        const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
-                        const double wo_ = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
-                        c3 = (float)((double)a.ep.a_offset_val * (ws * (double)s_w + (double)a.C * n_inside * wo_));
                     }
-                    a.out[obase + n * ostride] = fmaf(sC1[n], (float)s_xw, fmaf(sC2[n], fsx, c3));
-                    if (a.dbg_acc != nullptr) a.dbg_acc[obase + n * ostride] = s_xw;
+                    tc::tmem_ld_wait();
                 }
             }
+            tc::tc_fence_before_sync();
+            tc::mbar_arrive(&acc_empty[buf]);
         }
     }
     tc::tc_fence_before_sync();
@@ -278,23 +577,67 @@ conv_i8_kernel(const ConvArgs a, const ConvI8Plan p)
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
 }
 
+int sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
+    return sms;
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
 }  // namespace
 
 bool conv_i8_supported(const ConvArgs& c)
 {
     ConvI8Plan p;
-    return make_plan(c, p);
+    return make_plan(c, p, 148);
 }
 
 cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s)
 {
     ConvI8Plan p;
-    if (!make_plan(c, p)) return cudaErrorInvalidConfiguration;
+    if (!make_plan(c, p, sm_count())) return cudaErrorInvalidConfiguration;
+    CUtensorMap tmap;
+    memset(&tmap, 0, sizeof(tmap));
+    if (p.use_tma) {
+        EncodeTiledFn enc = encode_tiled_fn();
+        const cuuint64_t dims[4] = {(cuuint64_t)c.W, (cuuint64_t)c.H, (cuuint64_t)c.C, (cuuint64_t)c.B};
+        const cuuint64_t strides[3] = {(cuuint64_t)c.W * 4, (cuuint64_t)c.W * c.H * 4,
+                                       (cuuint64_t)c.W * c.H * c.C * 4};
+        const cuuint32_t box[4] = {(cuuint32_t)c.W, 1, 16, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc == nullptr ||
+            enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(c.x), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            // describing the input to TMA failed: let the converters load it themselves
+            p.use_tma = 0;
+            p.smem_bytes = p.off_stage;
+        }
+    }
     cudaError_t e = cudaFuncSetAttribute(conv_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
-    const int64_t grid = (p.total_q + (int64_t)p.TM * kTileM - 1) / ((int64_t)p.TM * kTileM);
-    conv_i8_kernel<<<(unsigned)grid, kThreads, p.smem_bytes, s>>>(c, p);
+    conv_i8_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(c, p, tmap);
     return cudaGetLastError();
 }
 
