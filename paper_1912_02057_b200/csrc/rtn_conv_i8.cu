@@ -176,7 +176,6 @@ __device__ __forceinline__ bool wait_or_die(uint64_t* bar, uint32_t parity, unsi
     for (uint32_t i = 0; i < tc::kWaitPolls; ++i) {
         if (tc::mbar_try_wait(bar, parity)) return true;
         if (*dead) return false;
-        if (i > 32) __nanosleep(64);
     }
     *dead = 1;
     atomicOr(status, kStatusWaitTimeout);

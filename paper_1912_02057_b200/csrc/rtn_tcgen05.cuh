@@ -28,28 +28,29 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+// One try: the hardware may park the thread for up to `suspend_ns` before answering, so a waiting
+// warp does not burn issue slots polling.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t suspend_ns = 2000)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(suspend_ns) : "memory");
     return ok != 0;
 }
 
-// Bounded wait for the phase of `parity` to complete.  Every poll that fails sleeps a little; after
-// kWaitPolls polls (about a second) the wait gives up, records it in the status word and returns
-// false, so a lost arrival can never hang the GPU.
-constexpr uint32_t kWaitPolls = 1u << 22;
+// Bounded wait for the phase of `parity` to complete.  After kWaitPolls tries (each parks the thread
+// for up to about 2 us: about a second in all) the wait gives up, records it in the status word and
+// returns false, so a lost arrival can never hang the GPU.
+constexpr uint32_t kWaitPolls = 1u << 19;
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned* status)
 {
     if (mbar_try_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < kWaitPolls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (i > 64) __nanosleep(128);
     }
     atomicOr(status, 2u);       // kStatusWaitTimeout
     return false;
