@@ -27,7 +27,7 @@
 //   warp  1       producer: one thread streams the new fp32 rows of tile i+1.. into the stage ring
 //                 with TMA (one box = 16 channels x one image row), ahead of the converters
 //   warps 4..11   epilogue: tcgen05.ld the accumulators of tile i-1, affine form, store fp32
-//   warps 12..23  converters: read a stage, ternarize, write the code array of tile i
+//   warps 2, 3, 12..17  converters: read a stage, ternarize, write the code array of tile i
 // When the input cannot be described to TMA (W not a multiple of 4, unaligned base) the converters
 // load the fp32 values themselves.
 #include "rtn_internal.cuh"
@@ -45,10 +45,12 @@ constexpr int kProdWarp = 1;
 constexpr int kEpiWarp0 = 4;                           // first epilogue warp (multiple of 4)
 constexpr int kEpiWarps = 8;                           // two per TMEM lane quarter
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kConvWarp0 = kEpiWarp0 + kEpiWarps;
-constexpr int kConvWarps = 12;
+constexpr int kConvWarps = 8;                          // warps 2, 3 and 12..17
 constexpr int kConvThreads = kConvWarps * 32;
-constexpr int kThreads = (kConvWarp0 + kConvWarps) * 32;
+constexpr int kWarps = kEpiWarp0 + kEpiWarps + kConvWarps - 2;
+constexpr int kThreads = kWarps * 32;
+__device__ __forceinline__ bool is_conv_warp(int w) { return w == 2 || w == 3 || w >= kEpiWarp0 + kEpiWarps; }
+__device__ __forceinline__ int conv_warp_index(int w) { return w < 4 ? w - 2 : w - (kEpiWarp0 + kEpiWarps) + 2; }
 constexpr int kMaxStages = 4;
 constexpr int kMaxMma = 160;                           // MMAs per sub-tile the descriptor table holds
 constexpr int kMaxSlots = 32;                          // row slots of a tile (rows + halo rows)
@@ -200,6 +202,32 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
                  ::"r"(tc::smem_addr(bar)), "r"(bytes) : "memory");
 }
 
+// Sixteen fp32 values -> sixteen int8 codes {-1,0,+1} in four words (byte e of the chunk = v[e]).
+// Branch-free: p = (v > hi), n = (v < lo) as 1.0f / 0.0f, then (1.5*2^23 + p) - n is a float whose
+// low mantissa byte is the two's-complement code; PRMT gathers the four low bytes of a word.  The
+// two comparisons never both hold: the set-up replaces t_lo by the float just above t_hi when
+// t_lo > t_hi, which keeps "+1 is tested first" (then -1 exactly when v <= t_hi).
+template <bool kPerLayer>
+__device__ __forceinline__ uint4 codes16(const float (&v)[16], const float* lo, const float* hi, int c0,
+                                         float lo0, float hi0)
+{
+    uint32_t t[16];
+    #pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        const float l = kPerLayer ? lo0 : lo[c0 + perm16(e)];
+        const float h = kPerLayer ? hi0 : hi[c0 + perm16(e)];
+        const float pos = v[e] > h ? 1.0f : 0.0f;
+        const float neg = v[e] < l ? 1.0f : 0.0f;
+        t[e] = __float_as_uint((12582912.0f + pos) - neg);
+    }
+    uint32_t w[4];
+    #pragma unroll
+    for (int k = 0; k < 4; ++k)
+        w[k] = __byte_perm(__byte_perm(t[4 * k], t[4 * k + 1], 0x0040),
+                           __byte_perm(t[4 * k + 2], t[4 * k + 3], 0x0040), 0x5410);
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // Issues NB MMAs whose descriptor low words are first gathered into registers: nothing but the
 // tcgen05.mma instructions then sits in the issue stream (loads left between MMAs would be
 // ordered after them by the asm's memory clobber and stall the single issuing thread).
@@ -260,8 +288,11 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     }
     for (int c = threadIdx.x; c < p.Cp; c += kThreads) {
         // channel padding: thresholds that code everything to 0
-        sLo[c] = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
-        sHi[c] = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
+        float lo = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
+        const float hi = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
+        if (lo > hi) lo = nextafterf(hi, INFINITY);      // v < lo  <=>  v <= hi: -1 unless +1
+        sLo[c] = lo;
+        sHi[c] = hi;
     }
     {   // per-output-channel constants in double, rounded once:
         //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
@@ -307,12 +338,14 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
 
-    if (warp >= kConvWarp0) {
+    if (is_conv_warp(warp)) {
         // ------------------------------------------------------------ converters
         // consecutive lanes take consecutive padded pixels: conflict-free reads of a staged row,
         // coalesced global loads on the direct path, conflict-free 16-byte stores of the codes
-        const int tid = threadIdx.x - kConvWarp0 * 32;
+        const int tid = conv_warp_index(warp) * 32 + lane;
         const int64_t cs = (int64_t)a.H * a.W;
+        const bool per_layer = a.n_thr == 1;
+        const float lo0 = sLo[0], hi0 = sHi[0];
         uint32_t st_count = 0;                                 // stages consumed so far
         int it = 0;
         for (int g = s0; g < s1; g += p.RT, ++it) {
@@ -345,55 +378,39 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                         const uint32_t G = (uint32_t)g + sl;
                         const uint32_t b = fdiv(G, p.div_ph);
                         const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
-                        uint32_t w[4] = {0, 0, 0, 0};
+                        uint4 w = make_uint4(0, 0, 0, 0);
                         if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
                             const float* src = stage + ((sl - (uint32_t)slot0) * 16u) * (uint32_t)a.W + (uint32_t)c;
                             float v[16];
                             #pragma unroll
                             for (int e = 0; e < 16; ++e) v[e] = src[perm16(e) * a.W];
-                            #pragma unroll
-                            for (int e = 0; e < 16; ++e) {
-                                const int cc = ch * 16 + perm16(e);
-                                bool nz, pos;
-                                ternarize(v[e], sLo[cc], sHi[cc], nz, pos);
-                                const uint32_t byte = pos ? 0x01u : (nz ? 0xFFu : 0x00u);
-                                w[e >> 2] |= byte << (8 * (e & 3));
-                            }
+                            w = per_layer ? codes16<true>(v, sLo, sHi, ch * 16, lo0, hi0)
+                                          : codes16<false>(v, sLo, sHi, ch * 16, lo0, hi0);
                         }
-                        sA[ch * p.ppix + pp] = make_uint4(w[0], w[1], w[2], w[3]);
+                        sA[ch * p.ppix + pp] = w;
                     }
                     tc::mbar_arrive(&st_empty[s]);
                 }
             } else {
-                // direct path: item = (padded pixel, group of 32 channels), 32 loads in flight
-                const int ngroup = p.Cp / 32, npix = pp1 - pp0;
-                for (int i = tid; i < ngroup * npix; i += kConvThreads) {
-                    const int grp = i / npix, pp = pp0 + (i - grp * npix);
+                // direct path: item = (padded pixel, chunk of 16 channels), 16 loads in flight
+                const int npix = pp1 - pp0;
+                for (int i = tid; i < nchunk * npix; i += kConvThreads) {
+                    const int ch = i / npix, pp = pp0 + (i - ch * npix);
                     const uint32_t sl = fdiv((uint32_t)pp, p.div_pw);
                     const int c = (int)((uint32_t)pp - sl * (uint32_t)p.PW) - a.pad;
                     const uint32_t G = (uint32_t)g + sl;
                     const uint32_t b = fdiv(G, p.div_ph);
                     const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
-                    uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                    uint4 w = make_uint4(0, 0, 0, 0);
                     if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
-                        const float* src = a.x + (((int64_t)b * a.C + grp * 32) * a.H + r) * a.W + c;
-                        float v[32];
+                        const float* src = a.x + (((int64_t)b * a.C + ch * 16) * a.H + r) * a.W + c;
+                        float v[16];
                         #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            const int cc = (e >> 4) * 16 + perm16(e & 15);       // channel within the group
-                            v[e] = (grp * 32 + cc < a.C) ? __ldg(src + cc * cs) : 0.0f;
-                        }
-                        #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            const int cc = grp * 32 + (e >> 4) * 16 + perm16(e & 15);
-                            bool nz, pos;
-                            ternarize(v[e], sLo[cc], sHi[cc], nz, pos);
-                            const uint32_t byte = pos ? 0x01u : (nz ? 0xFFu : 0x00u);
-                            w[e >> 2] |= byte << (8 * (e & 3));
-                        }
+                        for (int e = 0; e < 16; ++e)
+                            v[e] = (ch * 16 + perm16(e) < a.C) ? __ldg(src + perm16(e) * cs) : 0.0f;
+                        w = codes16<false>(v, sLo, sHi, ch * 16, lo0, hi0);
                     }
-                    sA[(2 * grp) * p.ppix + pp] = make_uint4(w[0], w[1], w[2], w[3]);
-                    sA[(2 * grp + 1) * p.ppix + pp] = make_uint4(w[4], w[5], w[6], w[7]);
+                    sA[ch * p.ppix + pp] = w;
                 }
             }
             tc::fence_smem_to_async_proxy();
@@ -480,7 +497,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 tc::mma_commit(&acc_full[buf]);
             }
         }
-    } else if (warp >= kEpiWarp0) {
+    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
         // ------------------------------------------------------------ epilogue (8 warps)
         //   out = c1*S_xw + c2*S_x + c3.  Warp w reads TMEM lanes 32 (w mod 4)..+31 (pixels); the two
         //   warps of a lane quarter split the 16-column blocks of the accumulator between them.
