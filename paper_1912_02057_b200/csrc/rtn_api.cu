@@ -211,7 +211,7 @@ rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, 
     c.B = (int)B; c.C = (int)C; c.H = (int)H; c.W = (int)W; c.N = (int)N; c.kh = (int)kh; c.kw = (int)kw;
     c.stride = (int)stride; c.pad = (int)pad;
     c.Ho = (int)rtn_conv_out_dim(H, kh, stride, pad); c.Wo = (int)rtn_conv_out_dim(W, kw, stride, pad);
-    return rtn::conv_i8_supported(c) ? RTN_VARIANT_I8 : RTN_VARIANT_POPC;
+    return rtn::conv_i8_any_supported(c) ? RTN_VARIANT_I8 : RTN_VARIANT_POPC;
 }
 
 rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
@@ -229,13 +229,13 @@ rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, i
     if (st != RTN_OK) return st;
     if (variant != RTN_VARIANT_AUTO && variant != RTN_VARIANT_POPC && variant != RTN_VARIANT_I8)
         return RTN_ERR_VALUE;
-    if (variant == RTN_VARIANT_AUTO) variant = rtn::conv_i8_supported(c) ? RTN_VARIANT_I8 : RTN_VARIANT_POPC;
-    if (variant == RTN_VARIANT_I8 && !rtn::conv_i8_supported(c)) return RTN_ERR_UNSUPPORTED;
+    if (variant == RTN_VARIANT_AUTO) variant = rtn::conv_i8_any_supported(c) ? RTN_VARIANT_I8 : RTN_VARIANT_POPC;
+    if (variant == RTN_VARIANT_I8 && !rtn::conv_i8_any_supported(c)) return RTN_ERR_UNSUPPORTED;
     if (variant == RTN_VARIANT_POPC && !rtn::conv_popc_supported(c)) return RTN_ERR_UNSUPPORTED;
     c.status = status_word();
     if (c.status == nullptr) return RTN_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const cudaError_t e = (variant == RTN_VARIANT_I8) ? rtn::launch_conv_i8(c, s)
+    const cudaError_t e = (variant == RTN_VARIANT_I8) ? rtn::launch_conv_i8_any(c, s)
                                                       : rtn::launch_conv_popc(c, s);
     return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
 }

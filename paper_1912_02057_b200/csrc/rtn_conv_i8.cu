@@ -32,6 +32,7 @@
 // load the fp32 values themselves.
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
+#include "rtn_conv_i8_common.cuh"
 
 #include <cuda.h>
 #include <string.h>
@@ -39,6 +40,8 @@
 namespace rtn {
 
 namespace {
+
+using namespace conv_detail;
 
 constexpr int kMmaWarp = 0;
 constexpr int kProdWarp = 1;
@@ -57,26 +60,6 @@ constexpr int kMaxSlots = 32;                          // row slots of a tile (r
 constexpr int kTileM = 128;                            // pixels per MMA (TMEM lanes)
 constexpr size_t kSmemLimit = 220 * 1024;
 constexpr int kConvBarrier = 1;                        // named barrier of the converter warps
-
-// channel (within a group of 16) held by byte e of a 16-byte chunk: tc::unpack32's order
-// (0,4,8,12, 2,6,10,14, 1,5,9,13, 3,7,11,15)
-__host__ __device__ constexpr int perm16(int e)
-{
-    return 4 * (e & 3) + ((e >> 2) == 0 ? 0 : (e >> 2) == 1 ? 2 : (e >> 2) == 2 ? 1 : 3);
-}
-
-// x / d for x*d < 2^32 (d >= 1): floor(x * ceil(2^32 / d) / 2^32)
-struct FastDiv {
-    uint32_t d, m;
-};
-inline FastDiv make_fastdiv(uint32_t d)
-{
-    FastDiv f;
-    f.d = d;
-    f.m = d <= 1 ? 0u : (uint32_t)(((uint64_t(1) << 32) + d - 1) / d);
-    return f;
-}
-__device__ __forceinline__ uint32_t fdiv(uint32_t x, FastDiv f) { return f.d <= 1 ? x : __umulhi(x, f.m); }
 
 struct ConvI8Plan {
     int PW, PH;            // padded image extent
@@ -170,20 +153,6 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     return true;
 }
 
-// Bounded wait that also gives up at once when another thread of the CTA has already timed out.
-__device__ __forceinline__ bool wait_or_die(uint64_t* bar, uint32_t parity, unsigned* status,
-                                            volatile int* dead)
-{
-    if (tc::mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < tc::kWaitPolls; ++i) {
-        if (tc::mbar_try_wait(bar, parity)) return true;
-        if (*dead) return false;
-    }
-    *dead = 1;
-    atomicOr(status, kStatusWaitTimeout);
-    return false;
-}
-
 // TMA: one box {W, 1, 16, 1} of the fp32 tensor viewed as (W, H, C, B) -> shared memory
 // [16 channels][W]; completion is counted in bytes on `bar`.  Channels outside the tensor read as
 // zero.  No multicast.
@@ -200,32 +169,6 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                  ::"r"(tc::smem_addr(bar)), "r"(bytes) : "memory");
-}
-
-// Sixteen fp32 values -> sixteen int8 codes {-1,0,+1} in four words (byte e of the chunk = v[e]).
-// Branch-free: p = (v > hi), n = (v < lo) as 1.0f / 0.0f, then (1.5*2^23 + p) - n is a float whose
-// low mantissa byte is the two's-complement code; PRMT gathers the four low bytes of a word.  The
-// two comparisons never both hold: the set-up replaces t_lo by the float just above t_hi when
-// t_lo > t_hi, which keeps "+1 is tested first" (then -1 exactly when v <= t_hi).
-template <bool kPerLayer>
-__device__ __forceinline__ uint4 codes16(const float (&v)[16], const float* lo, const float* hi, int c0,
-                                         float lo0, float hi0)
-{
-    uint32_t t[16];
-    #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-        const float l = kPerLayer ? lo0 : lo[c0 + perm16(e)];
-        const float h = kPerLayer ? hi0 : hi[c0 + perm16(e)];
-        const float pos = v[e] > h ? 1.0f : 0.0f;
-        const float neg = v[e] < l ? 1.0f : 0.0f;
-        t[e] = __float_as_uint((12582912.0f + pos) - neg);
-    }
-    uint32_t w[4];
-    #pragma unroll
-    for (int k = 0; k < 4; ++k)
-        w[k] = __byte_perm(__byte_perm(t[4 * k], t[4 * k + 1], 0x0040),
-                           __byte_perm(t[4 * k + 2], t[4 * k + 3], 0x0040), 0x5410);
-    return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // Issues NB MMAs whose descriptor low words are first gathered into registers: nothing but the

@@ -70,8 +70,15 @@ cudaError_t launch_conv_popc(const ConvArgs& c, cudaStream_t s);
 // Tensor-core (tcgen05 kind::i8) variants; *_supported say whether a shape can run there.
 bool gemm_i8_supported(int64_t M, int64_t N, int64_t K);
 cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s);
-bool conv_i8_supported(const ConvArgs& c);
+bool conv_i8_supported(const ConvArgs& c);       // filters resident in shared memory (stride 1)
 cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s);
+bool conv_i8s_supported(const ConvArgs& c);      // filters streamed (large layers, 1x1 of any stride)
+cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s);
+inline bool conv_i8_any_supported(const ConvArgs& c) { return conv_i8_supported(c) || conv_i8s_supported(c); }
+inline cudaError_t launch_conv_i8_any(const ConvArgs& c, cudaStream_t s)
+{
+    return conv_i8_supported(c) ? launch_conv_i8(c, s) : launch_conv_i8s(c, s);
+}
 
 // ----------------------------------------------------------------------------------------------
 // Device helpers
