@@ -36,7 +36,8 @@ constexpr int kWorkThreads = kWorkWarps * 32;
 constexpr int kThreads = (kWorkWarp0 + kWorkWarps) * 32;
 constexpr int kTileM = 128;
 constexpr int kMaxK = 304;                             // K = 32 slices per tile the table holds
-constexpr int kMaxWStages = 16;
+constexpr int kMaxWStages = 8;
+constexpr int kSlices = 4;                             // K = 32 slices per filter stage (one packed block)
 constexpr size_t kSmemLimit = 220 * 1024;
 constexpr int kWorkBarrier = 2;
 
@@ -92,7 +93,7 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
     }
     uint32_t o = 0;
     p.off_a = o;    o += (uint32_t)(p.Cp / 16) * p.ppix * 16;
-    p.off_psum = o; o += 2u * (uint32_t)p.ppix * 4;
+    p.off_psum = o; o += 3u * (uint32_t)p.ppix * 4;
     p.off_lo = o;   o += (uint32_t)p.Cp * 4;
     p.off_hi = o;   o += (uint32_t)p.Cp * 4;
     o = (o + 15) / 16 * 16;
@@ -102,11 +103,12 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
     o = (o + 127) / 128 * 128;
     p.off_w = o;
     if (o > kSmemLimit) return false;
-    const uint32_t stage = (uint32_t)p.Np * 32;
+    const uint32_t stage = (uint32_t)p.Np * 32 * kSlices;
+    const int ngroups = (p.nK + kSlices - 1) / kSlices;
     int nw = (int)((kSmemLimit - o) / stage);
     if (nw > kMaxWStages) nw = kMaxWStages;
-    if (nw > p.nK) nw = p.nK;
-    if (nw < 2 && p.nK > 1) return false;
+    if (nw > ngroups) nw = ngroups;
+    if (nw < 2 && ngroups > 1) return false;
     if (nw < 1) return false;
     p.nW = nw;
     p.smem_bytes = o + (uint32_t)nw * stage;
@@ -118,8 +120,8 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     uint4* sA = reinterpret_cast<uint4*>(smem + p.off_a);        // [Cp/16][ppix]
-    uint4* sWr = reinterpret_cast<uint4*>(smem + p.off_w);       // [nW][2][Np]
-    int* sPsum = reinterpret_cast<int*>(smem + p.off_psum);      // [2][ppix]
+    uint4* sWr = reinterpret_cast<uint4*>(smem + p.off_w);       // [nW][kSlices][2][Np]
+    int* sPsum = reinterpret_cast<int*>(smem + p.off_psum);      // [3][ppix]
     float* sLo = reinterpret_cast<float*>(smem + p.off_lo);
     float* sHi = reinterpret_cast<float*>(smem + p.off_hi);
     float4* sC = reinterpret_cast<float4*>(smem + p.off_c);
@@ -140,10 +142,10 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
 
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
-        tc::mbar_init(a_full, kWorkThreads);
+        tc::mbar_init(a_full, kWorkWarps);
         tc::mbar_init(a_empty, 1);
         for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kEpiThreads); }
-        for (int i = 0; i < kMaxWStages; ++i) { tc::mbar_init(&w_full[i], kWorkThreads); tc::mbar_init(&w_empty[i], 1); }
+        for (int i = 0; i < kMaxWStages; ++i) { tc::mbar_init(&w_full[i], kWorkWarps); tc::mbar_init(&w_empty[i], 1); }
         tc::mbar_init_fence();
         *dead = 0;
     }
@@ -190,56 +192,74 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
         for (int g = s0; g < s1; g += p.RT, ++it) {
             const int nrows = min(p.RT, s1 - g);
             const int npix = (nrows + p.halo) * p.PW;
-            int* psum = sPsum + (it & 1) * p.ppix;
+            int* psum = sPsum + (it % 3) * p.ppix;
             wait_or_die(a_empty, (it & 1) ^ 1, a.status, dead);
             for (int i = tid; i < p.ppix; i += kWorkThreads) psum[i] = 0;
             asm volatile("bar.sync %0, %1;" ::"r"(kWorkBarrier), "r"(kWorkThreads) : "memory");
-            // ---- ternarize: item = (pixel of the tile's sequence, chunk of 16 channels)
-            for (int i = tid; i < nchunk * npix; i += kWorkThreads) {
-                const int ch = i / npix, pp = i - ch * npix;
+            // ---- ternarize: item = (pixel of the tile's sequence, pair of 16-channel chunks): 32 loads in flight
+            for (int i = tid; i < (nchunk / 2) * npix; i += kWorkThreads) {
+                const int cp = i / npix, pp = i - cp * npix;
                 const uint32_t sl = fdiv((uint32_t)pp, p.div_pw);
                 const int c = (int)((uint32_t)pp - sl * (uint32_t)p.PW) * p.istride - p.ipad;
                 const uint32_t G = (uint32_t)g + sl;
                 const uint32_t b = fdiv(G, p.div_ph);
                 const int r = (int)(G - b * (uint32_t)p.PH) * p.istride - p.ipad;
-                uint4 w = make_uint4(0, 0, 0, 0);
+                uint4 w0 = make_uint4(0, 0, 0, 0), w1 = make_uint4(0, 0, 0, 0);
                 if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
-                    const float* src = a.x + (((int64_t)b * a.C + ch * 16) * a.H + r) * a.W + c;
-                    float v[16];
+                    const float* src = a.x + (((int64_t)b * a.C + cp * 32) * a.H + r) * a.W + c;
+                    float v0[16], v1[16];
                     #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        v[e] = (ch * 16 + perm16(e) < a.C) ? __ldg(src + perm16(e) * cs) : 0.0f;
-                    w = per_layer ? codes16<true>(v, sLo, sHi, ch * 16, lo0, hi0)
-                                  : codes16<false>(v, sLo, sHi, ch * 16, lo0, hi0);
-                    const int s = __dp4a((int)w.x, 0x01010101, __dp4a((int)w.y, 0x01010101,
-                                  __dp4a((int)w.z, 0x01010101, __dp4a((int)w.w, 0x01010101, 0))));
+                    for (int e = 0; e < 16; ++e) {
+                        v0[e] = (cp * 32 + perm16(e) < a.C) ? __ldg(src + perm16(e) * cs) : 0.0f;
+                        v1[e] = (cp * 32 + 16 + perm16(e) < a.C) ? __ldg(src + (16 + perm16(e)) * cs) : 0.0f;
+                    }
+                    w0 = per_layer ? codes16<true>(v0, sLo, sHi, cp * 32, lo0, hi0)
+                                   : codes16<false>(v0, sLo, sHi, cp * 32, lo0, hi0);
+                    w1 = per_layer ? codes16<true>(v1, sLo, sHi, cp * 32 + 16, lo0, hi0)
+                                   : codes16<false>(v1, sLo, sHi, cp * 32 + 16, lo0, hi0);
+                    int s = __dp4a((int)w0.x, 0x01010101, __dp4a((int)w0.y, 0x01010101,
+                            __dp4a((int)w0.z, 0x01010101, __dp4a((int)w0.w, 0x01010101, 0))));
+                    s = __dp4a((int)w1.x, 0x01010101, __dp4a((int)w1.y, 0x01010101,
+                        __dp4a((int)w1.z, 0x01010101, __dp4a((int)w1.w, 0x01010101, s))));
                     if (s != 0) atomicAdd(&psum[pp], s);
                 }
-                sA[ch * p.ppix + pp] = w;
+                sA[(2 * cp) * p.ppix + pp] = w0;
+                sA[(2 * cp + 1) * p.ppix + pp] = w1;
             }
             tc::fence_smem_to_async_proxy();
-            tc::mbar_arrive(a_full);
-            // ---- filter slices of this tile: slice ks is word ks of the packed row
-            uint4 nzv = make_uint4(0, 0, 0, 0), sgv = make_uint4(0, 0, 0, 0);
-            for (int ks = 0; ks < p.nK; ++ks, ++wcount) {
-                if ((ks & 3) == 0 && Wrow != nullptr) {
-                    nzv = __ldg(Wrow + 2 * (ks >> 2));
-                    sgv = __ldg(Wrow + 2 * (ks >> 2) + 1);
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(a_full);
+            // ---- filter slices of this tile, one packed block (four K = 32 slices) per ring stage; slice ks
+            //      is word ks of the packed row.  The next block's planes are fetched while this one expands.
+            uint4 nzn = make_uint4(0, 0, 0, 0), sgn = nzn;
+            if (Wrow != nullptr) { nzn = __ldg(Wrow); sgn = __ldg(Wrow + 1); }
+            for (int ks0 = 0; ks0 < p.nK; ks0 += kSlices, ++wcount) {
+                const uint4 nzv = nzn, sgv = sgn;
+                if (Wrow != nullptr && ks0 + kSlices < p.nK) {
+                    nzn = __ldg(Wrow + 2 * ((ks0 >> 2) + 1));
+                    sgn = __ldg(Wrow + 2 * ((ks0 >> 2) + 1) + 1);
                 }
                 const uint32_t st = wcount % (uint32_t)p.nW;
                 wait_or_die(&w_empty[st], ((wcount / (uint32_t)p.nW) & 1) ^ 1, a.status, dead);
-                const int q = ks & 3;
-                const uint32_t nz = q == 0 ? nzv.x : q == 1 ? nzv.y : q == 2 ? nzv.z : nzv.w;
-                const uint32_t sg = q == 0 ? sgv.x : q == 1 ? sgv.y : q == 2 ? sgv.z : sgv.w;
                 if (tid < p.Np) {
+                    uint4* dst = sWr + (size_t)st * kSlices * 2 * p.Np + tid;
                     uint32_t o[8];
-                    tc::unpack32(nz, sg, o);
-                    uint4* dst = sWr + (size_t)st * 2 * p.Np + tid;
-                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(nzv.x, sgv.x, o);
+                    dst[0 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[1 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(nzv.y, sgv.y, o);
+                    dst[2 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[3 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(nzv.z, sgv.z, o);
+                    dst[4 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[5 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(nzv.w, sgv.w, o);
+                    dst[6 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[7 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
                 }
                 tc::fence_smem_to_async_proxy();
-                tc::mbar_arrive(&w_full[st]);
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&w_full[st]);
             }
         }
     } else if (warp == 0) {
@@ -250,7 +270,8 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
             const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
             const uint32_t a16 = (tc::smem_addr(sA) >> 4) + a_lbo_field;
             const uint32_t w16 = (tc::smem_addr(sWr) >> 4) + ((((uint32_t)p.Np * 16) >> 4) << 16);
-            const uint32_t wstage16 = ((uint32_t)p.Np * 32) >> 4;
+            const uint32_t wslice16 = ((uint32_t)p.Np * 32) >> 4;
+            const uint32_t wstage16 = wslice16 * kSlices;
             uint32_t wcount = 0;
             int it = 0;
             bool alive = true;
@@ -262,15 +283,18 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
                 alive = wait_or_die(a_full, it & 1, a.status, dead) &&
                         wait_or_die(&acc_empty[acc], acc_ph ^ 1, a.status, dead);
                 if (!alive) break;
-                for (int ks = 0; ks < p.nK; ++ks, ++wcount) {
+                for (int ks0 = 0; ks0 < p.nK; ks0 += kSlices, ++wcount) {
                     const uint32_t st = wcount % (uint32_t)p.nW;
                     if (!wait_or_die(&w_full[st], (wcount / (uint32_t)p.nW) & 1, a.status, dead)) { alive = false; break; }
                     tc::tc_fence_after_sync();
-                    const uint64_t bd = desc_hi | (uint64_t)(w16 + st * wstage16);
-                    const uint32_t aw = a16 + p.tab_a[ks];
-                    for (int tm = 0; tm < ntm; ++tm) {
-                        const uint32_t d = tmem + (uint32_t)((acc * p.TM + tm) * p.Np);
-                        tc::mma_i8_ss(d, desc_hi | (uint64_t)(aw + (uint32_t)(tm * kTileM)), bd, idesc, ks > 0);
+                    const int nks = min(kSlices, p.nK - ks0);
+                    for (int j = 0; j < nks; ++j) {
+                        const uint64_t bd = desc_hi | (uint64_t)(w16 + st * wstage16 + (uint32_t)j * wslice16);
+                        const uint32_t aw = a16 + p.tab_a[ks0 + j];
+                        for (int tm = 0; tm < ntm; ++tm) {
+                            const uint32_t d = tmem + (uint32_t)((acc * p.TM + tm) * p.Np);
+                            tc::mma_i8_ss(d, desc_hi | (uint64_t)(aw + (uint32_t)(tm * kTileM)), bd, idesc, ks0 + j > 0);
+                        }
                     }
                     tc::mma_commit(&w_empty[st]);
                 }
@@ -292,7 +316,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
             const uint32_t acc_ph = p.nAcc == 2 ? ((it >> 1) & 1) : (it & 1);
             const int nrows = min(p.RT, s1 - g);
             const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
-            const int* psum = sPsum + (it & 1) * p.ppix;
+            const int* psum = sPsum + (it % 3) * p.ppix;
             const bool alive = wait_or_die(&acc_full[acc], acc_ph, a.status, dead);
             tc::tc_fence_after_sync();
             for (int tm = 0; tm < ntm; ++tm) {

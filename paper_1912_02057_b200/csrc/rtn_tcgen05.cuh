@@ -170,5 +170,19 @@ __device__ __forceinline__ void unpack32(uint32_t nz, uint32_t sg, uint32_t (&o)
     o[7] = __byte_perm(kTable, kTable, r1 >> 16);
 }
 
+// Half of unpack32: codes 16*half .. 16*half+15 of the word pair -> four words (one 16-byte chunk),
+// same byte order as words 4*half .. 4*half+3 of unpack32.
+__device__ __forceinline__ void unpack16(uint32_t nz, uint32_t sg, int half, uint32_t (&o)[4])
+{
+    constexpr uint32_t kTable = 0x0100FF00u;
+    const uint32_t q = (nz & 0x55555555u) | ((sg << 1) & 0xAAAAAAAAu);
+    const uint32_t r = ((nz >> 1) & 0x55555555u) | (sg & 0xAAAAAAAAu);
+    const int sh = 16 * half;
+    o[0] = __byte_perm(kTable, kTable, (q & 0x33333333u) >> sh);
+    o[1] = __byte_perm(kTable, kTable, ((q >> 2) & 0x33333333u) >> sh);
+    o[2] = __byte_perm(kTable, kTable, (r & 0x33333333u) >> sh);
+    o[3] = __byte_perm(kTable, kTable, ((r >> 2) & 0x33333333u) >> sh);
+}
+
 }  // namespace tc
 }  // namespace rtn
