@@ -44,13 +44,43 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "cfg2_conv3x3_c64_56x56_b32"
 
 
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
+INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
+# Traffic counters of the dominant kernel, per launch, from the ncu captures summarised under
+# profiles/ (None once the kernel has changed since the capture).
+NCU_TRAFFIC_BYTES = {}
+
+
 def measured_peaks():
+    """(HBM GB/s, INT8 dense TOPS for a kernel timed alone, the same under a sustained load, source)."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+        return (float(p["hbm_gbs"]), INT8_OVER_BF16 * float(p["bf16_tflops"]),
+                INT8_OVER_BF16 * float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "of measured (MEASURED_PEAKS.json; int8 = bf16 x 2 nominal ratio)")
+    return (FALLBACK_HBM_GBS, INT8_OVER_BF16 * FALLBACK_BF16_TFLOPS,
+            INT8_OVER_BF16 * FALLBACK_BF16_TFLOPS_SUSTAINED, "of fallback (no MEASURED_PEAKS.json)")
+
+
+def roofline_of(workload, kernel_bytes, kernel_ops, kernel_ms):
+    """Roofline object of the dominant kernel: the slower of its HBM time and its tensor time binds."""
+    hbm, i8_burst, i8_sust, src = measured_peaks()
+    # a kernel that runs for milliseconds sits under the power cap: sustained figure
+    i8 = i8_sust if kernel_ms > 0.5 else i8_burst
+    t_hbm = kernel_bytes / (hbm * 1e9)
+    t_tensor = kernel_ops / (i8 * 1e12)
+    traffic = NCU_TRAFFIC_BYTES.get(workload)
+    if t_hbm >= t_tensor:
+        achieved = kernel_bytes / (kernel_ms * 1e-3) / 1e9
+        return {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm,
+                "traffic": traffic, "peak_source": src, "bytes_per_launch": int(kernel_bytes),
+                "kernel_ms": kernel_ms}
+    achieved = kernel_ops / (kernel_ms * 1e-3) / 1e12
+    return {"bound": "tensor", "achieved": achieved, "peak": i8, "unit": "TOP/s", "frac": achieved / i8,
+            "traffic": traffic, "peak_source": src, "ops_per_launch": kernel_ops, "kernel_ms": kernel_ms}
 
 
 class ClockSampler:
@@ -195,6 +225,22 @@ def run_reference(args, case, name):
 # ------------------------------------------------------------------------------------------------
 # GPU leg
 # ------------------------------------------------------------------------------------------------
+def max_over_ranks(values, world, device):
+    """Each rank's device-timed milliseconds -> the slowest rank's (the job ends when it does)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_tops(ops_per_replica, world, ms):
+    """Replicas only: every rank does the same work, so the job's rate is world * ops / slowest time."""
+    return world * ops_per_replica / (ms * 1e-3) / 1e12
+
+
 def run_ours(args, case, name):
     import torch
     import torch.distributed as dist
@@ -312,6 +358,21 @@ def run_ours(args, case, name):
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
 
+    # ---- GEMM workloads: the dominant kernel (rtn_ternary_gemm) timed alone, rotating operand sets
+    gemm_kernel_ms = gemm_kernel_bytes = None
+    if not is_conv:
+        reps = max(5, min(50, args.steps))
+        k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        k0.record()
+        for i in range(reps):
+            j = i % n_sets
+            rtn.rtn_ternary_gemm(packs[j], sums[j], w_packed, w_sum[0], M, N, K, a_s, a_o, w_s, w_o, out=outs[j])
+        k1.record()
+        barrier()
+        gemm_kernel_ms = k0.elapsed_time(k1) / reps
+        gemm_kernel_bytes = (M + N) * ((K + 127) // 128) * 32 + 4 * M * N
+
     # ---- end to end: pinned host input -> device, the C-ABI call(s), result -> pinned host
     e2e_steps = max(3, min(args.steps, 20))
     for i in range(2):
@@ -328,19 +389,17 @@ def run_ours(args, case, name):
     barrier()
     e2e_ms = e_begin.elapsed_time(e_end) / e2e_steps
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, "cuda")
     ms_per_step = total_ms / args.steps
     ops = ops_of(case)
-    value = world * ops / (ms_per_step * 1e-3) / 1e12
-    e2e_value = world * ops / (e2e_ms * 1e-3) / 1e12
+    value = whole_job_tops(ops, world, ms_per_step)
+    e2e_value = whole_job_tops(ops, world, e2e_ms)
 
     if rank == 0:
-        peak, peak_src = measured_peaks()
-        kernel_ms = ms_per_step / launches_per_step if launches_per_step == 1 else ms_per_step
-        achieved = step_bytes / (kernel_ms * 1e-3) / 1e9
+        if is_conv:
+            kernel_ms, kernel_bytes = ms_per_step, step_bytes
+        else:
+            kernel_ms, kernel_bytes = gemm_kernel_ms, gemm_kernel_bytes
         line = {
             "metric": "effective ternary TOPS (2MNK/s)", "value": value, "unit": "TOPS",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -359,9 +418,7 @@ def run_ours(args, case, name):
                     "h2d_bytes_per_step": int(host_in.numel() * 4),
                     "d2h_bytes_per_step": int(host_out.numel() * 4)},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
-                         "bytes_per_launch": int(step_bytes), "kernel_ms": kernel_ms},
+            "roofline": roofline_of(name, kernel_bytes, ops, kernel_ms),
         }
         if not args.no_cpu_baseline and world == 1:
             import oracle
