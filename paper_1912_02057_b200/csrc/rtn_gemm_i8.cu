@@ -1,195 +1,325 @@
-// Packed ternary GEMM, tensor-core variant: the bit planes are expanded to int8 {-1,0,+1} in
-// shared memory and contracted with tcgen05.mma kind::i8 into int32 accumulators in tensor
-// memory; the affine epilogue reads them back with tcgen05.ld.
+// Packed ternary GEMM, tensor-core variant: the bit planes of both operands (Table 1; A1, A2, W1,
+// W2 of Eq. 9) are expanded to int8 {-1,0,+1} in shared memory and contracted with tcgen05.mma
+// kind::i8 into int32 accumulators in tensor memory; the affine epilogue (Eq. 10 with a weight
+// offset) reads them back with tcgen05.ld.
 //
-// One CTA (256 threads) owns a 128 x BN output tile.  Per packed block (128 codes of K):
-//   * thread t < 128 expands row t of the A tile, threads 128.. expand rows of the W tile
-//     (two 128-bit loads of the row's planes, PRMT table expansion, 16-byte shared stores),
-//   * after a CTA barrier one thread issues four K = 32 MMAs and commits them to the stage's
-//     mbarrier, which frees the stage for re-use kStages blocks later.
-// Operand tiles are K-major without swizzle: [k chunk of 16 bytes][row][16 bytes], so an
-// 8-row x 16-byte core matrix is 128 contiguous bytes, and consecutive threads (rows) store
-// consecutive 16-byte slots (no bank conflicts).
+// Persistent CTA per SM walking 128*TM x BN output tiles, warp-specialised and decoupled through
+// mbarriers (no CTA-wide barrier in the main loop):
+//   warps 12..19  expanders: per packed block (128 codes of K) each thread expands whole rows of
+//                 the A and W tiles (two 128-bit plane loads fetched two blocks ahead, PRMT table
+//                 expansion, 16-byte shared stores) into a ring of stages, then fences and arrives
+//   warp  0       one thread waits for a stage, issues its 4*TM MMAs (K = 32 each) and commits them
+//                 to the stage's "empty" barrier; after the last block it commits the accumulators
+//   warps 4..11   epilogue: tcgen05.ld, out = a_s (w_s S_xw + w_o S_x) + a_o (w_s S_w + K w_o)
+// Operand stages are K-major without swizzle: [16-byte k chunk][row][16 B]; an 8-row core matrix is
+// 128 contiguous bytes and consecutive threads (rows) store consecutive 16-byte slots.
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
+#include "rtn_conv_i8_common.cuh"
 
 namespace rtn {
 
 namespace {
 
-constexpr int kBM = 128;
-constexpr int kStages = 3;
-constexpr int kThreads = 256;
+using conv_detail::wait_or_die;
 
-template <int BN>
-struct GemmI8Smem {
-    // [stage][chunk 0..7][row][16 B]
-    uint4 a[kStages][8][kBM];
-    uint4 b[kStages][8][BN];
-    float p1[BN], p2[BN], p3[BN];       // per-column epilogue constants
-    uint64_t bar_free[kStages];
-    uint32_t tmem_base;
+constexpr int kEpiWarp0 = 4;
+constexpr int kEpiWarps = 8;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kExpWarp0 = kEpiWarp0 + kEpiWarps;
+constexpr int kExpWarps = 8;
+constexpr int kExpThreads = kExpWarps * 32;
+constexpr int kThreads = (kExpWarp0 + kExpWarps) * 32;
+constexpr int kMaxStages = 6;
+constexpr size_t kSmemLimit = 220 * 1024;
+constexpr int kEpiBarrier = 3;
+
+struct GemmI8Plan {
+    int TM;                 // 128-row sub-tiles per tile
+    int BN;                 // tile columns (multiple of 16, <= 256)
+    int nAcc;               // accumulator sets
+    int stages;
+    int rows;               // rows per stage: TM*128 + BN
+    int64_t tiles_m, tiles_n, tiles;
+    int grid;
+    uint32_t tmem_cols;
+    uint32_t stage_bytes, off_stage, off_c, off_bar, off_misc;
+    size_t smem_bytes;
 };
 
-template <int BN>
-__global__ void __launch_bounds__(kThreads)
-gemm_i8_kernel(const GemmArgs g)
+bool make_gemm_plan(int64_t M, int64_t N, int64_t K, GemmI8Plan& p, int sms)
 {
-    extern __shared__ __align__(128) uint8_t smem_raw[];
-    GemmI8Smem<BN>& sm = *reinterpret_cast<GemmI8Smem<BN>*>(smem_raw);
+    if (M < 1 || N < 1 || K < 1) return false;
+    p.BN = (int)((N >= 256) ? 256 : (N + 15) / 16 * 16);
+    p.TM = 2;
+    auto ntiles = [&](int tm, int bn) { return ((M + 128 * tm - 1) / (128 * tm)) * ((N + bn - 1) / bn); };
+    if (ntiles(p.TM, p.BN) < 2 * sms) p.TM = 1;
+    if (ntiles(p.TM, p.BN) < sms && p.BN > 128) p.BN = 128;
+    p.nAcc = (2 * p.TM * p.BN <= 512) ? 2 : 1;
+    p.tiles_m = (M + 128 * p.TM - 1) / (128 * p.TM);
+    p.tiles_n = (N + p.BN - 1) / p.BN;
+    p.tiles = p.tiles_m * p.tiles_n;
+    if (p.tiles > 0x7fffffff) return false;
+    p.grid = (int)(p.tiles < sms ? p.tiles : sms);
+    p.rows = p.TM * 128 + p.BN;
+    p.stage_bytes = (uint32_t)p.rows * 128;
+    uint32_t cols = 32;
+    while (cols < (uint32_t)(p.nAcc * p.TM * p.BN)) cols *= 2;
+    p.tmem_cols = cols;
+    uint32_t o = 0;
+    p.off_c = o;    o += (uint32_t)p.BN * 16;                  // float4 {p1, p2, p3, 0} per column
+    p.off_bar = o;  o += (4 + 2 * kMaxStages) * 8;             // acc_full[2] acc_empty[2] full[] empty[]
+    p.off_misc = o; o += 16;
+    o = (o + 127) / 128 * 128;
+    p.off_stage = o;
+    int ns = (int)((kSmemLimit - o) / p.stage_bytes);
+    if (ns > kMaxStages) ns = kMaxStages;
+    if (ns < 2) return false;
+    p.stages = ns;
+    p.smem_bytes = o + (uint32_t)ns * p.stage_bytes;
+    return true;
+}
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * kBM, n0 = (int64_t)blockIdx.y * BN;
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    float4* sC = reinterpret_cast<float4*>(smem + p.off_c);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
+    uint64_t* acc_full = bars;          // [2] MMA -> epilogue
+    uint64_t* acc_empty = bars + 2;     // [2] epilogue -> MMA
+    uint64_t* full = bars + 4;                      // [stages] expanders -> MMA
+    uint64_t* empty = bars + 4 + kMaxStages;        // [stages] MMA -> expanders
+    uint32_t* slot = reinterpret_cast<uint32_t*>(smem + p.off_misc);
+    volatile int* dead = reinterpret_cast<volatile int*>(smem + p.off_misc + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t nblk = (g.K + kBlockCodes - 1) / kBlockCodes;
-    constexpr int kRowsPerPass = kThreads;                 // rows expanded per pass over the threads
-    constexpr int kPasses = (kBM + BN) / kRowsPerPass;     // 1 (BN = 128) or ...
-    static_assert((kBM + BN) % kRowsPerPass == 0, "tile rows must fill the threads");
+    const int rowsA = p.TM * 128;
 
-    if (warp == 0) tc::tmem_alloc(&sm.tmem_base, BN);
-    if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) tc::mbar_init(&sm.bar_free[s], 1);
+    if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
+    if (threadIdx.x == 32) {
+        for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kEpiThreads); }
+        for (int i = 0; i < kMaxStages; ++i) { tc::mbar_init(&full[i], kExpWarps); tc::mbar_init(&empty[i], 1); }
         tc::mbar_init_fence();
-    }
-    // per-column constants, in double, rounded once:
-    //   p1 = w_s, p2 = w_o, p3 = w_s*S_w + K*w_o
-    for (int j = tid; j < BN; j += kThreads) {
-        const int64_t n = n0 + j;
-        float p1 = 0.f, p2 = 0.f, p3 = 0.f;
-        if (n < g.N) {
-            const double ws = g.ep.w_scale[g.ep.n_wparam == 1 ? 0 : n];
-            const double wo = g.ep.w_offset[g.ep.n_wparam == 1 ? 0 : n];
-            p1 = (float)ws; p2 = (float)wo;
-            p3 = (float)(ws * (double)g.w_sum[n] + (double)g.K * wo);
-        }
-        sm.p1[j] = p1; sm.p2[j] = p2; sm.p3[j] = p3;
+        *dead = 0;
     }
     tc::tc_fence_before_sync();
     __syncthreads();
     tc::tc_fence_after_sync();
-    const uint32_t tmem = sm.tmem_base;
+    const uint32_t tmem = *slot;
 
-    // rows this thread expands
-    const uint4* src[kPasses];
-    #pragma unroll
-    for (int p = 0; p < kPasses; ++p) {
-        const int r = tid + p * kRowsPerPass;              // 0..kBM-1: A rows, then W rows
-        const bool isA = r < kBM;
-        const int64_t grow = isA ? (m0 + r) : (n0 + r - kBM);
-        const bool ok = grow < (isA ? g.M : g.N);
-        src[p] = ok ? reinterpret_cast<const uint4*>((isA ? g.a_packed : g.w_packed) + grow * nblk * kBlockBytes)
-                    : nullptr;
-    }
-    uint4 nzv[kPasses], sgv[kPasses];
-    #pragma unroll
-    for (int p = 0; p < kPasses; ++p) {
-        nzv[p] = src[p] ? __ldg(src[p]) : make_uint4(0, 0, 0, 0);
-        sgv[p] = src[p] ? __ldg(src[p] + 1) : make_uint4(0, 0, 0, 0);
-    }
-
-    constexpr uint32_t kIdesc = tc::idesc_i8(kBM, BN);
-    bool alive = true;
-    for (int64_t kb = 0; kb < nblk; ++kb) {
-        const int s = (int)(kb % kStages);
-        if (kb >= kStages)
-            alive &= tc::mbar_wait(&sm.bar_free[s], (uint32_t)((kb / kStages - 1) & 1), g.status);
-        #pragma unroll
-        for (int p = 0; p < kPasses; ++p) {
-            const uint4 nz = nzv[p], sg = sgv[p];
-            if (kb + 1 < nblk && src[p]) {                 // prefetch the next block's planes
-                nzv[p] = __ldg(src[p] + 2 * (kb + 1));
-                sgv[p] = __ldg(src[p] + 2 * (kb + 1) + 1);
-            }
-            const int r = tid + p * kRowsPerPass;
-            uint4* dst = (r < kBM) ? &sm.a[s][0][r] : &sm.b[s][0][r - kBM];
-            const int stride = (r < kBM) ? kBM : BN;       // uint4 slots between k chunks
-            uint32_t o[8];
-            tc::unpack32(nz.x, sg.x, o);
-            dst[0 * stride] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[1 * stride] = make_uint4(o[4], o[5], o[6], o[7]);
-            tc::unpack32(nz.y, sg.y, o);
-            dst[2 * stride] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[3 * stride] = make_uint4(o[4], o[5], o[6], o[7]);
-            tc::unpack32(nz.z, sg.z, o);
-            dst[4 * stride] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[5 * stride] = make_uint4(o[4], o[5], o[6], o[7]);
-            tc::unpack32(nz.w, sg.w, o);
-            dst[6 * stride] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[7 * stride] = make_uint4(o[4], o[5], o[6], o[7]);
-        }
-        tc::fence_smem_to_async_proxy();
-        __syncthreads();
-        if (tid == 0) {
-            tc::tc_fence_after_sync();
-            const uint32_t a_base = tc::smem_addr(&sm.a[s][0][0]);
-            const uint32_t b_base = tc::smem_addr(&sm.b[s][0][0]);
+    if (warp >= kExpWarp0) {
+        // ------------------------------------------------------------ expanders
+        const int tid = threadIdx.x - kExpWarp0 * 32;
+        uint32_t count = 0;                                   // stages produced so far
+        for (int64_t tile = blockIdx.x; tile < p.tiles; tile += gridDim.x) {
+            const int64_t m0 = (tile / p.tiles_n) * rowsA, n0 = (tile % p.tiles_n) * p.BN;
+            // up to two rows per thread and stage: row r of the stage is A row m0 + r or W row n0 + r - rowsA
+            const uint4* src[2];
+            uint4* dst_off[2];
+            int stride[2];
             #pragma unroll
-            for (int j = 0; j < 4; ++j) {                  // K = 32 per MMA = two 16-byte chunks
-                const uint64_t ad = tc::smem_desc_kmajor(a_base + j * 2 * kBM * 16, kBM * 16, 128);
-                const uint64_t bd = tc::smem_desc_kmajor(b_base + j * 2 * BN * 16, BN * 16, 128);
-                tc::mma_i8_ss(tmem, ad, bd, kIdesc, kb > 0 || j > 0);
+            for (int k = 0; k < 2; ++k) {
+                const int r = tid + k * kExpThreads;
+                src[k] = nullptr; dst_off[k] = nullptr; stride[k] = 0;
+                if (r < p.rows) {
+                    const bool isA = r < rowsA;
+                    const int64_t grow = isA ? m0 + r : n0 + (r - rowsA);
+                    if (grow < (isA ? g.M : g.N))
+                        src[k] = reinterpret_cast<const uint4*>((isA ? g.a_packed : g.w_packed) + grow * nblk * kBlockBytes);
+                    // byte offset of this row's first chunk inside a stage
+                    dst_off[k] = reinterpret_cast<uint4*>((size_t)(isA ? r : rowsA * 8 + (r - rowsA)) * 16);
+                    stride[k] = isA ? rowsA : p.BN;
+                }
             }
-            tc::mma_commit(&sm.bar_free[s]);
-        }
-    }
-    // the last commit covers every MMA issued before it
-    {
-        const int64_t last = nblk - 1;
-        alive &= tc::mbar_wait(&sm.bar_free[last % kStages], (uint32_t)((last / kStages) & 1), g.status);
-    }
-    tc::tc_fence_after_sync();
-
-    // Epilogue.  Warp w reads TMEM lanes 32 (w mod 4) ..+31 (rows) and half of the columns.
-    //   out = a_s * (p1*S_xw + p2*S_x) + a_o * p3
-    {
-        const int q = warp & 3, half = warp >> 2;
-        const int64_t m = m0 + q * 32 + lane;
-        const bool row_ok = m < g.M;
-        float a_s = 0.f, a_o = 0.f, s_x = 0.f;
-        if (row_ok) {
-            a_s = g.ep.a_scale[g.ep.n_aparam == 1 ? 0 : m];
-            a_o = g.ep.a_offset[g.ep.n_aparam == 1 ? 0 : m];
-            s_x = (float)g.a_sum[m];
-        }
-        constexpr int kColsPerWarp = BN / 2;
-        #pragma unroll 1
-        for (int c0 = half * kColsPerWarp; c0 < (half + 1) * kColsPerWarp; c0 += 16) {
-            uint32_t v[16];
-            tc::tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-            tc::tmem_ld_wait();
-            if (row_ok && alive) {
+            // planes of the next two blocks, in registers
+            uint4 nz[2][2], sg[2][2];
+            #pragma unroll
+            for (int d = 0; d < 2; ++d)
                 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int64_t n = n0 + c0 + j;
-                    if (n < g.N) {
-                        const int s_xw = (int)v[j];
-                        const float u = fmaf(sm.p1[c0 + j], (float)s_xw, sm.p2[c0 + j] * s_x);
-                        g.out[m * g.N + n] = fmaf(a_s, u, a_o * sm.p3[c0 + j]);
-                        if (g.dbg_acc != nullptr) g.dbg_acc[m * g.N + n] = s_xw;
+                for (int k = 0; k < 2; ++k) {
+                    const bool ok = src[k] != nullptr && d < nblk;
+                    nz[d][k] = ok ? __ldg(src[k] + 2 * d) : make_uint4(0, 0, 0, 0);
+                    sg[d][k] = ok ? __ldg(src[k] + 2 * d + 1) : make_uint4(0, 0, 0, 0);
+                }
+            for (int64_t kb = 0; kb < nblk; ++kb, ++count) {
+                const uint32_t s = count % (uint32_t)p.stages;
+                uint4 cnz[2], csg[2];
+                #pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    cnz[k] = nz[0][k]; csg[k] = sg[0][k];
+                    nz[0][k] = nz[1][k]; sg[0][k] = sg[1][k];
+                    const bool ok = src[k] != nullptr && kb + 2 < nblk;
+                    nz[1][k] = ok ? __ldg(src[k] + 2 * (kb + 2)) : make_uint4(0, 0, 0, 0);
+                    sg[1][k] = ok ? __ldg(src[k] + 2 * (kb + 2) + 1) : make_uint4(0, 0, 0, 0);
+                }
+                wait_or_die(&empty[s], ((count / (uint32_t)p.stages) & 1) ^ 1, g.status, dead);
+                uint8_t* stage = smem + p.off_stage + s * p.stage_bytes;
+                #pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    if (stride[k] == 0) continue;
+                    uint4* dst = reinterpret_cast<uint4*>(stage + reinterpret_cast<size_t>(dst_off[k]));
+                    const int st = stride[k];
+                    uint32_t o[8];
+                    tc::unpack32(cnz[k].x, csg[k].x, o);
+                    dst[0 * st] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[1 * st] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(cnz[k].y, csg[k].y, o);
+                    dst[2 * st] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[3 * st] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(cnz[k].z, csg[k].z, o);
+                    dst[4 * st] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[5 * st] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(cnz[k].w, csg[k].w, o);
+                    dst[6 * st] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[7 * st] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+                tc::fence_smem_to_async_proxy();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&full[s]);
+            }
+        }
+    } else if (warp == 0) {
+        // ------------------------------------------------------------ MMA issue (one thread)
+        if (lane == 0) {
+            const uint32_t idesc = tc::idesc_i8(128, (uint32_t)p.BN);
+            const uint64_t desc_hi = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
+            const uint32_t a_lbo = (((uint32_t)rowsA * 16) >> 4) << 16, b_lbo = (((uint32_t)p.BN * 16) >> 4) << 16;
+            const uint32_t stage16 = tc::smem_addr(smem + p.off_stage) >> 4;
+            uint32_t count = 0, tc_ = 0;
+            bool alive = true;
+            for (int64_t tile = blockIdx.x; tile < p.tiles && alive; tile += gridDim.x, ++tc_) {
+                const int acc = p.nAcc == 2 ? (tc_ & 1) : 0;
+                const uint32_t acc_ph = p.nAcc == 2 ? ((tc_ >> 1) & 1) : (tc_ & 1);
+                alive = wait_or_die(&acc_empty[acc], acc_ph ^ 1, g.status, dead);
+                for (int64_t kb = 0; kb < nblk && alive; ++kb, ++count) {
+                    const uint32_t s = count % (uint32_t)p.stages;
+                    if (!wait_or_die(&full[s], (count / (uint32_t)p.stages) & 1, g.status, dead)) { alive = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint32_t a16 = stage16 + s * (p.stage_bytes >> 4) + a_lbo;
+                    const uint32_t b16 = stage16 + s * (p.stage_bytes >> 4) + (uint32_t)(rowsA * 8) + b_lbo;
+                    uint32_t la[8], lb[4];
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {                       // K = 32 per MMA = chunks 2j, 2j+1
+                        lb[j] = b16 + (uint32_t)(2 * j * p.BN);
+                        la[2 * j] = a16 + (uint32_t)(2 * j * rowsA);
+                        la[2 * j + 1] = la[2 * j] + 128;                // second 128-row sub-tile
+                    }
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        tc::mma_i8_ss(tmem + (uint32_t)(acc * p.TM * p.BN), desc_hi | la[2 * j], desc_hi | lb[j], idesc,
+                                      kb > 0 || j > 0);
+                        if (p.TM == 2)
+                            tc::mma_i8_ss(tmem + (uint32_t)((acc * p.TM + 1) * p.BN), desc_hi | la[2 * j + 1],
+                                          desc_hi | lb[j], idesc, kb > 0 || j > 0);
+                    }
+                    tc::mma_commit(&empty[s]);
+                }
+                if (alive) tc::mma_commit(&acc_full[acc]);
+            }
+        }
+    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
+        // ------------------------------------------------------------ epilogue
+        //   out = a_s * (p1*S_xw + p2*S_x) + a_o * p3,  p1 = w_s, p2 = w_o, p3 = w_s*S_w + K*w_o
+        const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
+        const int etid = threadIdx.x - kEpiWarp0 * 32;
+        uint32_t tc_ = 0;
+        for (int64_t tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++tc_) {
+            const int acc = p.nAcc == 2 ? (tc_ & 1) : 0;
+            const uint32_t acc_ph = p.nAcc == 2 ? ((tc_ >> 1) & 1) : (tc_ & 1);
+            const int64_t m0 = (tile / p.tiles_n) * rowsA, n0 = (tile % p.tiles_n) * p.BN;
+            // per-column constants of this tile, in double, rounded once (the previous tile's readers
+            // are past them: same warps, program order + barrier)
+            asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");
+            for (int j = etid; j < p.BN; j += kEpiThreads) {
+                const int64_t n = n0 + j;
+                float p1 = 0.f, p2 = 0.f, p3 = 0.f;
+                if (n < g.N) {
+                    const double ws = g.ep.w_scale[g.ep.n_wparam == 1 ? 0 : n];
+                    const double wo = g.ep.w_offset[g.ep.n_wparam == 1 ? 0 : n];
+                    p1 = (float)ws; p2 = (float)wo;
+                    p3 = (float)(ws * (double)g.w_sum[n] + (double)g.K * wo);
+                }
+                sC[j] = make_float4(p1, p2, p3, 0.f);
+            }
+            asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");
+            const bool alive = wait_or_die(&acc_full[acc], acc_ph, g.status, dead);
+            tc::tc_fence_after_sync();
+            const int cols_half = p.BN / 2;                       // BN is a multiple of 16; halves of >= 8
+            const int c_begin = half == 0 ? 0 : (cols_half + 15) / 16 * 16;
+            const int c_end = half == 0 ? ((cols_half + 15) / 16 * 16 < p.BN ? (cols_half + 15) / 16 * 16 : p.BN) : p.BN;
+            for (int tm = 0; tm < p.TM; ++tm) {
+                const int64_t m = m0 + tm * 128 + q * 32 + lane;
+                const bool row_ok = alive && m < g.M;
+                float a_s = 0.f, a_o = 0.f, s_x = 0.f;
+                if (row_ok) {
+                    a_s = g.ep.a_scale[g.ep.n_aparam == 1 ? 0 : m];
+                    a_o = g.ep.a_offset[g.ep.n_aparam == 1 ? 0 : m];
+                    s_x = (float)g.a_sum[m];
+                }
+                const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((acc * p.TM + tm) * p.BN);
+                for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+                    uint32_t v[16];
+                    tc::tmem_ld16(trow + (uint32_t)c0, v);
+                    tc::tmem_ld_wait();
+                    if (!row_ok) continue;
+                    float* orow = g.out + m * g.N + n0 + c0;
+                    if (n0 + c0 + 16 <= g.N && g.dbg_acc == nullptr && (((uintptr_t)orow) & 15) == 0) {
+                        #pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            float r[4];
+                            #pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float4 c = sC[c0 + j + e];
+                                r[e] = fmaf(a_s, fmaf(c.x, (float)(int)v[j + e], c.y * s_x), a_o * c.z);
+                            }
+                            *reinterpret_cast<float4*>(orow + j) = make_float4(r[0], r[1], r[2], r[3]);
+                        }
+                    } else {
+                        #pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (n0 + c0 + j >= g.N) continue;
+                            const float4 c = sC[c0 + j];
+                            const int s_xw = (int)v[j];
+                            orow[j] = fmaf(a_s, fmaf(c.x, (float)s_xw, c.y * s_x), a_o * c.z);
+                            if (g.dbg_acc != nullptr) g.dbg_acc[m * g.N + n0 + c0 + j] = s_xw;
+                        }
                     }
                 }
             }
+            tc::tc_fence_before_sync();
+            tc::mbar_arrive(&acc_empty[acc]);
         }
     }
     tc::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) tc::tmem_dealloc(tmem, BN);
+    if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
+}
+
+int sm_count_g()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
+    return sms;
 }
 
 }  // namespace
 
 bool gemm_i8_supported(int64_t M, int64_t N, int64_t K)
 {
-    return M >= 1 && N >= 1 && K >= 1 && (M + kBM - 1) / kBM <= 0x7fffffff && (N + 127) / 128 <= 65535;
+    GemmI8Plan p;
+    return make_gemm_plan(M, N, K, p, 148);
 }
 
 cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s)
 {
-    constexpr int BN = 128;
-    const size_t smem = sizeof(GemmI8Smem<BN>) + 128;
-    cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    GemmI8Plan p;
+    if (!make_gemm_plan(g.M, g.N, g.K, p, sm_count_g())) return cudaErrorInvalidConfiguration;
+    cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
-    dim3 grid((unsigned)((g.M + kBM - 1) / kBM), (unsigned)((g.N + BN - 1) / BN));
-    gemm_i8_kernel<BN><<<grid, kThreads, smem, s>>>(g);
+    gemm_i8_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(g, p);
     return cudaGetLastError();
 }
 
