@@ -25,7 +25,7 @@
 // input stages):
 //   warp  0       one thread issues the MMAs of tile i and commits them
 //   warp  1       producer: one thread streams the new fp32 rows of tile i+1.. into the stage ring
-//                 with TMA (one box = 16 channels x one image row), ahead of the converters
+//                 with TMA (one box = 32 channels x one image row), ahead of the converters
 //   warps 4..11   epilogue: tcgen05.ld the accumulators of tile i-1, affine form, store fp32
 //   warps 2, 3, 12..17  converters: read a stage, ternarize, write the code array of tile i
 // When the input cannot be described to TMA (W not a multiple of 4, unaligned base) the converters
@@ -55,6 +55,7 @@ constexpr int kThreads = kWarps * 32;
 __device__ __forceinline__ bool is_conv_warp(int w) { return w == 2 || w == 3 || w >= kEpiWarp0 + kEpiWarps; }
 __device__ __forceinline__ int conv_warp_index(int w) { return w < 4 ? w - 2 : w - (kEpiWarp0 + kEpiWarps) + 2; }
 constexpr int kMaxStages = 4;
+constexpr int kMaxGroups = 16;                          // groups of 32 input channels (C <= 512)
 constexpr int kMaxMma = 160;                           // MMAs per sub-tile the descriptor table holds
 constexpr int kMaxSlots = 32;                          // row slots of a tile (rows + halo rows)
 constexpr int kTileM = 128;                            // pixels per MMA (TMEM lanes)
@@ -77,7 +78,7 @@ struct ConvI8Plan {
     int n_mma;             // MMAs per sub-tile: taps * groups of 32 channels
     int use_tma;           // input rows staged by TMA (else loaded by the converters)
     int stages;            // depth of the staging ring
-    uint32_t box_bytes;    // one TMA box: 16 channels x one image row of fp32
+    uint32_t box_bytes;    // one TMA box: 32 channels x one image row of fp32
     uint32_t stage_bytes;
     uint32_t off_stage;
     uint32_t off_a[2], off_w, off_lo, off_hi, off_c, off_rows, off_bar, off_misc;
@@ -99,6 +100,7 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     p.T = c.kh * c.kw;
     p.halo = c.kh - 1;
     if (p.Np > 256) return false;
+    if (p.Cp / 32 > kMaxGroups) return false;
     if ((int64_t)c.B * p.PH > (1 << 20)) return false;                // fast division ranges
     p.total_rows = c.B * p.PH;
     // two sub-tiles when the accumulators fit twice (double buffered) and there is enough work
@@ -118,7 +120,7 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     p.n_mma = p.T * (p.Cp / 32);
     if (p.n_mma > kMaxMma) return false;
     for (int i = 0; i < p.n_mma; ++i) {
-        const int t = i / (p.Cp / 32), h = i % (p.Cp / 32);
+        const int h = i / p.T, t = i % p.T;              // channel group outer, tap inner
         p.tab_a[i] = (uint32_t)(2 * h) * p.ppix + (uint32_t)((t / c.kw) * p.PW + (t % c.kw));
         p.tab_b[i] = (uint32_t)((t * (p.Cp / 16) + 2 * h) * p.Np);
     }
@@ -132,12 +134,12 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     o = (o + 15) / 16 * 16;
     p.off_c = o;    o += (uint32_t)p.Np * 16;           // float4 {c1, c2, c3, 0} per column
     p.off_rows = o; o += kMaxSlots * 4;                 // producer's row table
-    p.off_bar = o;  o += (8 + 2 * kMaxStages) * 8;      // a_full[2] a_empty[2] acc_full[2] acc_empty[2] st_full[] st_empty[]
+    p.off_bar = o;  o += (6 + 2 * kMaxStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] st_full[] st_empty[] a_full[2][groups]
     p.off_misc = o; o += 16;                            // tmem slot, dead flag
     if (o > kSmemLimit) return false;
     // staging ring for TMA: as many stages (2..4) as fit
     p.use_tma = 0; p.stages = 0; p.off_stage = o;
-    p.box_bytes = 16u * (uint32_t)c.W * 4u;
+    p.box_bytes = 32u * (uint32_t)c.W * 4u;
     p.stage_bytes = (uint32_t)(p.RT + p.halo) * p.box_bytes;
     const bool tma_ok = (c.W % 4 == 0) && (reinterpret_cast<uintptr_t>(c.x) % 16 == 0);
     if (tma_ok) {
@@ -153,8 +155,8 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     return true;
 }
 
-// TMA: one box {W, 1, 16, 1} of the fp32 tensor viewed as (W, H, C, B) -> shared memory
-// [16 channels][W]; completion is counted in bytes on `bar`.  Channels outside the tensor read as
+// TMA: one box {W, 1, 32, 1} of the fp32 tensor viewed as (W, H, C, B) -> shared memory
+// [32 channels][W]; completion is counted in bytes on `bar`.  Channels outside the tensor read as
 // zero.  No multicast.
 __device__ __forceinline__ void tma_load_row(uint32_t dst, const CUtensorMap* map, int r, int c0, int b,
                                              uint32_t bar)
@@ -196,12 +198,12 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     float4* sC = reinterpret_cast<float4*>(smem + p.off_c);     // {c1, c2, c3, 0} per column
     uint32_t* sRows = reinterpret_cast<uint32_t*>(smem + p.off_rows);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-    uint64_t* a_full = bars;            // [2] converters -> MMA: code buffer written
-    uint64_t* a_empty = bars + 2;       // [2] MMA -> converters: MMAs that read the buffer are done
-    uint64_t* acc_full = bars + 4;      // [2] MMA -> epilogue: accumulators complete
-    uint64_t* acc_empty = bars + 6;     // [2] epilogue -> MMA: accumulators read out
-    uint64_t* st_full = bars + 8;                   // [stages] TMA -> converters: stage landed
-    uint64_t* st_empty = bars + 8 + kMaxStages;     // [stages] converters -> producer: stage read
+    uint64_t* a_empty = bars;           // [2] MMA -> converters: MMAs that read the buffer are done
+    uint64_t* acc_full = bars + 2;      // [2] MMA -> epilogue: accumulators complete
+    uint64_t* acc_empty = bars + 4;     // [2] epilogue -> MMA: accumulators read out
+    uint64_t* st_full = bars + 6;                   // [stages] TMA -> converters: stage landed
+    uint64_t* st_empty = bars + 6 + kMaxStages;     // [stages] converters -> producer: stage read
+    uint64_t* a_full = bars + 6 + 2 * kMaxStages;   // [2][kMaxGroups] converters -> MMA: 32 channels of codes written
     uint32_t* slot = reinterpret_cast<uint32_t*>(smem + p.off_misc);
     volatile int* dead = reinterpret_cast<volatile int*>(smem + p.off_misc + 8);
 
@@ -214,8 +216,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     // ---------------------------------------------------------------- set-up (all threads)
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
-        tc::mbar_init(&a_full[0], kConvThreads);
-        tc::mbar_init(&a_full[1], kConvThreads);
+        for (int i = 0; i < 2 * kMaxGroups; ++i) tc::mbar_init(&a_full[i], kConvThreads);
         tc::mbar_init(&a_empty[0], 1);
         tc::mbar_init(&a_empty[1], 1);
         tc::mbar_init(&acc_full[0], 1);
@@ -288,6 +289,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         const int tid = conv_warp_index(warp) * 32 + lane;
         const int64_t cs = (int64_t)a.H * a.W;
         const bool per_layer = a.n_thr == 1;
+        const int ngroup = p.Cp / 32;
         const float lo0 = sLo[0], hi0 = sHi[0];
         uint32_t st_count = 0;                                 // stages consumed so far
         int it = 0;
@@ -310,11 +312,16 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 }
             }
             if (p.use_tma) {
-                for (int ch = 0; ch < nchunk; ++ch, ++st_count) {
+                const int npix = pp1 - pp0;
+                for (int grp = 0; grp < ngroup; ++grp, ++st_count) {
                     const uint32_t s = st_count % (uint32_t)p.stages;
                     wait_or_die(&st_full[s], (st_count / (uint32_t)p.stages) & 1, a.status, dead);
                     const float* stage = reinterpret_cast<const float*>(smem + p.off_stage + s * p.stage_bytes);
-                    for (int pp = pp0 + tid; pp < pp1; pp += kConvThreads) {
+                    // item = (padded pixel, half of the group's 32 channels)
+                    for (int i = tid; i < 2 * npix; i += kConvThreads) {
+                        const int hf = i >= npix ? 1 : 0;
+                        const int pp = pp0 + i - hf * npix;
+                        const int ch = 2 * grp + hf;
                         // padded pixel -> (row slot, column) -> (image, row)
                         const uint32_t sl = fdiv((uint32_t)pp, p.div_pw);
                         const int c = (int)((uint32_t)pp - sl * (uint32_t)p.PW) - a.pad;
@@ -323,7 +330,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                         const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
                         uint4 w = make_uint4(0, 0, 0, 0);
                         if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
-                            const float* src = stage + ((sl - (uint32_t)slot0) * 16u) * (uint32_t)a.W + (uint32_t)c;
+                            const float* src = stage + ((sl - (uint32_t)slot0) * 32u + 16u * hf) * (uint32_t)a.W + (uint32_t)c;
                             float v[16];
                             #pragma unroll
                             for (int e = 0; e < 16; ++e) v[e] = src[perm16(e) * a.W];
@@ -333,6 +340,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                         sA[ch * p.ppix + pp] = w;
                     }
                     tc::mbar_arrive(&st_empty[s]);
+                    tc::fence_smem_to_async_proxy();
+                    tc::mbar_arrive(&a_full[buf * kMaxGroups + grp]);
                 }
             } else {
                 // direct path: item = (padded pixel, chunk of 16 channels), 16 loads in flight
@@ -356,8 +365,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     sA[ch * p.ppix + pp] = w;
                 }
             }
-            tc::fence_smem_to_async_proxy();
-            tc::mbar_arrive(&a_full[buf]);
+            if (!p.use_tma) {
+                tc::fence_smem_to_async_proxy();
+                for (int grp = 0; grp < ngroup; ++grp) tc::mbar_arrive(&a_full[buf * kMaxGroups + grp]);
+            }
         }
     } else if (warp == kProdWarp) {
         // ------------------------------------------------------------ producer
@@ -381,7 +392,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 __syncwarp();
                 sRows[lane] = info;
                 __syncwarp();
-                for (int ch = 0; ch < nchunk; ++ch, ++st_count) {
+                for (int grp = 0; grp < p.Cp / 32; ++grp, ++st_count) {
                     const uint32_t s = st_count % (uint32_t)p.stages;
                     const bool ok = wait_or_die(&st_empty[s], ((st_count / (uint32_t)p.stages) & 1) ^ 1, a.status, dead);
                     if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
@@ -397,7 +408,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                                 const int j = __ffs(m) - 1;
                                 m &= m - 1;
                                 const uint32_t inf = sRows[j];
-                                tma_load_row(stage + (uint32_t)j * p.box_bytes, &tmap, (int)(inf & 0x7FFu), ch * 16,
+                                tma_load_row(stage + (uint32_t)j * p.box_bytes, &tmap, (int)(inf & 0x7FFu), grp * 32,
                                              (int)(inf >> 11), bar);
                             }
                         }
@@ -420,22 +431,27 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 const uint32_t ph = (it >> 1) & 1;
                 const int nrows = min(p.RT, s1 - g);
                 const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;          // sub-tiles with any row
-                const bool ok1 = wait_or_die(&a_full[buf], ph, a.status, dead);
-                const bool ok2 = wait_or_die(&acc_empty[buf], ph ^ 1, a.status, dead);
-                if (!(ok1 && ok2)) break;
-                tc::tc_fence_after_sync();
+                if (!wait_or_die(&acc_empty[buf], ph ^ 1, a.status, dead)) break;
                 const uint32_t a16 = tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4;
-                for (int tm = 0; tm < ntm; ++tm) {
-                    const uint32_t d = tmem + (uint32_t)((buf * p.TM + tm) * p.Np);
-                    const uint32_t a_tm = a16 + (uint32_t)(tm * kTileM) + a_lbo_field;
-                    int i = 0;
-                    for (; i + 18 <= p.n_mma; i += 18) issue_mmas<18>(p, i, d, a_tm, w16, desc_hi, idesc);
-                    if (i + 8 <= p.n_mma) { issue_mmas<8>(p, i, d, a_tm, w16, desc_hi, idesc); i += 8; }
-                    if (i + 8 <= p.n_mma) { issue_mmas<8>(p, i, d, a_tm, w16, desc_hi, idesc); i += 8; }
-                    if (i + 4 <= p.n_mma) { issue_mmas<4>(p, i, d, a_tm, w16, desc_hi, idesc); i += 4; }
-                    if (i + 2 <= p.n_mma) { issue_mmas<2>(p, i, d, a_tm, w16, desc_hi, idesc); i += 2; }
-                    if (i + 1 <= p.n_mma) { issue_mmas<1>(p, i, d, a_tm, w16, desc_hi, idesc); i += 1; }
+                bool alive = true;
+                // channel group by channel group, as the converters finish them
+                for (int grp = 0; grp < p.Cp / 32 && alive; ++grp) {
+                    alive = wait_or_die(&a_full[buf * kMaxGroups + grp], ph, a.status, dead);
+                    if (!alive) break;
+                    tc::tc_fence_after_sync();
+                    for (int tm = 0; tm < ntm; ++tm) {
+                        const uint32_t d = tmem + (uint32_t)((buf * p.TM + tm) * p.Np);
+                        const uint32_t a_tm = a16 + (uint32_t)(tm * kTileM) + a_lbo_field;
+                        int i = grp * p.T;
+                        const int i_end = i + p.T;
+                        for (; i + 9 <= i_end; i += 9) issue_mmas<9>(p, i, d, a_tm, w16, desc_hi, idesc);
+                        if (i + 8 <= i_end) { issue_mmas<8>(p, i, d, a_tm, w16, desc_hi, idesc); i += 8; }
+                        if (i + 4 <= i_end) { issue_mmas<4>(p, i, d, a_tm, w16, desc_hi, idesc); i += 4; }
+                        if (i + 2 <= i_end) { issue_mmas<2>(p, i, d, a_tm, w16, desc_hi, idesc); i += 2; }
+                        if (i + 1 <= i_end) { issue_mmas<1>(p, i, d, a_tm, w16, desc_hi, idesc); i += 1; }
+                    }
                 }
+                if (!alive) break;
                 tc::mma_commit(&a_empty[buf]);
                 tc::mma_commit(&acc_full[buf]);
             }
@@ -582,7 +598,7 @@ cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s)
         const cuuint64_t dims[4] = {(cuuint64_t)c.W, (cuuint64_t)c.H, (cuuint64_t)c.C, (cuuint64_t)c.B};
         const cuuint64_t strides[3] = {(cuuint64_t)c.W * 4, (cuuint64_t)c.W * c.H * 4,
                                        (cuuint64_t)c.W * c.H * c.C * 4};
-        const cuuint32_t box[4] = {(cuuint32_t)c.W, 1, 16, 1};
+        const cuuint32_t box[4] = {(cuuint32_t)c.W, 1, 32, 1};
         const cuuint32_t estr[4] = {1, 1, 1, 1};
         if (enc == nullptr ||
             enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(c.x), dims, strides, box, estr,
