@@ -200,6 +200,26 @@ def test_conv_config3_sampled(p_zero, variant):
     run_or_skip_unsupported(lambda: conv_parity_sampled(b, variant, oracle.PAD_CODE_ZERO, 5000, seed=3), variant)
 
 
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_conv_thresholds_out_of_order(variant):
+    # t_lo > t_hi on some channels: "+1 is tested first" still decides (Eq. 3 lists the +1 case first)
+    case = inputs.conv_case("conv_lo_gt_hi", 2, 64, 12, 12, 48, 3, 1, 1, seed=77, p_zero=0.4,
+                            thresholds=(0.3, 1.0), per_channel_thresholds=True)
+    case.t_lo[::3] = 1.2          # above t_hi (about 1.0) on every third channel
+    case.x[0, 0, 0, :4] = case.t_hi[0]      # ties with t_hi on such a channel: not > t_hi, but < t_lo -> -1
+    codes = run_or_skip_unsupported(lambda: conv_parity(case, variant), variant)
+    assert (codes[:, 0] == 0).sum() == 0    # a channel with t_lo > t_hi has no zero codes
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("shape", [(256, 512, 4096), (384, 272, 1152), (130, 520, 260)], ids=lambda s: "x".join(map(str, s)))
+def test_gemm_multi_tile_shapes(shape, variant):
+    M, N, K = shape
+    case = inputs.gemm_case(f"gemm_{M}x{N}x{K}", M, N, K, seed=M + K, p_zero=0.3, act="uniform3",
+                            thresholds=(-0.5, 0.5), per_row_act_params=True)
+    run_or_skip_unsupported(lambda: gemm_parity(case, variant), variant)
+
+
 def test_conv_variants_agree_bit_for_bit():
     case = inputs.config2(batch=2, thresholds=(0.3, 1.0))
     a1, o1, _, _ = conv_through_abi(case, rtn.VARIANT_POPC, oracle.PAD_CODE_ZERO)
