@@ -61,6 +61,7 @@ constexpr int kMaxSlots = 32;                          // row slots of a tile (r
 constexpr int kTileM = 128;                            // pixels per MMA (TMEM lanes)
 constexpr size_t kSmemLimit = 220 * 1024;
 constexpr int kConvBarrier = 1;                        // named barrier of the converter warps
+constexpr int kEpiBarrier = 2;                         // named barrier of the epilogue warps
 
 struct ConvI8Plan {
     int PW, PH;            // padded image extent
@@ -153,6 +154,15 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     }
     p.smem_bytes = o;
     return true;
+}
+
+// One warp of a role waits on the mbarrier; the role's other warps sleep on a hardware named
+// barrier until it gets there (a polling warp costs issue slots, a warp parked on bar.sync none).
+__device__ __forceinline__ void role_wait(bool leader, uint64_t* bar, uint32_t parity, unsigned* status,
+                                          volatile int* dead, int barrier_id, int nthreads)
+{
+    if (leader) wait_or_die(bar, parity, status, dead);
+    asm volatile("bar.sync %0, %1;" ::"r"(barrier_id), "r"(nthreads) : "memory");
 }
 
 // TMA: one box {W, 1, 32, 1} of the fp32 tensor viewed as (W, H, C, B) -> shared memory
@@ -257,23 +267,24 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         const int cwords = p.Cp / 32;
         const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
         const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
-        for (int it = threadIdx.x; it < p.T * cwords * p.Np; it += kThreads) {
-            const int n = it % p.Np;
-            const int wd = it / p.Np;                    // word index in the row: t*cwords + cw
-            uint32_t nz = 0, sg = 0;
-            if (n < a.N) {
-                const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
-                nz = __ldg(blk + (wd & 3));
-                sg = __ldg(blk + 4 + (wd & 3));
-            } else if (n == a.N) {
-                nz = 0xFFFFFFFFu; sg = 0xFFFFFFFFu;
-            }
-            uint32_t o[8];
-            tc::unpack32(nz, sg, o);
+        // a warp takes one 32-channel word of every filter row at a time (no per-item divisions)
+        for (int wd = warp; wd < p.T * cwords; wd += kWarps) {
             const int t = wd / cwords, cw = wd % cwords;
-            uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Np + n);
-            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+            for (int n = lane; n < p.Np; n += 32) {
+                uint32_t nz = 0, sg = 0;
+                if (n < a.N) {
+                    const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
+                    nz = __ldg(blk + (wd & 3));
+                    sg = __ldg(blk + 4 + (wd & 3));
+                } else if (n == a.N) {
+                    nz = 0xFFFFFFFFu; sg = 0xFFFFFFFFu;
+                }
+                uint32_t o[8];
+                tc::unpack32(nz, sg, o);
+                uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Np + n);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
         }
     }
     tc::fence_smem_to_async_proxy();
@@ -299,11 +310,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             const int nrows = min(p.RT, s1 - g);
             const int slot0 = it == 0 ? 0 : p.halo;            // first row slot that is new
             const int pp0 = slot0 * p.PW, pp1 = (nrows + p.halo) * p.PW;
-            wait_or_die(&a_empty[buf], ((it >> 1) & 1) ^ 1, a.status, dead);
+            // (the barrier inside also orders this tile after every converter's writes to the previous buffer)
+            role_wait(tid < 32, &a_empty[buf], ((it >> 1) & 1) ^ 1, a.status, dead, kConvBarrier, kConvThreads);
             if (it > 0) {
-                // the kh-1 rows shared with the previous tile: copy their codes (all converter
-                // threads must have finished writing the previous buffer first)
-                asm volatile("bar.sync %0, %1;" ::"r"(kConvBarrier), "r"(kConvThreads) : "memory");
+                // the kh-1 rows shared with the previous tile: copy their codes
                 const uint4* prev = reinterpret_cast<const uint4*>(smem + (buf ? p.off_a[0] : p.off_a[1]));
                 const int ncopy = p.halo * p.PW;
                 for (int i = tid; i < nchunk * ncopy; i += kConvThreads) {
@@ -315,7 +325,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 const int npix = pp1 - pp0;
                 for (int grp = 0; grp < ngroup; ++grp, ++st_count) {
                     const uint32_t s = st_count % (uint32_t)p.stages;
-                    wait_or_die(&st_full[s], (st_count / (uint32_t)p.stages) & 1, a.status, dead);
+                    role_wait(tid < 32, &st_full[s], (st_count / (uint32_t)p.stages) & 1, a.status, dead,
+                              kConvBarrier, kConvThreads);
                     const float* stage = reinterpret_cast<const float*>(smem + p.off_stage + s * p.stage_bytes);
                     // item = (padded pixel, half of the group's 32 channels)
                     for (int i = tid; i < 2 * npix; i += kConvThreads) {
@@ -470,7 +481,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             const int buf = it & 1;
             const int nrows = min(p.RT, s1 - g);
             const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
-            const bool alive = wait_or_die(&acc_full[buf], (it >> 1) & 1, a.status, dead);
+            role_wait(warp == kEpiWarp0, &acc_full[buf], (it >> 1) & 1, a.status, dead, kEpiBarrier, kEpiThreads);
+            const bool alive = !*dead;
             tc::tc_fence_after_sync();
             for (int tm = 0; tm < ntm; ++tm) {
                 const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);     // pixel within the tile
