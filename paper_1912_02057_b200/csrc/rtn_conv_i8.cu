@@ -135,7 +135,7 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     o = (o + 15) / 16 * 16;
     p.off_c = o;    o += (uint32_t)p.Np * 16;           // float4 {c1, c2, c3, 0} per column
     p.off_rows = o; o += kMaxSlots * 4;                 // producer's row table
-    p.off_bar = o;  o += (6 + 2 * kMaxStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] st_full[] st_empty[] a_full[2][groups]
+    p.off_bar = o;  o += (7 + 2 * kMaxStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] st_full[] st_empty[] a_full[2][groups]
     p.off_misc = o; o += 16;                            // tmem slot, dead flag
     if (o > kSmemLimit) return false;
     // staging ring for TMA: as many stages (2..4) as fit
@@ -214,6 +214,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     uint64_t* st_full = bars + 6;                   // [stages] TMA -> converters: stage landed
     uint64_t* st_empty = bars + 6 + kMaxStages;     // [stages] converters -> producer: stage read
     uint64_t* a_full = bars + 6 + 2 * kMaxStages;   // [2][kMaxGroups] converters -> MMA: 32 channels of codes written
+    uint64_t* w_ready = bars + 6 + 2 * kMaxStages + 2 * kMaxGroups;     // epilogue warps -> MMA: filters expanded
     uint32_t* slot = reinterpret_cast<uint32_t*>(smem + p.off_misc);
     volatile int* dead = reinterpret_cast<volatile int*>(smem + p.off_misc + 8);
 
@@ -227,6 +228,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
         for (int i = 0; i < 2 * kMaxGroups; ++i) tc::mbar_init(&a_full[i], kConvThreads);
+        tc::mbar_init(w_ready, kEpiThreads);
         tc::mbar_init(&a_empty[0], 1);
         tc::mbar_init(&a_empty[1], 1);
         tc::mbar_init(&acc_full[0], 1);
@@ -240,54 +242,6 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         tc::mbar_init_fence();
         *dead = 0;
     }
-    for (int c = threadIdx.x; c < p.Cp; c += kThreads) {
-        // channel padding: thresholds that code everything to 0
-        float lo = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
-        const float hi = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
-        if (lo > hi) lo = nextafterf(hi, INFINITY);      // v < lo  <=>  v <= hi: -1 unless +1
-        sLo[c] = lo;
-        sHi[c] = hi;
-    }
-    {   // per-output-channel constants in double, rounded once:
-        //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
-        const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
-        for (int n = threadIdx.x; n < p.Np; n += kThreads) {
-            float c1 = 0.f, c2 = 0.f, c3 = 0.f;
-            if (n < a.N) {
-                const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
-                const double wo = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
-                c1 = (float)(a_s * ws);
-                c2 = (float)(a_s * wo);
-                c3 = (float)(a_o * (ws * (double)a.w_sum[n] + (double)a.C * p.T * wo));
-            }
-            sC[n] = make_float4(c1, c2, c3, 0.f);
-        }
-    }
-    {   // filters: bit planes -> int8, [tap][chunk][n]; row N is all +1, rows above it are 0
-        const int cwords = p.Cp / 32;
-        const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
-        const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
-        // a warp takes one 32-channel word of every filter row at a time (no per-item divisions)
-        for (int wd = warp; wd < p.T * cwords; wd += kWarps) {
-            const int t = wd / cwords, cw = wd % cwords;
-            for (int n = lane; n < p.Np; n += 32) {
-                uint32_t nz = 0, sg = 0;
-                if (n < a.N) {
-                    const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
-                    nz = __ldg(blk + (wd & 3));
-                    sg = __ldg(blk + 4 + (wd & 3));
-                } else if (n == a.N) {
-                    nz = 0xFFFFFFFFu; sg = 0xFFFFFFFFu;
-                }
-                uint32_t o[8];
-                tc::unpack32(nz, sg, o);
-                uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Np + n);
-                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
-            }
-        }
-    }
-    tc::fence_smem_to_async_proxy();
     tc::tc_fence_before_sync();
     __syncthreads();
     tc::tc_fence_after_sync();
@@ -298,6 +252,16 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         // consecutive lanes take consecutive padded pixels: conflict-free reads of a staged row,
         // coalesced global loads on the direct path, conflict-free 16-byte stores of the codes
         const int tid = conv_warp_index(warp) * 32 + lane;
+        // thresholds (their global-load latency overlaps the first TMA loads, already in flight)
+        for (int c = tid; c < p.Cp; c += kConvThreads) {
+            // channel padding: thresholds that code everything to 0
+            float lo = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
+            const float hi = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
+            if (lo > hi) lo = nextafterf(hi, INFINITY);      // v < lo  <=>  v <= hi: -1 unless +1
+            sLo[c] = lo;
+            sHi[c] = hi;
+        }
+        asm volatile("bar.sync %0, %1;" ::"r"(kConvBarrier), "r"(kConvThreads) : "memory");
         const int64_t cs = (int64_t)a.H * a.W;
         const bool per_layer = a.n_thr == 1;
         const int ngroup = p.Cp / 32;
@@ -437,7 +401,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
             const uint32_t w16 = (tc::smem_addr(sW) >> 4) + ((((uint32_t)p.Np * 16) >> 4) << 16);
             int it = 0;
-            for (int g = s0; g < s1; g += p.RT, ++it) {
+            bool filters_ok = wait_or_die(w_ready, 0, a.status, dead);
+            for (int g = s0; g < s1 && filters_ok; g += p.RT, ++it) {
                 const int buf = it & 1;
                 const uint32_t ph = (it >> 1) & 1;
                 const int nrows = min(p.RT, s1 - g);
@@ -471,6 +436,51 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         // ------------------------------------------------------------ epilogue (8 warps)
         //   out = c1*S_xw + c2*S_x + c3.  Warp w reads TMEM lanes 32 (w mod 4)..+31 (pixels); the two
         //   warps of a lane quarter split the 16-column blocks of the accumulator between them.
+        // While the first input rows are in flight these warps, idle until the first accumulators are
+        // complete, expand the filters and work out the epilogue constants.
+        const int etid = threadIdx.x - kEpiWarp0 * 32;
+        {   // per-output-channel constants in double, rounded once:
+            //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
+            const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
+            for (int n = etid; n < p.Np; n += kEpiThreads) {
+                float c1 = 0.f, c2 = 0.f, c3 = 0.f;
+                if (n < a.N) {
+                    const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
+                    const double wo = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
+                    c1 = (float)(a_s * ws);
+                    c2 = (float)(a_s * wo);
+                    c3 = (float)(a_o * (ws * (double)a.w_sum[n] + (double)a.C * p.T * wo));
+                }
+                sC[n] = make_float4(c1, c2, c3, 0.f);
+            }
+        }
+        {   // filters: bit planes -> int8, [tap][chunk][n]; row N is all +1, rows above it are 0
+            const int cwords = p.Cp / 32;
+            const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
+            const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
+            // a warp takes one 32-channel word of every filter row at a time (no per-item divisions)
+            for (int wd = warp - kEpiWarp0; wd < p.T * cwords; wd += kEpiWarps) {
+                const int t = wd / cwords, cw = wd % cwords;
+                for (int n = lane; n < p.Np; n += 32) {
+                    uint32_t nz = 0, sg = 0;
+                    if (n < a.N) {
+                        const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
+                        nz = __ldg(blk + (wd & 3));
+                        sg = __ldg(blk + 4 + (wd & 3));
+                    } else if (n == a.N) {
+                        nz = 0xFFFFFFFFu; sg = 0xFFFFFFFFu;
+                    }
+                    uint32_t o[8];
+                    tc::unpack32(nz, sg, o);
+                    uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Np + n);
+                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+            }
+        }
+        tc::fence_smem_to_async_proxy();
+        tc::mbar_arrive(w_ready);
+        asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;      // kEpiWarp0 is a multiple of 4
         const int64_t ostride = (int64_t)a.Ho * a.Wo;
         const int nblk16 = (a.N + 15) / 16;
