@@ -70,11 +70,14 @@ struct ConvI8Plan {
     int T;                 // taps
     int TM;                // 128-pixel sub-tiles per tile
     int RT;                // padded rows per tile
+    int R0;                // padded rows of a strip's first tile (<= RT)
     int halo;              // kh - 1 rows shared with the next tile
     int ppix;              // pixels allocated per code buffer
     int total_rows;        // B*PH
     int grid;              // CTAs = strips
     uint32_t tmem_cols;
+    int const_tmem;        // epilogue constants replicated in tensor memory (columns cbase..), not read from smem
+    uint32_t cbase, Nc;    // first constant column; columns per constant = N rounded up to 16
     FastDiv div_pw, div_ph;
     int n_mma;             // MMAs per sub-tile: taps * groups of 32 channels
     int use_tma;           // input rows staged by TMA (else loaded by the converters)
@@ -110,11 +113,18 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     p.RT = p.TM * kTileM / p.PW;
     if (p.RT > kMaxSlots - p.halo) p.RT = kMaxSlots - p.halo;
     if (p.RT < 1) return false;
+    // A CTA's first tile is half as tall when its strip has several tiles: the tensor core and the
+    // epilogue then start after half the input, and (the strip length permitting) the last tile,
+    // whose epilogue nothing overlaps, is short as well.
+    p.R0 = (p.RT >= 2 && (int64_t)p.total_rows >= (int64_t)2 * p.RT * sms) ? p.RT / 2 : p.RT;
     p.ppix = (p.TM * kTileM + p.halo * p.PW + (c.kw - 1) + 7) / 8 * 8;
     const int tiles = (p.total_rows + p.RT - 1) / p.RT;
     p.grid = tiles < sms ? tiles : sms;
+    p.Nc = (uint32_t)((c.N + 15) / 16 * 16);
+    p.cbase = (uint32_t)(2 * p.TM * p.Np);
+    p.const_tmem = (p.cbase + 3 * p.Nc <= 512) ? 1 : 0;
     uint32_t cols = 32;
-    while (cols < (uint32_t)(2 * p.TM * p.Np)) cols *= 2;
+    while (cols < p.cbase + (p.const_tmem ? 3 * p.Nc : 0)) cols *= 2;
     p.tmem_cols = cols;
     p.div_pw = make_fastdiv((uint32_t)p.PW);
     p.div_ph = make_fastdiv((uint32_t)p.PH);
@@ -268,10 +278,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         const float lo0 = sLo[0], hi0 = sHi[0];
         uint32_t st_count = 0;                                 // stages consumed so far
         int it = 0;
-        for (int g = s0; g < s1; g += p.RT, ++it) {
+        for (int g = s0; g < s1; g += it == 0 ? p.R0 : p.RT, ++it) {
             const int buf = it & 1;
             uint4* sA = reinterpret_cast<uint4*>(smem + (buf ? p.off_a[1] : p.off_a[0]));      // [Cp/16][ppix]
-            const int nrows = min(p.RT, s1 - g);
+            const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
             const int slot0 = it == 0 ? 0 : p.halo;            // first row slot that is new
             const int pp0 = slot0 * p.PW, pp1 = (nrows + p.halo) * p.PW;
             // (the barrier inside also orders this tile after every converter's writes to the previous buffer)
@@ -280,9 +290,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 // the kh-1 rows shared with the previous tile: copy their codes
                 const uint4* prev = reinterpret_cast<const uint4*>(smem + (buf ? p.off_a[0] : p.off_a[1]));
                 const int ncopy = p.halo * p.PW;
+                const int prev_rows = it == 1 ? p.R0 : p.RT;      // rows of the previous tile
                 for (int i = tid; i < nchunk * ncopy; i += kConvThreads) {
                     const int ch = i / ncopy, x = i - ch * ncopy;
-                    sA[ch * p.ppix + x] = prev[ch * p.ppix + p.RT * p.PW + x];
+                    sA[ch * p.ppix + x] = prev[ch * p.ppix + prev_rows * p.PW + x];
                 }
             }
             if (p.use_tma) {
@@ -351,8 +362,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             uint32_t st_count = 0;
             bool alive = true;
             int it = 0;
-            for (int g = s0; g < s1 && alive; g += p.RT, ++it) {
-                const int nrows = min(p.RT, s1 - g);
+            for (int g = s0; g < s1 && alive; g += it == 0 ? p.R0 : p.RT, ++it) {
+                const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
                 const int slot0 = it == 0 ? 0 : p.halo;
                 const int nnew = nrows + p.halo - slot0;           // new row slots (<= 32)
                 // lane j looks at new slot j: which image row is it, if any
@@ -400,12 +411,22 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             const uint64_t desc_hi = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
             const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
             const uint32_t w16 = (tc::smem_addr(sW) >> 4) + ((((uint32_t)p.Np * 16) >> 4) << 16);
+            // Filters of up to nine taps: the taps' operand offsets stay in registers, so that nothing
+            // but arithmetic sits between two batches of MMAs (the tensor core's queue is short: while
+            // the issuing thread waits for a table load, the tensor core idles).
+            const bool taps_in_regs = p.T <= 9;
+            uint32_t ta[9], tb[9];
+            #pragma unroll
+            for (int t = 0; t < 9; ++t) {
+                ta[t] = taps_in_regs && t < p.T ? p.tab_a[t] : 0u;
+                tb[t] = taps_in_regs && t < p.T ? p.tab_b[t] : 0u;
+            }
             int it = 0;
             bool filters_ok = wait_or_die(w_ready, 0, a.status, dead);
-            for (int g = s0; g < s1 && filters_ok; g += p.RT, ++it) {
+            for (int g = s0; g < s1 && filters_ok; g += it == 0 ? p.R0 : p.RT, ++it) {
                 const int buf = it & 1;
                 const uint32_t ph = (it >> 1) & 1;
-                const int nrows = min(p.RT, s1 - g);
+                const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
                 const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;          // sub-tiles with any row
                 if (!wait_or_die(&acc_empty[buf], ph ^ 1, a.status, dead)) break;
                 const uint32_t a16 = tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4;
@@ -418,6 +439,23 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     for (int tm = 0; tm < ntm; ++tm) {
                         const uint32_t d = tmem + (uint32_t)((buf * p.TM + tm) * p.Np);
                         const uint32_t a_tm = a16 + (uint32_t)(tm * kTileM) + a_lbo_field;
+                        if (taps_in_regs) {
+                            const uint32_t ag = a_tm + (uint32_t)(2 * grp) * (uint32_t)p.ppix;
+                            const uint32_t bg = w16 + (uint32_t)(2 * grp) * (uint32_t)p.Np;
+                            if (p.T == 9) {
+                                tc::mma_i8_ss(d, desc_hi | (ag + ta[0]), desc_hi | (bg + tb[0]), idesc, grp > 0);
+                                #pragma unroll
+                                for (int t = 1; t < 9; ++t)
+                                    tc::mma_i8_ss_acc(d, desc_hi | (ag + ta[t]), desc_hi | (bg + tb[t]), idesc);
+                            } else {
+                                #pragma unroll
+                                for (int t = 0; t < 9; ++t)
+                                    if (t < p.T)
+                                        tc::mma_i8_ss(d, desc_hi | (ag + ta[t]), desc_hi | (bg + tb[t]), idesc,
+                                                      grp > 0 || t > 0);
+                            }
+                            continue;
+                        }
                         int i = grp * p.T;
                         const int i_end = i + p.T;
                         for (; i + 9 <= i_end; i += 9) issue_mmas<9>(p, i, d, a_tm, w16, desc_hi, idesc);
@@ -486,10 +524,28 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         const int nblk16 = (a.N + 15) / 16;
         const int blk_begin = half == 0 ? 0 : (nblk16 + 1) / 2;
         const int blk_end = half == 0 ? (nblk16 + 1) / 2 : nblk16;
+        // The constants of this warp's columns go to tensor memory, replicated in each of its 32 lanes:
+        // the epilogue then fetches them with tcgen05.ld, which does not compete with the tensor core,
+        // the converters and TMA for shared-memory bandwidth as a broadcast shared load per output did.
+        const uint32_t cq = tmem + ((uint32_t)(q * 32) << 16) + p.cbase;
+        if (p.const_tmem) {
+            for (int blk = blk_begin; blk < blk_end; ++blk) {
+                uint32_t k1[16], k2[16], k3[16];
+                #pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float4 c = sC[blk * 16 + j];
+                    k1[j] = __float_as_uint(c.x); k2[j] = __float_as_uint(c.y); k3[j] = __float_as_uint(c.z);
+                }
+                tc::tmem_st16(cq + (uint32_t)(blk * 16), k1);
+                tc::tmem_st16(cq + p.Nc + (uint32_t)(blk * 16), k2);
+                tc::tmem_st16(cq + 2 * p.Nc + (uint32_t)(blk * 16), k3);
+            }
+            tc::tmem_st_wait();
+        }
         int it = 0;
-        for (int g = s0; g < s1; g += p.RT, ++it) {
+        for (int g = s0; g < s1; g += it == 0 ? p.R0 : p.RT, ++it) {
             const int buf = it & 1;
-            const int nrows = min(p.RT, s1 - g);
+            const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
             const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
             role_wait(warp == kEpiWarp0, &acc_full[buf], (it >> 1) & 1, a.status, dead, kEpiBarrier, kEpiThreads);
             const bool alive = !*dead;
@@ -518,20 +574,56 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 uint32_t sx_raw;
                 asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
                              : "=r"(sx_raw) : "r"(trow + (uint32_t)a.N) : "memory");
-                uint32_t v[16];
-                if (blk_begin < blk_end) tc::tmem_ld16(trow + (uint32_t)(blk_begin * 16), v);
-                tc::tmem_ld_wait();
-                const float fsx = (float)(int)sx_raw;
+                bool sx_ready = false;
+                float fsx = 0.f;
+                // uniform over the warp: whole blocks with constants in tensor memory and no debug output
+                const bool tm_path = p.const_tmem && a.dbg_acc == nullptr;
                 for (int blk = blk_begin; blk < blk_end; ++blk) {
-                    // take the block's values, then start the next block's load before the stores
-                    uint32_t u[16];
-                    #pragma unroll
-                    for (int j = 0; j < 16; ++j) u[j] = v[j];
-                    if (blk + 1 < blk_end) tc::tmem_ld16(trow + (uint32_t)((blk + 1) * 16), v);
                     const int n0 = blk * 16;
+                    if (tm_path && n0 + 16 <= a.N) {
+                        // eight columns at a time: accumulators and the three constants from tensor memory
+                        #pragma unroll
+                        for (int h8 = 0; h8 < 16; h8 += 8) {
+                            uint32_t u8[8], k1[8], k2[8], k3[8];
+                            tc::tmem_ld8(trow + (uint32_t)(n0 + h8), u8);
+                            tc::tmem_ld8(cq + (uint32_t)(n0 + h8), k1);
+                            tc::tmem_ld8(cq + p.Nc + (uint32_t)(n0 + h8), k2);
+                            tc::tmem_ld8(cq + 2 * p.Nc + (uint32_t)(n0 + h8), k3);
+                            tc::tmem_ld_wait();
+                            if (!sx_ready) { fsx = (float)(int)sx_raw; sx_ready = true; }
+                            if (ok && !border) {
+                                #pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    optr[(int64_t)(n0 + h8 + j) * ostride] =
+                                        fmaf(__uint_as_float(k1[j]), (float)(int)u8[j],
+                                             fmaf(__uint_as_float(k2[j]), fsx, __uint_as_float(k3[j])));
+                            } else if (ok) {
+                                // value-zero padding at an image border: S_w and K over inside taps only
+                                #pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    const int n = n0 + h8 + j;
+                                    int s_w = 0;
+                                    for (int t = 0; t < p.T; ++t) {
+                                        const int h = ho - a.pad + t / a.kw, vv = wo - a.pad + t % a.kw;
+                                        if (h >= 0 && h < a.H && vv >= 0 && vv < a.W) s_w += a.w_sum[(1 + t) * a.N + n];
+                                    }
+                                    const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
+                                    const double wo_ = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
+                                    const float c3 = (float)((double)a.ep.a_offset_val *
+                                                             (ws * (double)s_w + (double)a.C * n_inside * wo_));
+                                    optr[(int64_t)n * ostride] = fmaf(__uint_as_float(k1[j]), (float)(int)u8[j],
+                                                                      fmaf(__uint_as_float(k2[j]), fsx, c3));
+                                }
+                            }
+                        }
+                        continue;
+                    }
+                    uint32_t u[16];
+                    tc::tmem_ld16(trow + (uint32_t)n0, u);
+                    tc::tmem_ld_wait();
+                    if (!sx_ready) { fsx = (float)(int)sx_raw; sx_ready = true; }
                     if (ok) {
                         if (!border && dptr == nullptr && n0 + 16 <= a.N) {
-                            // fast path: a whole block, code-zero padding (or an interior pixel)
                             #pragma unroll
                             for (int j = 0; j < 16; ++j) {
                                 const float4 c = sC[n0 + j];
@@ -562,8 +654,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                             }
                         }
                     }
-                    tc::tmem_ld_wait();
                 }
+                if (blk_begin >= blk_end) tc::tmem_ld_wait();      // the S_x load still has to land
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[buf]);
