@@ -54,7 +54,7 @@ constexpr int kWarps = kEpiWarp0 + kEpiWarps + kConvWarps - 2;
 constexpr int kThreads = kWarps * 32;
 __device__ __forceinline__ bool is_conv_warp(int w) { return w == 2 || w == 3 || w >= kEpiWarp0 + kEpiWarps; }
 __device__ __forceinline__ int conv_warp_index(int w) { return w < 4 ? w - 2 : w - (kEpiWarp0 + kEpiWarps) + 2; }
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 8;                         // input batches (one tile's rows of 32 channels) in flight
 constexpr int kMaxGroups = 16;                          // groups of 32 input channels (C <= 512)
 constexpr int kMaxMma = 160;                           // MMAs per sub-tile the descriptor table holds
 constexpr int kMaxSlots = 32;                          // row slots of a tile (rows + halo rows)
@@ -79,11 +79,12 @@ struct ConvI8Plan {
     int const_tmem;        // epilogue constants replicated in tensor memory (columns cbase..), not read from smem
     uint32_t cbase, Nc;    // first constant column; columns per constant = N rounded up to 16
     FastDiv div_pw, div_ph;
+    FastDiv div_np, div_cw;    // by Np and by Cp/32 (filter expansion)
     int n_mma;             // MMAs per sub-tile: taps * groups of 32 channels
     int use_tma;           // input rows staged by TMA (else loaded by the converters)
     int stages;            // depth of the staging ring
     uint32_t box_bytes;    // one TMA box: 32 channels x one image row of fp32
-    uint32_t stage_bytes;
+    int nslots;            // row slots of the TMA ring
     uint32_t off_stage;
     uint32_t off_a[2], off_w, off_lo, off_hi, off_c, off_rows, off_bar, off_misc;
     size_t smem_bytes;
@@ -128,6 +129,8 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     p.tmem_cols = cols;
     p.div_pw = make_fastdiv((uint32_t)p.PW);
     p.div_ph = make_fastdiv((uint32_t)p.PH);
+    p.div_np = make_fastdiv((uint32_t)p.Np);
+    p.div_cw = make_fastdiv((uint32_t)(p.Cp / 32));
     p.n_mma = p.T * (p.Cp / 32);
     if (p.n_mma > kMaxMma) return false;
     for (int i = 0; i < p.n_mma; ++i) {
@@ -148,18 +151,21 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     p.off_bar = o;  o += (7 + 2 * kMaxStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] st_full[] st_empty[] a_full[2][groups]
     p.off_misc = o; o += 16;                            // tmem slot, dead flag
     if (o > kSmemLimit) return false;
-    // staging ring for TMA: as many stages (2..4) as fit
-    p.use_tma = 0; p.stages = 0; p.off_stage = o;
+    // staging ring for TMA
+    p.use_tma = 0; p.stages = 0; p.nslots = 0; p.off_stage = o;
     p.box_bytes = 32u * (uint32_t)c.W * 4u;
-    p.stage_bytes = (uint32_t)(p.RT + p.halo) * p.box_bytes;
     const bool tma_ok = (c.W % 4 == 0) && (reinterpret_cast<uintptr_t>(c.x) % 16 == 0);
     if (tma_ok) {
         const uint32_t base = (o + 127) / 128 * 128;
-        int ns = (int)((kSmemLimit - base) / p.stage_bytes);
-        if (ns > kMaxStages) ns = kMaxStages;
-        if (ns >= 2) {
-            p.use_tma = 1; p.stages = ns; p.off_stage = base;
-            o = base + (uint32_t)ns * p.stage_bytes;
+        // A ring of row slots (one TMA box each); a batch takes as many as the tile has new rows.  Two
+        // steady-state batches in flight measured fastest (a deeper ring lost 3 %), so the ring is
+        // capped at two tiles' worth of new rows.
+        int ns = base < kSmemLimit ? (int)((kSmemLimit - base) / p.box_bytes) : 0;
+        const int cap = 2 * p.RT > p.RT + p.halo ? 2 * p.RT : p.RT + p.halo;
+        if (ns > cap) ns = cap;
+        if (ns >= p.RT + p.halo) {
+            p.use_tma = 1; p.stages = kMaxStages; p.nslots = ns; p.off_stage = base;
+            o = base + (uint32_t)ns * p.box_bytes;
         }
     }
     p.smem_bytes = o;
@@ -276,7 +282,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         const bool per_layer = a.n_thr == 1;
         const int ngroup = p.Cp / 32;
         const float lo0 = sLo[0], hi0 = sHi[0];
-        uint32_t st_count = 0;                                 // stages consumed so far
+        uint32_t st_count = 0;                                 // batches consumed so far
+        int row_base = 0;                                      // ring slot of the batch's first row
         int it = 0;
         for (int g = s0; g < s1; g += it == 0 ? p.R0 : p.RT, ++it) {
             const int buf = it & 1;
@@ -299,10 +306,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             if (p.use_tma) {
                 const int npix = pp1 - pp0;
                 for (int grp = 0; grp < ngroup; ++grp, ++st_count) {
-                    const uint32_t s = st_count % (uint32_t)p.stages;
-                    role_wait(tid < 32, &st_full[s], (st_count / (uint32_t)p.stages) & 1, a.status, dead,
+                    const uint32_t s = st_count % (uint32_t)kMaxStages;
+                    role_wait(tid < 32, &st_full[s], (st_count / (uint32_t)kMaxStages) & 1, a.status, dead,
                               kConvBarrier, kConvThreads);
-                    const float* stage = reinterpret_cast<const float*>(smem + p.off_stage + s * p.stage_bytes);
+                    const float* ring = reinterpret_cast<const float*>(smem + p.off_stage);
                     // item = (padded pixel, half of the group's 32 channels)
                     for (int i = tid; i < 2 * npix; i += kConvThreads) {
                         const int hf = i >= npix ? 1 : 0;
@@ -316,7 +323,9 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                         const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
                         uint4 w = make_uint4(0, 0, 0, 0);
                         if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
-                            const float* src = stage + ((sl - (uint32_t)slot0) * 32u + 16u * hf) * (uint32_t)a.W + (uint32_t)c;
+                            int rs = row_base + (int)sl - slot0;
+                            if (rs >= p.nslots) rs -= p.nslots;
+                            const float* src = ring + ((uint32_t)rs * 32u + 16u * hf) * (uint32_t)a.W + (uint32_t)c;
                             float v[16];
                             #pragma unroll
                             for (int e = 0; e < 16; ++e) v[e] = src[perm16(e) * a.W];
@@ -328,6 +337,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     tc::mbar_arrive(&st_empty[s]);
                     tc::fence_smem_to_async_proxy();
                     tc::mbar_arrive(&a_full[buf * kMaxGroups + grp]);
+                    row_base += nrows + p.halo - slot0;
+                    if (row_base >= p.nslots) row_base -= p.nslots;
                 }
             } else {
                 // direct path: item = (padded pixel, chunk of 16 channels), 16 loads in flight
@@ -359,7 +370,11 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     } else if (warp == kProdWarp) {
         // ------------------------------------------------------------ producer
         if (p.use_tma) {
-            uint32_t st_count = 0;
+            const int ngroup = p.Cp / 32;
+            uint32_t st_count = 0;              // batches issued
+            uint32_t rel = 0;                   // batches known to be released by the converters
+            int rel_it = 0, rel_grp = 0;        // (tile, channel group) of batch `rel`
+            int head = 0, used = 0;             // ring: next free row slot, row slots held by batches rel..
             bool alive = true;
             int it = 0;
             for (int g = s0; g < s1 && alive; g += it == 0 ? p.R0 : p.RT, ++it) {
@@ -378,27 +393,42 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 __syncwarp();
                 sRows[lane] = info;
                 __syncwarp();
-                for (int grp = 0; grp < p.Cp / 32; ++grp, ++st_count) {
-                    const uint32_t s = st_count % (uint32_t)p.stages;
-                    const bool ok = wait_or_die(&st_empty[s], ((st_count / (uint32_t)p.stages) & 1) ^ 1, a.status, dead);
-                    if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+                for (int grp = 0; grp < ngroup && alive; ++grp, ++st_count) {
+                    // room in the ring and a free pair of barriers: retire the oldest batches
+                    while (used + nnew > p.nslots || st_count - rel >= (uint32_t)kMaxStages) {
+                        const bool ok = wait_or_die(&st_empty[rel % (uint32_t)kMaxStages],
+                                                    (rel / (uint32_t)kMaxStages) & 1, a.status, dead);
+                        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+                        const int rg = s0 + (rel_it == 0 ? 0 : p.R0 + (rel_it - 1) * p.RT);
+                        const int rrows = min(rel_it == 0 ? p.R0 : p.RT, s1 - rg);
+                        used -= rel_it == 0 ? rrows + p.halo : rrows;
+                        ++rel;
+                        if (++rel_grp == ngroup) { rel_grp = 0; ++rel_it; }
+                    }
+                    if (!alive) break;
+                    const uint32_t s = st_count % (uint32_t)kMaxStages;
                     if (lane == 0) {
                         if (mask == 0) {
                             tc::mbar_arrive(&st_full[s]);
                         } else {
                             mbar_expect_tx(&st_full[s], (uint32_t)__popc(mask) * p.box_bytes);
-                            const uint32_t stage = tc::smem_addr(smem + p.off_stage + s * p.stage_bytes);
+                            const uint32_t ring = tc::smem_addr(smem + p.off_stage);
                             const uint32_t bar = tc::smem_addr(&st_full[s]);
                             uint32_t m = mask;
                             while (m) {
                                 const int j = __ffs(m) - 1;
                                 m &= m - 1;
                                 const uint32_t inf = sRows[j];
-                                tma_load_row(stage + (uint32_t)j * p.box_bytes, &tmap, (int)(inf & 0x7FFu), grp * 32,
+                                int rs = head + j;
+                                if (rs >= p.nslots) rs -= p.nslots;
+                                tma_load_row(ring + (uint32_t)rs * p.box_bytes, &tmap, (int)(inf & 0x7FFu), grp * 32,
                                              (int)(inf >> 11), bar);
                             }
                         }
                     }
+                    head += nnew;
+                    if (head >= p.nslots) head -= p.nslots;
+                    used += nnew;
                     __syncwarp();
                 }
             }
@@ -477,7 +507,49 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         // While the first input rows are in flight these warps, idle until the first accumulators are
         // complete, expand the filters and work out the epilogue constants.
         const int etid = threadIdx.x - kEpiWarp0 * 32;
-        {   // per-output-channel constants in double, rounded once:
+        {   // filters: bit planes -> int8, [tap][chunk][n]; row N is all +1, rows above it are 0.
+            // item = (32-channel word of a tap, filter row); a thread's loads of six items are in flight
+            // together (the expansion is on the path to the first MMA, and each load is a trip to HBM)
+            const int cwords = p.Cp / 32;
+            const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
+            const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
+            const int items = p.T * cwords * p.Np;
+            constexpr int kBatch = 6;
+            for (int base = etid; base < items; base += kBatch * kEpiThreads) {
+                uint32_t nz[kBatch], sg[kBatch];
+                #pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int i = base + u * kEpiThreads;
+                    nz[u] = 0; sg[u] = 0;
+                    if (i < items) {
+                        const int wd = (int)fdiv((uint32_t)i, p.div_np), n = i - wd * p.Np;
+                        if (n < a.N) {
+                            const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
+                            nz[u] = __ldg(blk + (wd & 3));
+                            sg[u] = __ldg(blk + 4 + (wd & 3));
+                        } else if (n == a.N) {
+                            nz[u] = 0xFFFFFFFFu; sg[u] = 0xFFFFFFFFu;
+                        }
+                    }
+                }
+                #pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int i = base + u * kEpiThreads;
+                    if (i < items) {
+                        const int wd = (int)fdiv((uint32_t)i, p.div_np), n = i - wd * p.Np;
+                        const int t = (int)fdiv((uint32_t)wd, p.div_cw), cw = wd - t * cwords;
+                        uint32_t o[8];
+                        tc::unpack32(nz[u], sg[u], o);
+                        uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Np + n);
+                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                        dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    }
+                }
+            }
+        }
+        tc::fence_smem_to_async_proxy();
+        tc::mbar_arrive(w_ready);
+        {   // per-output-channel constants in double, rounded once (first needed by the first epilogue):
             //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
             const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
             for (int n = etid; n < p.Np; n += kEpiThreads) {
@@ -492,32 +564,6 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 sC[n] = make_float4(c1, c2, c3, 0.f);
             }
         }
-        {   // filters: bit planes -> int8, [tap][chunk][n]; row N is all +1, rows above it are 0
-            const int cwords = p.Cp / 32;
-            const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
-            const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
-            // a warp takes one 32-channel word of every filter row at a time (no per-item divisions)
-            for (int wd = warp - kEpiWarp0; wd < p.T * cwords; wd += kEpiWarps) {
-                const int t = wd / cwords, cw = wd % cwords;
-                for (int n = lane; n < p.Np; n += 32) {
-                    uint32_t nz = 0, sg = 0;
-                    if (n < a.N) {
-                        const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
-                        nz = __ldg(blk + (wd & 3));
-                        sg = __ldg(blk + 4 + (wd & 3));
-                    } else if (n == a.N) {
-                        nz = 0xFFFFFFFFu; sg = 0xFFFFFFFFu;
-                    }
-                    uint32_t o[8];
-                    tc::unpack32(nz, sg, o);
-                    uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Np + n);
-                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
-                }
-            }
-        }
-        tc::fence_smem_to_async_proxy();
-        tc::mbar_arrive(w_ready);
         asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;      // kEpiWarp0 is a multiple of 4
         const int64_t ostride = (int64_t)a.Ho * a.Wo;
