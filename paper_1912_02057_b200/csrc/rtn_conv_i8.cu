@@ -241,6 +241,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
 
     // ---------------------------------------------------------------- set-up (all threads)
+    tc::pdl_trigger();
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
         for (int i = 0; i < 2 * kMaxGroups; ++i) tc::mbar_init(&a_full[i], kConvThreads);
@@ -278,6 +279,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             sHi[c] = hi;
         }
         asm volatile("bar.sync %0, %1;" ::"r"(kConvBarrier), "r"(kConvThreads) : "memory");
+        if (!p.use_tma) tc::pdl_wait();             // the direct path reads x
         const int64_t cs = (int64_t)a.H * a.W;
         const bool per_layer = a.n_thr == 1;
         const int ngroup = p.Cp / 32;
@@ -370,6 +372,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     } else if (warp == kProdWarp) {
         // ------------------------------------------------------------ producer
         if (p.use_tma) {
+            tc::pdl_wait();                         // x may be the previous kernel's output
             const int ngroup = p.Cp / 32;
             uint32_t st_count = 0;              // batches issued
             uint32_t rel = 0;                   // batches known to be released by the converters
@@ -565,6 +568,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             }
         }
         asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible
+        tc::pdl_wait();                             // out may still be read by the previous kernel
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;      // kEpiWarp0 is a multiple of 4
         const int64_t ostride = (int64_t)a.Ho * a.Wo;
         const int nblk16 = (a.N + 15) / 16;
@@ -772,8 +776,7 @@ cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s)
     cudaError_t e = cudaFuncSetAttribute(conv_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
-    conv_i8_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(c, p, tmap);
-    return cudaGetLastError();
+    return launch_pdl(conv_i8_kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p, tmap);
 }
 
 }  // namespace rtn

@@ -140,6 +140,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
     const int s0 = (int)((int64_t)blockIdx.x * p.total_rows / p.grid);
     const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
 
+    tc::pdl_trigger();
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
         tc::mbar_init(a_full, kWorkWarps);
@@ -175,6 +176,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
+    tc::pdl_wait();         // from here on: x, out (the set-up above read only the layer's parameters)
 
     if (warp >= kWorkWarp0) {
         // ------------------------------------------------------------ workers
@@ -413,8 +415,7 @@ cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s)
     cudaError_t e = cudaFuncSetAttribute(conv_i8s_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
-    conv_i8s_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(c, p);
-    return cudaGetLastError();
+    return launch_pdl(conv_i8s_kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p);
 }
 
 }  // namespace rtn

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of librtn_b200 (not installed).
 #pragma once
+#include <cstring>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include "rtn.h"
@@ -99,6 +100,27 @@ __device__ __forceinline__ float epilogue_f64(int s_xw, int s_x, int s_w, double
     const double r = a_s * w_s * (double)s_xw + a_s * w_o * (double)s_x
                    + a_o * w_s * (double)s_w + k_eff * a_o * w_o;
     return (float)r;
+}
+
+// Launch that allows the kernel's CTAs to start while the stream's previous kernel is still
+// draining (programmatic dependent launch); the kernel orders itself with tc::pdl_wait().  Inside a
+// stream capture the launch becomes a programmatic edge of the graph.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem_bytes, cudaStream_t s,
+                              Args&&... args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 #endif  // __CUDACC__

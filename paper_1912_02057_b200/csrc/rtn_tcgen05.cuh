@@ -56,6 +56,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
     return false;
 }
 
+// ------------------------------------------------------------------------------------ launch overlap
+// Programmatic dependent launch.  The kernel is launched so that its CTAs may start while the
+// previous kernel of the stream is still draining: every access to tensors that kernel may write or read sits behind
+// pdl_wait(), which returns once that kernel has completed and its writes are visible; the set-up
+// before it reads only the layer's parameters.  pdl_trigger() lets the next kernel of the stream do the same.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------------------------ fences
 // Shared-memory writes made with ordinary stores become visible to the tensor core (async proxy).
 __device__ __forceinline__ void fence_smem_to_async_proxy()
