@@ -6,17 +6,23 @@
 // implicit GEMM of a stride-1 conv done by shifting the A window by (i*PW + j) pixels per filter
 // tap, tcgen05.mma kind::i8 into int32 accumulators in tensor memory, affine epilogue fused.
 // Differences:
-//   * the filters are expanded from their bit planes (Table 1) to int8 one K = 32 slice at a time
-//     into a ring of shared-memory stages, by the same warps that ternarized the tile, while the
-//     tensor core consumes earlier slices;
+//   * the filters are expanded from their bit planes (Table 1) to int8 one packed block (four
+//     K = 32 slices) at a time into a ring of shared-memory stages by warps of their own, while the
+//     tensor core consumes earlier stages; expanding costs a quarter of the SM's issue slots per
+//     256-pixel tile, so a CTA's tile is made 256 pixels whenever its strip has that many;
+//   * when C is a multiple of 128 the K loop runs 128-channel block by block (all taps of a block,
+//     then the next block), and the ternarizer hands the code buffer over in 32-channel groups, so
+//     the tensor core starts on a tile before all of its input has arrived;
 //   * S_x comes from per-pixel code sums the ternarizer leaves in shared memory (summed over the
 //     taps in the epilogue), so all 256 accumulator columns are free for output channels;
 //   * a 1x1 convolution (any stride, no padding) uses the same code with "rows" = output rows and a
 //     strided pixel gather in the ternarizer (no halo, one tap).
 //
-// Warp roles: warp 0 issues MMAs (one thread); warps 4..11 epilogue; warps 12..19 workers
-// (ternarize the tile, then expand filter slices).  One code buffer, one accumulator set (two when
-// they fit), mbarrier hand-offs with bounded waits.
+// Warp roles: warp 0 issues MMAs (one thread); warps 12..19 expand filters; warps 4..11 ternarize
+// tile i+1 and then run the epilogue of tile i; warps 1..3 only ternarize.  One or two code buffers
+// and accumulator sets (as fit), mbarrier hand-offs with bounded waits.  Every CTA takes an equal
+// strip of the padded rows and cuts it into equal tiles, so that all SMs are busy whatever the
+// batch size.
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
 #include "rtn_conv_i8_common.cuh"
@@ -30,29 +36,37 @@ using namespace conv_detail;
 constexpr int kEpiWarp0 = 4;
 constexpr int kEpiWarps = 8;
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kWorkWarp0 = kEpiWarp0 + kEpiWarps;
-constexpr int kWorkWarps = 8;
-constexpr int kWorkThreads = kWorkWarps * 32;
-constexpr int kThreads = (kWorkWarp0 + kWorkWarps) * 32;
+constexpr int kExpWarp0 = 12;
+constexpr int kExpWarps = 8;
+constexpr int kExpThreads = kExpWarps * 32;
+constexpr int kTernWarps = 11;                         // warps 1..11
+constexpr int kTernThreads = kTernWarps * 32;
+constexpr int kThreads = 20 * 32;
 constexpr int kTileM = 128;
 constexpr int kMaxK = 304;                             // K = 32 slices per tile the table holds
 constexpr int kMaxWStages = 8;
 constexpr int kSlices = 4;                             // K = 32 slices per filter stage (one packed block)
+constexpr int kMaxGroups = 16;                         // 32-channel groups (C <= 512)
+constexpr int kPsumRing = 4;
 constexpr size_t kSmemLimit = 220 * 1024;
-constexpr int kWorkBarrier = 2;
+constexpr int kEpiBarrier = 1, kTernBarrier = 2, kExpBarrier = 3;
 
 struct ConvI8SPlan {
     int PW, PH;            // row length / rows per image of the pixel sequence (padded for k > 1)
     int istride, ipad;     // input pixel of sequence pixel (r, c): (r*istride - ipad, c*istride - ipad)
     int Cp, Np, T, TM, RT, halo, ppix, total_rows, grid;
-    int nK;                // K = 32 slices per tile: taps * Cp/32
+    int nK;                // K = 32 slices per tile in stage order, padded to whole packed blocks
     int nW;                // filter ring depth
     int nAcc;              // accumulator sets (1 or 2)
+    int nA;                // code buffers (1 or 2)
     uint32_t tmem_cols;
-    FastDiv div_pw, div_ph;
-    uint32_t off_a, off_w, off_psum, off_lo, off_hi, off_c, off_bar, off_misc;
+    FastDiv div_pw, div_ph, div_T;   // div_T: stage -> (128-channel block, tap)
+    uint32_t off_a[2], off_w, off_psum, off_lo, off_hi, off_c, off_bar, off_misc;
     size_t smem_bytes;
-    uint32_t tab_a[kMaxK]; // per slice: start of the A window in 16-byte units of the code buffer
+    int blocks_major;      // stage order: 128-channel block outer, tap inner (else the packed order)
+    uint32_t tab_a[kMaxK]; // per slice of the stage order: start of the A window in 16-byte units of
+                           // the code buffer (bits 0..23) and its 32-channel group (bits 24..27);
+                           // 0xFFFFFFFF for the padding slices of the last packed block
 };
 
 bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
@@ -71,82 +85,121 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
     p.Cp = (c.C + 31) / 32 * 32;
     p.Np = (c.N + 15) / 16 * 16;
     if (p.Np > 256) return false;
-    if ((int64_t)c.C * p.T > (int64_t(1) << 24)) return false;
+    if (p.Cp / 32 > kMaxGroups) return false;
     p.total_rows = c.B * p.PH;
-    p.TM = (2 * p.Np <= 512 && (int64_t)p.total_rows * p.PW >= (int64_t)2 * 148 * kTileM) ? 2 : 1;
+    p.grid = p.total_rows < sms ? p.total_rows : sms;
+    // 256-pixel tiles whenever a CTA's strip has more than 128 pixels: a tile's filter stream costs
+    // the same whatever its size
+    const int strip_rows = (p.total_rows + p.grid - 1) / p.grid;
+    p.TM = (2 * p.Np <= 512 && strip_rows * p.PW > kTileM) ? 2 : 1;
     p.nAcc = (2 * p.TM * p.Np <= 512) ? 2 : 1;
     p.RT = p.TM * kTileM / p.PW;
     if (p.RT < 1) return false;
     p.ppix = (p.TM * kTileM + p.halo * p.PW + (c.kw - 1) + 7) / 8 * 8;
-    const int tiles = (p.total_rows + p.RT - 1) / p.RT;
-    p.grid = tiles < sms ? tiles : sms;
     uint32_t cols = 32;
     while (cols < (uint32_t)(p.nAcc * p.TM * p.Np)) cols *= 2;
     p.tmem_cols = cols;
     p.div_pw = make_fastdiv((uint32_t)p.PW);
     p.div_ph = make_fastdiv((uint32_t)p.PH);
-    p.nK = p.T * (p.Cp / 32);
+    p.div_T = make_fastdiv((uint32_t)p.T);
+    const int cwords = p.Cp / 32;
+    const int nwords = p.T * cwords;
+    const int nblocks = (nwords + kSlices - 1) / kSlices;
+    p.nK = nblocks * kSlices;
     if (p.nK > kMaxK) return false;
-    for (int i = 0; i < p.nK; ++i) {
-        const int t = i / (p.Cp / 32), h = i % (p.Cp / 32);
-        p.tab_a[i] = (uint32_t)(2 * h) * p.ppix + (uint32_t)((t / c.kw) * p.PW + (t % c.kw));
+    p.blocks_major = (cwords % kSlices == 0) ? 1 : 0;
+    for (int st = 0; st < nblocks; ++st) {
+        // packed block of stage st
+        const int blk = p.blocks_major ? (st % p.T) * (cwords / kSlices) + st / p.T : st;
+        for (int j = 0; j < kSlices; ++j) {
+            const int word = blk * kSlices + j;
+            uint32_t e = 0xFFFFFFFFu;
+            if (word < nwords) {
+                const int t = word / cwords, h = word % cwords;
+                e = ((uint32_t)(2 * h) * p.ppix + (uint32_t)((t / c.kw) * p.PW + (t % c.kw))) | ((uint32_t)h << 24);
+            }
+            p.tab_a[st * kSlices + j] = e;
+        }
     }
-    uint32_t o = 0;
-    p.off_a = o;    o += (uint32_t)(p.Cp / 16) * p.ppix * 16;
-    p.off_psum = o; o += 3u * (uint32_t)p.ppix * 4;
-    p.off_lo = o;   o += (uint32_t)p.Cp * 4;
-    p.off_hi = o;   o += (uint32_t)p.Cp * 4;
-    o = (o + 15) / 16 * 16;
-    p.off_c = o;    o += (uint32_t)p.Np * 16;
-    p.off_bar = o;  o += (6 + 2 * kMaxWStages) * 8;     // a_full a_empty acc_full[2] acc_empty[2] w_full[] w_empty[]
-    p.off_misc = o; o += 16;
-    o = (o + 127) / 128 * 128;
-    p.off_w = o;
-    if (o > kSmemLimit) return false;
+    const uint32_t a_bytes = (uint32_t)(p.Cp / 16) * p.ppix * 16;
     const uint32_t stage = (uint32_t)p.Np * 32 * kSlices;
-    const int ngroups = (p.nK + kSlices - 1) / kSlices;
-    int nw = (int)((kSmemLimit - o) / stage);
-    if (nw > kMaxWStages) nw = kMaxWStages;
-    if (nw > ngroups) nw = ngroups;
-    if (nw < 2 && ngroups > 1) return false;
-    if (nw < 1) return false;
-    p.nW = nw;
-    p.smem_bytes = o + (uint32_t)nw * stage;
-    return true;
+    const int nstages = p.nK / kSlices;
+    // two code buffers when they leave room for a filter ring of four stages (or all of them)
+    for (p.nA = 2; p.nA >= 1; --p.nA) {
+        uint32_t o = 0;
+        p.off_a[0] = o; o += a_bytes;
+        p.off_a[1] = o; if (p.nA == 2) o += a_bytes;
+        p.off_psum = o; o += (uint32_t)kPsumRing * (uint32_t)p.ppix * 4;
+        p.off_lo = o;   o += (uint32_t)p.Cp * 4;
+        p.off_hi = o;   o += (uint32_t)p.Cp * 4;
+        o = (o + 15) / 16 * 16;
+        p.off_c = o;    o += (uint32_t)p.Np * 16;
+        p.off_bar = o;  o += (6 + 2 * kMaxWStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] w_full[] w_empty[] a_full[2][]
+        p.off_misc = o; o += 16;
+        o = (o + 127) / 128 * 128;
+        p.off_w = o;
+        if (o > kSmemLimit) continue;
+        int nw = (int)((kSmemLimit - o) / stage);
+        if (nw > kMaxWStages) nw = kMaxWStages;
+        if (nw > nstages) nw = nstages;
+        const int want = nstages < 4 ? nstages : 4;
+        if (nw < want && p.nA == 2) continue;
+        if (nw < 2 && nstages > 1) return false;
+        if (nw < 1) return false;
+        p.nW = nw;
+        p.smem_bytes = o + (uint32_t)nw * stage;
+        return true;
+    }
+    return false;
+}
+
+// One warp of a role waits on the mbarrier; the role's other warps sleep on a hardware named
+// barrier until it gets there.
+__device__ __forceinline__ void role_wait(bool leader, uint64_t* bar, uint32_t parity, unsigned* status,
+                                          volatile int* dead, int barrier_id, int nthreads)
+{
+    if (leader) wait_or_die(bar, parity, status, dead);
+    asm volatile("bar.sync %0, %1;" ::"r"(barrier_id), "r"(nthreads) : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    uint4* sA = reinterpret_cast<uint4*>(smem + p.off_a);        // [Cp/16][ppix]
     uint4* sWr = reinterpret_cast<uint4*>(smem + p.off_w);       // [nW][kSlices][2][Np]
-    int* sPsum = reinterpret_cast<int*>(smem + p.off_psum);      // [3][ppix]
+    int* sPsum = reinterpret_cast<int*>(smem + p.off_psum);      // [kPsumRing][ppix]
     float* sLo = reinterpret_cast<float*>(smem + p.off_lo);
     float* sHi = reinterpret_cast<float*>(smem + p.off_hi);
     float4* sC = reinterpret_cast<float4*>(smem + p.off_c);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-    uint64_t* a_full = bars;            // workers -> MMA: codes of the tile written
-    uint64_t* a_empty = bars + 1;       // MMA -> workers: the tile's MMAs are done
+    uint64_t* a_empty = bars;           // [2] MMA -> ternarizers: the MMAs that read the code buffer are done
     uint64_t* acc_full = bars + 2;      // [2] MMA -> epilogue
     uint64_t* acc_empty = bars + 4;     // [2] epilogue -> MMA
-    uint64_t* w_full = bars + 6;                    // [nW] workers -> MMA: filter slice expanded
-    uint64_t* w_empty = bars + 6 + kMaxWStages;     // [nW] MMA -> workers: slice consumed
+    uint64_t* w_full = bars + 6;                    // [nW] expanders -> MMA: filter stage expanded
+    uint64_t* w_empty = bars + 6 + kMaxWStages;     // [nW] MMA -> expanders: stage consumed
+    uint64_t* a_full = bars + 6 + 2 * kMaxWStages;  // [2][kMaxGroups] ternarizers -> MMA: 32 channels of codes written
     uint32_t* slot = reinterpret_cast<uint32_t*>(smem + p.off_misc);
     volatile int* dead = reinterpret_cast<volatile int*>(smem + p.off_misc + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nchunk = p.Cp / 16;
+    const int ngroup = p.Cp / 32;
+    const int nstages = p.nK / kSlices;
+    // this CTA's strip of rows, cut into equal tiles of at most RT rows
     const int s0 = (int)((int64_t)blockIdx.x * p.total_rows / p.grid);
     const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
+    const int ntile = (s1 - s0 + p.RT - 1) / p.RT;
+    const int rt = ntile > 0 ? (s1 - s0 + ntile - 1) / ntile : 1;
 
     tc::pdl_trigger();
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
-        tc::mbar_init(a_full, kWorkWarps);
-        tc::mbar_init(a_empty, 1);
-        for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kEpiThreads); }
-        for (int i = 0; i < kMaxWStages; ++i) { tc::mbar_init(&w_full[i], kWorkWarps); tc::mbar_init(&w_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) {
+            tc::mbar_init(&a_empty[i], 1);
+            tc::mbar_init(&acc_full[i], 1);
+            tc::mbar_init(&acc_empty[i], kEpiThreads);
+        }
+        for (int i = 0; i < kMaxWStages; ++i) { tc::mbar_init(&w_full[i], kExpWarps); tc::mbar_init(&w_empty[i], 1); }
+        for (int i = 0; i < 2 * kMaxGroups; ++i) tc::mbar_init(&a_full[i], kTernThreads);
         tc::mbar_init_fence();
         *dead = 0;
     }
@@ -178,29 +231,39 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
     const uint32_t tmem = *slot;
     tc::pdl_wait();         // from here on: x, out (the set-up above read only the layer's parameters)
 
-    if (warp >= kWorkWarp0) {
-        // ------------------------------------------------------------ workers
-        const int tid = threadIdx.x - kWorkWarp0 * 32;
+    if (warp >= 1 && warp < 1 + kTernWarps) {
+        // ------------------------------------------------------------ ternarizers / epilogue
+        // Ternarizing: item = (32-channel group, pixel of the tile's sequence), groups outer; a thread
+        // arrives on a group's barrier when its next item lies beyond the group, so nobody idles at
+        // a group's end.  Warps 4..11 then run the epilogue of the tile before: the tensor core works
+        // on tile i while they ternarize tile i+1 (second code buffer) or write out tile i-1.
+        const int tid = (warp - 1) * 32 + lane;
+        const bool epi_warp = warp >= kEpiWarp0;
         const int64_t cs = (int64_t)a.H * a.W;
         const bool per_layer = a.n_thr == 1;
         const float lo0 = sLo[0], hi0 = sHi[0];
-        // filter row of this thread: planes of packed block j are two uint4 at Wrow + 2 j
-        const int cwords = p.Cp / 32;
-        const int64_t row_blocks = ((int64_t)p.T * cwords + 3) / 4;
-        const uint4* Wrow = tid < a.N ? reinterpret_cast<const uint4*>(a.w_packed) + (int64_t)tid * row_blocks * 2
-                                      : nullptr;
-        uint32_t wcount = 0;
-        int it = 0;
-        for (int g = s0; g < s1; g += p.RT, ++it) {
-            const int nrows = min(p.RT, s1 - g);
+        const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
+        const int64_t ostride = (int64_t)a.Ho * a.Wo;
+        const int nblk16 = (a.N + 15) / 16;
+        const int blk_begin = half == 0 ? 0 : (nblk16 + 1) / 2;
+        const int blk_end = half == 0 ? (nblk16 + 1) / 2 : nblk16;
+        for (int step = 0; step <= ntile; ++step) {
+            if (step < ntile) {
+                const int it = step, g = s0 + it * rt;
+                const int nrows = min(rt, s1 - g);
+            const int buf = p.nA == 2 ? (it & 1) : 0;
+            const uint32_t use_ph = p.nA == 2 ? ((it >> 1) & 1) : (it & 1);
+            uint4* sA = reinterpret_cast<uint4*>(smem + (buf ? p.off_a[1] : p.off_a[0]));      // [Cp/16][ppix]
             const int npix = (nrows + p.halo) * p.PW;
-            int* psum = sPsum + (it % 3) * p.ppix;
-            wait_or_die(a_empty, (it & 1) ^ 1, a.status, dead);
-            for (int i = tid; i < p.ppix; i += kWorkThreads) psum[i] = 0;
-            asm volatile("bar.sync %0, %1;" ::"r"(kWorkBarrier), "r"(kWorkThreads) : "memory");
-            // ---- ternarize: item = (pixel of the tile's sequence, pair of 16-channel chunks): 32 loads in flight
-            for (int i = tid; i < (nchunk / 2) * npix; i += kWorkThreads) {
-                const int cp = i / npix, pp = i - cp * npix;
+            int* psum = sPsum + (it & (kPsumRing - 1)) * p.ppix;
+            role_wait(tid < 32, &a_empty[buf], use_ph ^ 1, a.status, dead, kTernBarrier, kTernThreads);
+            for (int i = tid; i < p.ppix; i += kTernThreads) psum[i] = 0;
+            asm volatile("bar.sync %0, %1;" ::"r"(kTernBarrier), "r"(kTernThreads) : "memory");
+            uint64_t* full = &a_full[buf * kMaxGroups];
+            int h = 0, pp = tid, arrived = 0;
+            while (pp >= npix && h < ngroup) { pp -= npix; ++h; }
+            for (; arrived < h && arrived < ngroup; ++arrived) tc::mbar_arrive(&full[arrived]);
+            while (h < ngroup) {
                 const uint32_t sl = fdiv((uint32_t)pp, p.div_pw);
                 const int c = (int)((uint32_t)pp - sl * (uint32_t)p.PW) * p.istride - p.ipad;
                 const uint32_t G = (uint32_t)g + sl;
@@ -208,118 +271,42 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
                 const int r = (int)(G - b * (uint32_t)p.PH) * p.istride - p.ipad;
                 uint4 w0 = make_uint4(0, 0, 0, 0), w1 = make_uint4(0, 0, 0, 0);
                 if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
-                    const float* src = a.x + (((int64_t)b * a.C + cp * 32) * a.H + r) * a.W + c;
+                    const float* src = a.x + (((int64_t)b * a.C + h * 32) * a.H + r) * a.W + c;
                     float v0[16], v1[16];
                     #pragma unroll
                     for (int e = 0; e < 16; ++e) {
-                        v0[e] = (cp * 32 + perm16(e) < a.C) ? __ldg(src + perm16(e) * cs) : 0.0f;
-                        v1[e] = (cp * 32 + 16 + perm16(e) < a.C) ? __ldg(src + (16 + perm16(e)) * cs) : 0.0f;
+                        v0[e] = (h * 32 + perm16(e) < a.C) ? __ldg(src + perm16(e) * cs) : 0.0f;
+                        v1[e] = (h * 32 + 16 + perm16(e) < a.C) ? __ldg(src + (16 + perm16(e)) * cs) : 0.0f;
                     }
-                    w0 = per_layer ? codes16<true>(v0, sLo, sHi, cp * 32, lo0, hi0)
-                                   : codes16<false>(v0, sLo, sHi, cp * 32, lo0, hi0);
-                    w1 = per_layer ? codes16<true>(v1, sLo, sHi, cp * 32 + 16, lo0, hi0)
-                                   : codes16<false>(v1, sLo, sHi, cp * 32 + 16, lo0, hi0);
+                    w0 = per_layer ? codes16<true>(v0, sLo, sHi, h * 32, lo0, hi0)
+                                   : codes16<false>(v0, sLo, sHi, h * 32, lo0, hi0);
+                    w1 = per_layer ? codes16<true>(v1, sLo, sHi, h * 32 + 16, lo0, hi0)
+                                   : codes16<false>(v1, sLo, sHi, h * 32 + 16, lo0, hi0);
                     int s = __dp4a((int)w0.x, 0x01010101, __dp4a((int)w0.y, 0x01010101,
                             __dp4a((int)w0.z, 0x01010101, __dp4a((int)w0.w, 0x01010101, 0))));
                     s = __dp4a((int)w1.x, 0x01010101, __dp4a((int)w1.y, 0x01010101,
                         __dp4a((int)w1.z, 0x01010101, __dp4a((int)w1.w, 0x01010101, s))));
                     if (s != 0) atomicAdd(&psum[pp], s);
                 }
-                sA[(2 * cp) * p.ppix + pp] = w0;
-                sA[(2 * cp + 1) * p.ppix + pp] = w1;
-            }
-            tc::fence_smem_to_async_proxy();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(a_full);
-            // ---- filter slices of this tile, one packed block (four K = 32 slices) per ring stage; slice ks
-            //      is word ks of the packed row.  The next block's planes are fetched while this one expands.
-            uint4 nzn = make_uint4(0, 0, 0, 0), sgn = nzn;
-            if (Wrow != nullptr) { nzn = __ldg(Wrow); sgn = __ldg(Wrow + 1); }
-            for (int ks0 = 0; ks0 < p.nK; ks0 += kSlices, ++wcount) {
-                const uint4 nzv = nzn, sgv = sgn;
-                if (Wrow != nullptr && ks0 + kSlices < p.nK) {
-                    nzn = __ldg(Wrow + 2 * ((ks0 >> 2) + 1));
-                    sgn = __ldg(Wrow + 2 * ((ks0 >> 2) + 1) + 1);
+                sA[(2 * h) * p.ppix + pp] = w0;
+                sA[(2 * h + 1) * p.ppix + pp] = w1;
+                pp += kTernThreads;
+                while (pp >= npix && h < ngroup) { pp -= npix; ++h; }
+                if (arrived < h) {
+                    tc::fence_smem_to_async_proxy();
+                    for (; arrived < h && arrived < ngroup; ++arrived) tc::mbar_arrive(&full[arrived]);
                 }
-                const uint32_t st = wcount % (uint32_t)p.nW;
-                wait_or_die(&w_empty[st], ((wcount / (uint32_t)p.nW) & 1) ^ 1, a.status, dead);
-                if (tid < p.Np) {
-                    uint4* dst = sWr + (size_t)st * kSlices * 2 * p.Np + tid;
-                    uint32_t o[8];
-                    tc::unpack32(nzv.x, sgv.x, o);
-                    dst[0 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[1 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
-                    tc::unpack32(nzv.y, sgv.y, o);
-                    dst[2 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[3 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
-                    tc::unpack32(nzv.z, sgv.z, o);
-                    dst[4 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[5 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
-                    tc::unpack32(nzv.w, sgv.w, o);
-                    dst[6 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[7 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
-                }
-                tc::fence_smem_to_async_proxy();
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&w_full[st]);
             }
-        }
-    } else if (warp == 0) {
-        // ------------------------------------------------------------ MMA issue (one thread)
-        if (lane == 0) {
-            const uint32_t idesc = tc::idesc_i8(kTileM, (uint32_t)p.Np);
-            const uint64_t desc_hi = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
-            const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
-            const uint32_t a16 = (tc::smem_addr(sA) >> 4) + a_lbo_field;
-            const uint32_t w16 = (tc::smem_addr(sWr) >> 4) + ((((uint32_t)p.Np * 16) >> 4) << 16);
-            const uint32_t wslice16 = ((uint32_t)p.Np * 32) >> 4;
-            const uint32_t wstage16 = wslice16 * kSlices;
-            uint32_t wcount = 0;
-            int it = 0;
-            bool alive = true;
-            for (int g = s0; g < s1 && alive; g += p.RT, ++it) {
-                const int acc = p.nAcc == 2 ? (it & 1) : 0;
-                const uint32_t acc_ph = p.nAcc == 2 ? ((it >> 1) & 1) : (it & 1);
-                const int nrows = min(p.RT, s1 - g);
-                const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
-                alive = wait_or_die(a_full, it & 1, a.status, dead) &&
-                        wait_or_die(&acc_empty[acc], acc_ph ^ 1, a.status, dead);
-                if (!alive) break;
-                for (int ks0 = 0; ks0 < p.nK; ks0 += kSlices, ++wcount) {
-                    const uint32_t st = wcount % (uint32_t)p.nW;
-                    if (!wait_or_die(&w_full[st], (wcount / (uint32_t)p.nW) & 1, a.status, dead)) { alive = false; break; }
-                    tc::tc_fence_after_sync();
-                    const int nks = min(kSlices, p.nK - ks0);
-                    for (int j = 0; j < nks; ++j) {
-                        const uint64_t bd = desc_hi | (uint64_t)(w16 + st * wstage16 + (uint32_t)j * wslice16);
-                        const uint32_t aw = a16 + p.tab_a[ks0 + j];
-                        for (int tm = 0; tm < ntm; ++tm) {
-                            const uint32_t d = tmem + (uint32_t)((acc * p.TM + tm) * p.Np);
-                            tc::mma_i8_ss(d, desc_hi | (uint64_t)(aw + (uint32_t)(tm * kTileM)), bd, idesc, ks0 + j > 0);
-                        }
-                    }
-                    tc::mma_commit(&w_empty[st]);
-                }
-                if (!alive) break;
-                tc::mma_commit(a_empty);
-                tc::mma_commit(&acc_full[acc]);
             }
-        }
-    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
-        // ------------------------------------------------------------ epilogue: out = c1*S_xw + c2*S_x + c3
-        const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
-        const int64_t ostride = (int64_t)a.Ho * a.Wo;
-        const int nblk16 = (a.N + 15) / 16;
-        const int blk_begin = half == 0 ? 0 : (nblk16 + 1) / 2;
-        const int blk_end = half == 0 ? (nblk16 + 1) / 2 : nblk16;
-        int it = 0;
-        for (int g = s0; g < s1; g += p.RT, ++it) {
+            if (step >= 1 && epi_warp) {
+                const int it = step - 1, g = s0 + it * rt;
+                const int nrows = min(rt, s1 - g);
             const int acc = p.nAcc == 2 ? (it & 1) : 0;
             const uint32_t acc_ph = p.nAcc == 2 ? ((it >> 1) & 1) : (it & 1);
-            const int nrows = min(p.RT, s1 - g);
             const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
-            const int* psum = sPsum + (it % 3) * p.ppix;
-            const bool alive = wait_or_die(&acc_full[acc], acc_ph, a.status, dead);
+            const int* psum = sPsum + (it & (kPsumRing - 1)) * p.ppix;
+            role_wait(warp == kEpiWarp0, &acc_full[acc], acc_ph, a.status, dead, kEpiBarrier, kEpiThreads);
+            const bool alive = !*dead;
             tc::tc_fence_after_sync();
             for (int tm = 0; tm < ntm; ++tm) {
                 const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);
@@ -385,6 +372,127 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[acc]);
+            }
+        }
+    } else if (warp >= kExpWarp0 && warp < kExpWarp0 + kExpWarps) {
+        // ------------------------------------------------------------ filter expanders
+        // thread = filter row; a stage = one packed block of the row (four K = 32 slices).  The
+        // planes of the next two stages are in flight while this one expands.
+        const int tid = threadIdx.x - kExpWarp0 * 32;
+        const int cwords = p.Cp / 32;
+        const int64_t row_blocks = ((int64_t)p.T * cwords + 3) / 4;
+        const uint4* Wrow = tid < a.N ? reinterpret_cast<const uint4*>(a.w_packed) + (int64_t)tid * row_blocks * 2
+                                      : nullptr;
+        const int cblocks = cwords / kSlices;
+        auto block_of = [&](int st) {
+            if (!p.blocks_major) return st;
+            const int cb = (int)fdiv((uint32_t)st, p.div_T), t = st - cb * p.T;
+            return t * cblocks + cb;
+        };
+        uint32_t wcount = 0;
+        for (int it = 0; it < ntile; ++it) {
+            uint4 nz1 = make_uint4(0, 0, 0, 0), sg1 = nz1, nz2 = nz1, sg2 = nz1;
+            if (Wrow != nullptr) {
+                const int b0 = block_of(0);
+                nz1 = __ldg(Wrow + 2 * b0); sg1 = __ldg(Wrow + 2 * b0 + 1);
+                if (nstages > 1) { const int b1 = block_of(1); nz2 = __ldg(Wrow + 2 * b1); sg2 = __ldg(Wrow + 2 * b1 + 1); }
+            }
+            for (int s = 0; s < nstages; ++s, ++wcount) {
+                const uint4 nzv = nz1, sgv = sg1;
+                nz1 = nz2; sg1 = sg2;
+                if (Wrow != nullptr && s + 2 < nstages) {
+                    const int b2 = block_of(s + 2);
+                    nz2 = __ldg(Wrow + 2 * b2); sg2 = __ldg(Wrow + 2 * b2 + 1);
+                }
+                const uint32_t st = wcount % (uint32_t)p.nW;
+                role_wait(tid < 32, &w_empty[st], ((wcount / (uint32_t)p.nW) & 1) ^ 1, a.status, dead, kExpBarrier,
+                          kExpThreads);
+                if (tid < p.Np) {
+                    uint4* dst = sWr + (size_t)st * kSlices * 2 * p.Np + tid;
+                    uint32_t o[8];
+                    tc::unpack32(nzv.x, sgv.x, o);
+                    dst[0 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[1 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(nzv.y, sgv.y, o);
+                    dst[2 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[3 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(nzv.z, sgv.z, o);
+                    dst[4 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[5 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                    tc::unpack32(nzv.w, sgv.w, o);
+                    dst[6 * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[7 * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+                tc::fence_smem_to_async_proxy();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&w_full[st]);
+            }
+        }
+    } else if (warp == 0) {
+        // ------------------------------------------------------------ MMA issue (one thread)
+        // The tensor core's queue is short, so whatever the issuing thread does between two MMAs is
+        // tensor-core idle time: the A offsets of a stage are fetched one stage ahead.
+        if (lane == 0) {
+            const uint32_t idesc = tc::idesc_i8(kTileM, (uint32_t)p.Np);
+            const uint64_t desc_hi = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
+            const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
+            const uint32_t w16 = (tc::smem_addr(sWr) >> 4) + ((((uint32_t)p.Np * 16) >> 4) << 16);
+            const uint32_t wslice16 = ((uint32_t)p.Np * 32) >> 4;
+            const uint32_t wstage16 = wslice16 * kSlices;
+            uint32_t wcount = 0;
+            int it = 0;
+            bool alive = true;
+            for (int g = s0; g < s1 && alive; g += rt, ++it) {
+                const int buf = p.nA == 2 ? (it & 1) : 0;
+                const uint32_t use_ph = p.nA == 2 ? ((it >> 1) & 1) : (it & 1);
+                const int acc = p.nAcc == 2 ? (it & 1) : 0;
+                const uint32_t acc_ph = p.nAcc == 2 ? ((it >> 1) & 1) : (it & 1);
+                const int nrows = min(rt, s1 - g);
+                const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
+                const uint32_t a16 = (tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4) + a_lbo_field;
+                uint64_t* full = &a_full[buf * kMaxGroups];
+                alive = wait_or_die(&acc_empty[acc], acc_ph ^ 1, a.status, dead);
+                if (!alive) break;
+                uint32_t ta[kSlices], tn[kSlices];
+                #pragma unroll
+                for (int j = 0; j < kSlices; ++j) tn[j] = p.tab_a[j];
+                uint32_t ready = 0;             // 32-channel groups whose codes are known to be written
+                bool accum = false;
+                for (int s = 0; s < nstages && alive; ++s, ++wcount) {
+                    #pragma unroll
+                    for (int j = 0; j < kSlices; ++j) {
+                        ta[j] = tn[j];
+                        tn[j] = p.tab_a[min((s + 1) * kSlices + j, p.nK - 1)];
+                    }
+                    const uint32_t st = wcount % (uint32_t)p.nW;
+                    if (!wait_or_die(&w_full[st], (wcount / (uint32_t)p.nW) & 1, a.status, dead)) { alive = false; break; }
+                    tc::tc_fence_after_sync();
+                    #pragma unroll
+                    for (int j = 0; j < kSlices; ++j) {
+                        if (ta[j] != 0xFFFFFFFFu && alive) {
+                            const uint32_t h = ta[j] >> 24;
+                            if (!((ready >> h) & 1u)) {
+                                alive = wait_or_die(&full[h], use_ph, a.status, dead);
+                                tc::tc_fence_after_sync();
+                                ready |= 1u << h;
+                            }
+                            if (alive) {
+                                const uint64_t bd = desc_hi | (uint64_t)(w16 + st * wstage16 + (uint32_t)j * wslice16);
+                                const uint32_t aw = a16 + (ta[j] & 0xFFFFFFu);
+                                tc::mma_i8_ss(tmem + (uint32_t)((acc * p.TM) * p.Np), desc_hi | (uint64_t)aw, bd, idesc, accum);
+                                if (ntm == 2)
+                                    tc::mma_i8_ss(tmem + (uint32_t)((acc * p.TM + 1) * p.Np),
+                                                  desc_hi | (uint64_t)(aw + (uint32_t)kTileM), bd, idesc, accum);
+                                accum = true;
+                            }
+                        }
+                    }
+                    if (alive) tc::mma_commit(&w_empty[st]);
+                }
+                if (!alive) break;
+                tc::mma_commit(&a_empty[buf]);
+                tc::mma_commit(&acc_full[acc]);
+            }
         }
     }
     tc::tc_fence_before_sync();
