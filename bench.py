@@ -136,11 +136,15 @@ class ClockSampler:
 
 
 def algorithmic_bytes(case):
-    """Bytes the method must move per step: fp32 input once, fp32 output once, packed weights once."""
+    """Bytes the method must move per step: the fp32 input it touches once, fp32 output once, packed weights once."""
     if isinstance(case, inputs.ConvCase):
         M, N, K = case.gemm_mnk
         kc = case.kh * case.kw * ((case.C + 31) // 32 * 32)
-        return case.x.nbytes + 4 * M * N + N * ((kc + 127) // 128) * 32
+        # input pixels some filter tap lands on (a strided 1x1 layer touches a fraction of them)
+        rows = {ho * case.stride - case.pad + i for ho in range(case.Ho) for i in range(case.kh)}
+        cols = {wo * case.stride - case.pad + j for wo in range(case.Wo) for j in range(case.kw)}
+        touched = len([r for r in rows if 0 <= r < case.H]) * len([c for c in cols if 0 <= c < case.W])
+        return 4 * case.B * case.C * touched + 4 * M * N + N * ((kc + 127) // 128) * 32
     M, N, K = case.M, case.N, case.K
     packed = lambda r: r * ((K + 127) // 128) * 32
     # ternarize+pack: read fp32, write planes; GEMM: read both packed operands, write fp32

@@ -50,11 +50,23 @@ struct GemmI8Plan {
 bool make_gemm_plan(int64_t M, int64_t N, int64_t K, GemmI8Plan& p, int sms)
 {
     if (M < 1 || N < 1 || K < 1) return false;
-    p.BN = (int)((N >= 256) ? 256 : (N + 15) / 16 * 16);
-    p.TM = 2;
-    auto ntiles = [&](int tm, int bn) { return ((M + 128 * tm - 1) / (128 * tm)) * ((N + bn - 1) / bn); };
-    if (ntiles(p.TM, p.BN) < 2 * sms) p.TM = 1;
-    if (ntiles(p.TM, p.BN) < sms && p.BN > 128) p.BN = 128;
+    // Tile shape by a cost model: a K = 128 stage costs the slower of its MMAs (2 TM BN cycles) and of
+    // expanding its rows from bit planes (about 4 cycles per row of A or W; this is what binds), and
+    // a CTA runs ceil(tiles / SMs) tiles.  Larger tiles expand fewer rows per MAC, smaller ones
+    // fill the machine more evenly.
+    const int bn_full = (int)((N >= 256) ? 256 : (N + 15) / 16 * 16);
+    double best = 0.0;
+    p.TM = 2; p.BN = bn_full;
+    for (int tm = 2; tm >= 1; --tm) {
+        for (int bn = bn_full; bn >= 128 || bn == bn_full; bn = (bn > 128 ? 128 : 0)) {
+            const int64_t nt = ((M + 128 * tm - 1) / (128 * tm)) * ((N + bn - 1) / bn);
+            const int64_t rounds = (nt + sms - 1) / sms;
+            const double mma = 2.0 * tm * bn, expand = 4.0 * (128 * tm + bn);
+            const double cost = (double)rounds * (mma > expand ? mma : expand);
+            if (best == 0.0 || cost < best) { best = cost; p.TM = tm; p.BN = bn; }
+            if (bn <= 128) break;
+        }
+    }
     p.nAcc = (2 * p.TM * p.BN <= 512) ? 2 : 1;
     p.tiles_m = (M + 128 * p.TM - 1) / (128 * p.TM);
     p.tiles_n = (N + p.BN - 1) / p.BN;
