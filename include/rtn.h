@@ -119,7 +119,14 @@ rtn_status rtn_ternary_gemm(const void* a_packed, const int32_t* a_sum,
  *   a_scale,a_offset  per-layer gamma, beta (by value); w_scale,w_offset as in the GEMM
  *   out      fp32 [B][N][Ho][Wo], Ho = rtn_conv_out_dim(H,kh,stride,pad), same for Wo
  *   dbg_acc  NULL, or int32 of out's shape that receives the raw S_xw
- * out[b][n][ho][wo] = sum over taps of (a_s*x + a_o)*(w_s*w + w_o) under pad_mode's rule. */
+ * out[b][n][ho][wo] = sum over taps of (a_s*x + a_o)*(w_s*w + w_o) under pad_mode's rule.
+ * Stream order: x, out and dbg_acc are ordered after all earlier work of the stream, as usual.  The
+ * tensor-core kernels start their set-up while the stream's previous kernel is still draining
+ * (programmatic dependent launch), and that set-up reads the layer's parameters: t_lo, t_hi,
+ * w_packed, w_sum, w_scale, w_offset must therefore not be buffers that an earlier
+ * rtn_ternary_conv2d call of the same stream writes (its out or dbg_acc), unless the stream was
+ * synchronized or ran another kernel in between (they are constants of the layer in every intended
+ * use). */
 rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
                               const float* t_lo, const float* t_hi, int64_t n_thr,
                               const void* w_packed, const int32_t* w_sum,
