@@ -281,7 +281,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         asm volatile("bar.sync %0, %1;" ::"r"(kConvBarrier), "r"(kConvThreads) : "memory");
         if (!p.use_tma) tc::pdl_wait();             // the direct path reads x
         const int64_t cs = (int64_t)a.H * a.W;
-        const bool per_layer = a.n_thr == 1;
+        const bool per_layer = a.n_thr == 1 && a.C == p.Cp;     // padding channels need their own (infinite) thresholds
         const int ngroup = p.Cp / 32;
         const float lo0 = sLo[0], hi0 = sHi[0];
         uint32_t st_count = 0;                                 // batches consumed so far

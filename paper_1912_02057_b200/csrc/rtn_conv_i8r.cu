@@ -1,0 +1,539 @@
+// Ternary conv2d, tensor-core variant for stride-1 layers with more than 256 filters or a filter bank
+// the other variants cannot hold (e.g. 512 -> 512, 3x3): two kernels and a scratch buffer of int8
+// codes.  (On 256 -> 256, 3x3 it runs at 44 us against 38 us of the streamed-filter kernel, which
+// therefore keeps that shape.)
+//
+//   conv_codes_kernel   ternarizes the fp32 NCHW input once (Eq. 3) into int8 codes {-1,0,+1} laid out
+//                       [16-channel chunk][padded pixel][16 B] over the whole batch, zero padding
+//                       included, plus the per-pixel code sum over all channels.  4 B read and
+//                       about 1 B written per value: a stream through HBM.
+//   conv_i8r_kernel     implicit GEMM on the codes.  The filter bank is SPLIT over CTAs: a CTA keeps
+//                       the int8 expansion of N/S filters (all taps, all channels) resident in shared
+//                       memory for its whole life and walks pixel tiles; the S CTAs of a tile each
+//                       produce their share of the output channels.  Nothing is expanded in the main
+//                       loop (a streamed filter bank costs a quarter of the SM's integer pipe per
+//                       tile and paces the tensor core) and the fp32 input is ternarized once, not
+//                       once per filter group.
+//
+// The code layout in the scratch buffer is the shared-memory operand layout, so a tile's window of
+// one 16-channel chunk is one contiguous run of bytes: the producer moves it with one bulk
+// asynchronous copy (cp.async.bulk, completion counted on an mbarrier; no tensor map, no multicast).
+// Shifted-window implicit GEMM as in the other conv kernels: tap (i, j) reads the same rows of
+// shared memory from a start shifted by i*PW + j pixels.  K loop: 32-channel group outer, tap inner;
+// unit of the pipeline = (tile, group) = two chunk windows in one ring slot, 9 MMAs for a 3x3 filter.
+// S_x of a pixel = sum over the taps of the per-pixel code sums (read from the scratch buffer in
+// the epilogue), so all accumulator columns are output channels.
+//
+// Roles of conv_i8r_kernel (384 threads): warp 0 issues MMAs (one thread), warp 1 issues the bulk
+// copies (one thread), warps 4..11 epilogue; all threads expand the CTA's filters at set-up, which
+// overlaps the code kernel through programmatic dependent launch.
+#include "rtn_internal.cuh"
+#include "rtn_tcgen05.cuh"
+#include "rtn_conv_i8_common.cuh"
+
+namespace rtn {
+
+namespace {
+
+using namespace conv_detail;
+
+constexpr int kTileM = 128;
+constexpr int kEpiWarp0 = 4;
+constexpr int kEpiWarps = 8;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kThreads = (kEpiWarp0 + kEpiWarps) * 32;
+constexpr int kMaxSlots = 16;
+constexpr int kMaxAcc = 4;
+constexpr int kMaxTaps = 25;
+constexpr int kMaxSplit = 32;                          // filter groups at most
+constexpr size_t kSmemLimit = 220 * 1024;
+constexpr int kEpiBarrier = 1;
+constexpr int kCodePixels = 64;                        // pixels per block of the code kernel
+constexpr int kCodeGroups = 8;                         // 32-channel groups it works on at a time
+
+struct ConvI8RPlan {
+    int PW, PH;            // padded row length / rows per image
+    int Cp, T, halo, RT;   // channels rounded to 32, taps, kh-1, padded rows per tile
+    int ppix;              // pixels of a slot's window: 128 + halo*PW + kw-1, rounded up to 8
+    int total_rows, ntiles;
+    int S, Nq;             // filter groups; filters per group (multiple of 16)
+    int cpg, grid;         // CTAs per filter group; grid = S * cpg
+    int ngroup;            // 32-channel groups
+    int gps;               // groups per ring slot (2 when their number is even: fewer hand-offs)
+    int nslots, nAcc;
+    uint32_t tmem_cols;
+    int64_t Ptot, Pstride; // padded pixels of the batch; pixels per chunk row of the scratch (with slack)
+    FastDiv div_pw, div_ph, div_nq, div_cw;
+    uint32_t off_w, off_c, off_bar, off_misc, off_slot, slot_bytes;
+    size_t smem_bytes;
+    size_t codes_bytes, scratch_bytes;     // scratch = codes, then the per-pixel sums
+    uint32_t tap_shift[kMaxTaps];          // i*PW + j
+};
+
+bool make_plan_r(const ConvArgs& c, ConvI8RPlan& p, int sms)
+{
+    if (c.stride != 1) return false;
+    if (c.Ho <= 0 || c.Wo <= 0) return false;
+    p.T = c.kh * c.kw;
+    if (p.T > kMaxTaps) return false;
+    p.PW = c.W + 2 * c.pad;
+    p.PH = c.H + 2 * c.pad;
+    if (p.PW > kTileM || p.PH > 2048) return false;
+    if ((int64_t)c.B * p.PH > (1 << 20)) return false;
+    p.Cp = (c.C + 31) / 32 * 32;
+    p.ngroup = p.Cp / 32;
+    if (p.ngroup > 16) return false;
+    p.halo = c.kh - 1;
+    p.RT = kTileM / p.PW;
+    p.ppix = (kTileM + p.halo * p.PW + (c.kw - 1) + 7) / 8 * 8;
+    p.total_rows = c.B * p.PH;
+    p.ntiles = (p.total_rows + p.RT - 1) / p.RT;
+    p.Ptot = (int64_t)p.total_rows * p.PW;
+    p.Pstride = p.Ptot + p.ppix;
+    p.gps = (p.ngroup % 2 == 0) ? 2 : 1;
+    p.slot_bytes = (uint32_t)p.gps * 2u * (uint32_t)p.ppix * 16u;
+    p.div_pw = make_fastdiv((uint32_t)p.PW);
+    p.div_ph = make_fastdiv((uint32_t)p.PH);
+    p.div_cw = make_fastdiv((uint32_t)p.ngroup);
+    for (int t = 0; t < p.T; ++t) p.tap_shift[t] = (uint32_t)((t / c.kw) * p.PW + (t % c.kw));
+    // fewest filter groups whose share of the bank leaves room for a ring of at least four slots
+    for (p.S = 1; p.S <= kMaxSplit; p.S *= 2) {
+        if (p.S > sms) return false;
+        p.Nq = ((c.N + p.S - 1) / p.S + 15) / 16 * 16;
+        if (p.Nq > 256) continue;
+        uint32_t o = 0;
+        p.off_w = o;    o += (uint32_t)p.T * (uint32_t)(p.Cp / 16) * (uint32_t)p.Nq * 16u;
+        p.off_c = o;    o += (uint32_t)p.Nq * 16u;
+        p.off_bar = o;  o += (2 * kMaxSlots + 2 * kMaxAcc + 1) * 8;
+        p.off_misc = o; o += 16;
+        o = (o + 127) / 128 * 128;
+        p.off_slot = o;
+        if (o >= kSmemLimit) continue;
+        int ns = (int)((kSmemLimit - o) / p.slot_bytes);
+        if (ns > kMaxSlots) ns = kMaxSlots;
+        if (ns < 4) continue;
+        p.nslots = ns;
+        p.smem_bytes = o + (size_t)ns * p.slot_bytes;
+        break;
+    }
+    if (p.S > kMaxSplit) return false;
+    p.div_nq = make_fastdiv((uint32_t)p.Nq);
+    p.cpg = sms / p.S;
+    if (p.cpg > p.ntiles) p.cpg = p.ntiles;
+    if (p.cpg < 1) return false;
+    p.grid = p.S * p.cpg;
+    p.nAcc = 512 / p.Nq < kMaxAcc ? 512 / p.Nq : kMaxAcc;
+    uint32_t cols = 32;
+    while (cols < (uint32_t)(p.nAcc * p.Nq)) cols *= 2;
+    p.tmem_cols = cols;
+    p.codes_bytes = (size_t)(p.Cp / 16) * (size_t)p.Pstride * 16;
+    p.scratch_bytes = p.codes_bytes + ((size_t)p.Pstride * 4 + 255) / 256 * 256;
+    return true;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Kernel 1: fp32 NCHW -> int8 codes [chunk][padded pixel][16 B] + per-pixel code sums.
+// Block = 64 consecutive padded pixels x up to 8 channel groups; lanes run along pixels, so the
+// loads of one channel are coalesced along an image row and the 16-byte code stores are contiguous.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kCodePixels * kCodeGroups)
+conv_codes_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, uint4* __restrict__ codes,
+                  int* __restrict__ psum)
+{
+    extern __shared__ __align__(16) uint8_t smem_c[];
+    float* sLo = reinterpret_cast<float*>(smem_c);
+    float* sHi = sLo + p.Cp;
+    int* sSum = reinterpret_cast<int*>(sHi + p.Cp);            // [kCodeGroups][kCodePixels]
+    tc::pdl_trigger();          // the contraction kernel may start its set-up (it reads no codes there)
+    for (int c = threadIdx.x; c < p.Cp; c += blockDim.x) {
+        float lo = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
+        const float hi = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
+        if (lo > hi) lo = nextafterf(hi, INFINITY);      // v < lo  <=>  v <= hi: -1 unless +1
+        sLo[c] = lo;
+        sHi[c] = hi;
+    }
+    __syncthreads();
+    const int px = threadIdx.x % kCodePixels, gi = threadIdx.x / kCodePixels;
+    const int64_t P = (int64_t)blockIdx.x * kCodePixels + px;
+    const bool per_layer = a.n_thr == 1 && a.C == p.Cp;     // padding channels need their own (infinite) thresholds
+    const float lo0 = sLo[0], hi0 = sHi[0];
+    const int64_t cs = (int64_t)a.H * a.W;
+    // padded pixel -> (image, row, column) of the input, if any
+    bool inside = false;
+    const float* src0 = nullptr;
+    if (P < p.Ptot) {
+        const uint32_t G = fdiv((uint32_t)P, p.div_pw);
+        const int col = (int)((uint32_t)P - G * (uint32_t)p.PW) - a.pad;
+        const uint32_t b = fdiv(G, p.div_ph);
+        const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
+        inside = r >= 0 && r < a.H && col >= 0 && col < a.W;
+        if (inside) src0 = a.x + (((int64_t)b * a.C) * a.H + r) * a.W + col;
+    }
+    int sum = 0;
+    for (int h = gi; h < p.ngroup; h += kCodeGroups) {
+        uint4 w0 = make_uint4(0, 0, 0, 0), w1 = make_uint4(0, 0, 0, 0);
+        if (inside) {
+            const float* src = src0 + (int64_t)(h * 32) * cs;
+            float v0[16], v1[16];
+            #pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                v0[e] = (h * 32 + perm16(e) < a.C) ? __ldg(src + perm16(e) * cs) : 0.0f;
+                v1[e] = (h * 32 + 16 + perm16(e) < a.C) ? __ldg(src + (16 + perm16(e)) * cs) : 0.0f;
+            }
+            w0 = per_layer ? codes16<true>(v0, sLo, sHi, h * 32, lo0, hi0)
+                           : codes16<false>(v0, sLo, sHi, h * 32, lo0, hi0);
+            w1 = per_layer ? codes16<true>(v1, sLo, sHi, h * 32 + 16, lo0, hi0)
+                           : codes16<false>(v1, sLo, sHi, h * 32 + 16, lo0, hi0);
+            sum = __dp4a((int)w0.x, 0x01010101, __dp4a((int)w0.y, 0x01010101,
+                  __dp4a((int)w0.z, 0x01010101, __dp4a((int)w0.w, 0x01010101, sum))));
+            sum = __dp4a((int)w1.x, 0x01010101, __dp4a((int)w1.y, 0x01010101,
+                  __dp4a((int)w1.z, 0x01010101, __dp4a((int)w1.w, 0x01010101, sum))));
+        }
+        if (P < p.Pstride) {
+            codes[(int64_t)(2 * h) * p.Pstride + P] = w0;
+            codes[(int64_t)(2 * h + 1) * p.Pstride + P] = w1;
+        }
+    }
+    sSum[gi * kCodePixels + px] = sum;
+    __syncthreads();
+    if (gi == 0 && P < p.Pstride) {
+        int s = 0;
+        for (int k = 0; k < kCodeGroups; ++k) s += sSum[k * kCodePixels + px];
+        psum[P] = s;
+    }
+}
+
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_r(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                 ::"r"(tc::smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void role_wait_r(bool leader, uint64_t* bar, uint32_t parity, unsigned* status,
+                                            volatile int* dead, int barrier_id, int nthreads)
+{
+    if (leader) wait_or_die(bar, parity, status, dead);
+    asm volatile("bar.sync %0, %1;" ::"r"(barrier_id), "r"(nthreads) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// Kernel 2: the contraction and the epilogue.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const uint4* __restrict__ codes,
+                const int* __restrict__ psum)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint4* sW = reinterpret_cast<uint4*>(smem + p.off_w);        // [T][Cp/16][Nq]
+    float4* sC = reinterpret_cast<float4*>(smem + p.off_c);     // {c1, c2, c3, 0} per column
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
+    uint64_t* slot_full = bars;                     // [kMaxSlots] bulk copies -> MMA
+    uint64_t* slot_empty = bars + kMaxSlots;        // [kMaxSlots] MMA -> producer
+    uint64_t* acc_full = bars + 2 * kMaxSlots;      // [kMaxAcc] MMA -> epilogue
+    uint64_t* acc_empty = acc_full + kMaxAcc;       // [kMaxAcc] epilogue -> MMA
+    uint32_t* slot = reinterpret_cast<uint32_t*>(smem + p.off_misc);
+    volatile int* dead = reinterpret_cast<volatile int*>(smem + p.off_misc + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nchunk = p.Cp / 16;
+    const int fq = blockIdx.x % p.S;                 // filter group of this CTA
+    const int first_tile = blockIdx.x / p.S;         // it takes tiles first_tile, first_tile + cpg, ...
+    const int n_base = fq * p.Nq;
+
+    // ---------------------------------------------------------------- set-up (all threads)
+    tc::pdl_trigger();
+    if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
+    if (threadIdx.x == 32) {
+        for (int i = 0; i < kMaxSlots; ++i) { tc::mbar_init(&slot_full[i], 1); tc::mbar_init(&slot_empty[i], 1); }
+        for (int i = 0; i < kMaxAcc; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kEpiThreads); }
+        tc::mbar_init_fence();
+        *dead = 0;
+    }
+    {   // this group's filters: bit planes -> int8, [tap][chunk][row]; rows beyond N are zero.
+        // item = (32-channel word of a tap, filter row); six items' loads in flight per thread
+        const int cwords = p.ngroup;
+        const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
+        const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
+        const int items = p.T * cwords * p.Nq;
+        constexpr int kBatch = 6;
+        for (int base = threadIdx.x; base < items; base += kBatch * kThreads) {
+            uint32_t nz[kBatch], sg[kBatch];
+            #pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int i = base + u * kThreads;
+                nz[u] = 0; sg[u] = 0;
+                if (i < items) {
+                    const int wd = (int)fdiv((uint32_t)i, p.div_nq), r = i - wd * p.Nq;
+                    const int n = n_base + r;
+                    if (n < a.N) {
+                        const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
+                        nz[u] = __ldg(blk + (wd & 3));
+                        sg[u] = __ldg(blk + 4 + (wd & 3));
+                    }
+                }
+            }
+            #pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int i = base + u * kThreads;
+                if (i < items) {
+                    const int wd = (int)fdiv((uint32_t)i, p.div_nq), r = i - wd * p.Nq;
+                    const int t = (int)fdiv((uint32_t)wd, p.div_cw), cw = wd - t * cwords;
+                    uint32_t o[8];
+                    tc::unpack32(nz[u], sg[u], o);
+                    uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Nq + r);
+                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[p.Nq] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+            }
+        }
+    }
+    {   // per-output-channel constants in double, rounded once:
+        //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
+        const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
+        for (int r = threadIdx.x; r < p.Nq; r += kThreads) {
+            const int n = n_base + r;
+            float c1 = 0.f, c2 = 0.f, c3 = 0.f;
+            if (n < a.N) {
+                const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
+                const double wo = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
+                c1 = (float)(a_s * ws);
+                c2 = (float)(a_s * wo);
+                c3 = (float)(a_o * (ws * (double)a.w_sum[n] + (double)a.C * p.T * wo));
+            }
+            sC[r] = make_float4(c1, c2, c3, 0.f);
+        }
+    }
+    tc::fence_smem_to_async_proxy();
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem = *slot;
+    tc::pdl_wait();         // from here on: the codes and sums of the code kernel, and out
+
+    if (warp == 1) {
+        // ------------------------------------------------------------ producer (one thread)
+        if (lane == 0) {
+            const uint32_t ring = tc::smem_addr(smem + p.off_slot);
+            const uint32_t win_bytes = (uint32_t)p.ppix * 16u;
+            uint32_t s = 0, ph = 0;             // ring slot and its phase
+            bool alive = true;
+            for (int tile = first_tile; tile < p.ntiles && alive; tile += p.cpg) {
+                const int64_t P0 = (int64_t)tile * p.RT * p.PW;
+                for (int h = 0; h < p.ngroup; h += p.gps) {
+                    if (!wait_or_die(&slot_empty[s], ph ^ 1, a.status, dead)) { alive = false; break; }
+                    mbar_expect_tx_r(&slot_full[s], (uint32_t)(2 * p.gps) * win_bytes);
+                    const uint32_t dst = ring + s * p.slot_bytes, bar = tc::smem_addr(&slot_full[s]);
+                    for (int c = 0; c < 2 * p.gps; ++c)
+                        bulk_copy_g2s(dst + (uint32_t)c * win_bytes, codes + (int64_t)(2 * h + c) * p.Pstride + P0, win_bytes, bar);
+                    if (++s == (uint32_t)p.nslots) { s = 0; ph ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 0) {
+        // ------------------------------------------------------------ MMA issue (one thread)
+        if (lane == 0) {
+            const uint32_t idesc = tc::idesc_i8(kTileM, (uint32_t)p.Nq);
+            const uint64_t desc_hi = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
+            const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
+            const uint32_t ring16 = (tc::smem_addr(smem + p.off_slot) >> 4) + a_lbo_field;
+            const uint32_t slot16 = p.slot_bytes >> 4;
+            const uint32_t w16 = (tc::smem_addr(sW) >> 4) + ((((uint32_t)p.Nq * 16) >> 4) << 16);
+            const uint32_t wtap16 = (uint32_t)nchunk * (uint32_t)p.Nq;      // 16-byte units between taps
+            // up to nine taps keep their operand offsets in registers: nothing but arithmetic between MMAs
+            const bool taps_in_regs = p.T <= 9;
+            uint32_t ta[9], tb[9];
+            #pragma unroll
+            for (int t = 0; t < 9; ++t) {
+                ta[t] = taps_in_regs && t < p.T ? p.tap_shift[t] : 0u;
+                tb[t] = (uint32_t)t * wtap16;
+            }
+            // The tensor core's queue is short: whatever this thread does between two MMAs is idle time
+            // for it.  So no division in the loop (slot, phase and accumulator advance by increments),
+            // and the next unit's barrier is tested before this unit's MMAs are issued: the producer
+            // runs slots ahead, the test succeeds, and the next unit issues without a wait.
+            uint32_t s = 0, ph = 0;             // ring slot and its phase
+            int acc = 0;
+            uint32_t acc_ph = 0;
+            bool alive = true, have = false;    // have: slot s is known to be full
+            for (int tile = first_tile; tile < p.ntiles && alive; tile += p.cpg) {
+                if (!wait_or_die(&acc_empty[acc], acc_ph ^ 1, a.status, dead)) break;
+                const uint32_t d = tmem + (uint32_t)(acc * p.Nq);
+                for (int h0 = 0; h0 < p.ngroup && alive; h0 += p.gps) {
+                    if (!have && !wait_or_die(&slot_full[s], ph, a.status, dead)) { alive = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint32_t s_cur = s;
+                    if (++s == (uint32_t)p.nslots) { s = 0; ph ^= 1; }
+                    have = tc::mbar_test(&slot_full[s], ph);
+                  for (int hh = 0; hh < p.gps; ++hh) {
+                    const int h = h0 + hh;
+                    const uint32_t ag = ring16 + s_cur * slot16 + (uint32_t)(2 * hh) * (uint32_t)p.ppix;
+                    const uint32_t bg = w16 + (uint32_t)(2 * h) * (uint32_t)p.Nq;
+                    if (p.T == 9) {
+                        // straight-line issue: one predicate set-up, then nothing but the MMAs
+                        tc::mma_i8_ss(d, desc_hi | (uint64_t)(ag + ta[0]), desc_hi | (uint64_t)(bg + tb[0]), idesc, h > 0);
+                        #pragma unroll
+                        for (int t = 1; t < 9; ++t)
+                            tc::mma_i8_ss_acc(d, desc_hi | (uint64_t)(ag + ta[t]), desc_hi | (uint64_t)(bg + tb[t]), idesc);
+                    } else if (taps_in_regs) {
+                        #pragma unroll
+                        for (int t = 0; t < 9; ++t)
+                            if (t < p.T)
+                                tc::mma_i8_ss(d, desc_hi | (uint64_t)(ag + ta[t]), desc_hi | (uint64_t)(bg + tb[t]), idesc,
+                                              h > 0 || t > 0);
+                    } else {
+                        for (int t = 0; t < p.T; ++t)
+                            tc::mma_i8_ss(d, desc_hi | (uint64_t)(ag + p.tap_shift[t]),
+                                          desc_hi | (uint64_t)(bg + (uint32_t)t * wtap16), idesc, h > 0 || t > 0);
+                    }
+                  }
+                    tc::mma_commit(&slot_empty[s_cur]);
+                }
+                if (!alive) break;
+                tc::mma_commit(&acc_full[acc]);
+                if (++acc == p.nAcc) { acc = 0; acc_ph ^= 1; }
+            }
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ------------------------------------------------------------ epilogue: out = c1*S_xw + c2*S_x + c3
+        const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
+        const int64_t ostride = (int64_t)a.Ho * a.Wo;
+        const int nblk16 = p.Nq / 16;
+        const int blk_begin = half == 0 ? 0 : (nblk16 + 1) / 2;
+        const int blk_end = half == 0 ? (nblk16 + 1) / 2 : nblk16;
+        int acc = 0;
+        uint32_t acc_ph = 0;
+        for (int tile = first_tile; tile < p.ntiles; tile += p.cpg) {
+            const int g = tile * p.RT;
+            const int nrows = min(p.RT, p.total_rows - g);
+            role_wait_r(warp == kEpiWarp0, &acc_full[acc], acc_ph, a.status, dead, kEpiBarrier, kEpiThreads);
+            const bool alive = !*dead;
+            tc::tc_fence_after_sync();
+            const uint32_t pl = (uint32_t)(q * 32 + lane);         // pixel within the tile
+            const uint32_t row = fdiv(pl, p.div_pw);
+            const int wo = (int)(pl - row * (uint32_t)p.PW);
+            const uint32_t G = (uint32_t)g + row;
+            const uint32_t b = fdiv(G, p.div_ph);
+            const int ho = (int)(G - b * (uint32_t)p.PH);
+            const bool ok = alive && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
+            int n_inside = p.T, s_x = 0;
+            if (ok) {
+                const int* ps = psum + (int64_t)g * p.PW + pl;
+                for (int t = 0; t < p.T; ++t) s_x += __ldg(ps + p.tap_shift[t]);
+                if (a.pad_mode == RTN_PAD_VALUE_ZERO) {
+                    n_inside = 0;
+                    for (int t = 0; t < p.T; ++t) {
+                        const int h = ho - a.pad + t / a.kw, v = wo - a.pad + t % a.kw;
+                        n_inside += (h >= 0 && h < a.H && v >= 0 && v < a.W);
+                    }
+                }
+            }
+            const bool border = n_inside < p.T;
+            const float fsx = (float)s_x;
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.Nq);
+            const int64_t obase = (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
+            for (int blk = blk_begin; blk < blk_end; ++blk) {
+                uint32_t v[16];
+                tc::tmem_ld16(trow + (uint32_t)(blk * 16), v);
+                tc::tmem_ld_wait();
+                if (!ok) continue;
+                const int r0 = blk * 16;                   // column of the accumulator = row of the filter group
+                const int n0 = n_base + r0;
+                float* optr = a.out + obase + (int64_t)n0 * ostride;
+                if (!border && a.dbg_acc == nullptr && n0 + 16 <= a.N) {
+                    #pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float4 c = sC[r0 + j];
+                        optr[(int64_t)j * ostride] = fmaf(c.x, (float)(int)v[j], fmaf(c.y, fsx, c.z));
+                    }
+                } else {
+                    #pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int n = n0 + j;
+                        if (n >= a.N) continue;
+                        const int s_xw = (int)v[j];
+                        const float4 c = sC[r0 + j];
+                        float c3 = c.z;
+                        if (border) {
+                            // value-zero padding at an image border: S_w and K over inside taps only
+                            int s_w = 0;
+                            for (int t = 0; t < p.T; ++t) {
+                                const int h = ho - a.pad + t / a.kw, vv = wo - a.pad + t % a.kw;
+                                if (h >= 0 && h < a.H && vv >= 0 && vv < a.W) s_w += a.w_sum[(1 + t) * a.N + n];
+                            }
+                            const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
+                            const double wo_ = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
+                            c3 = (float)((double)a.ep.a_offset_val *
+                                         (ws * (double)s_w + (double)a.C * n_inside * wo_));
+                        }
+                        optr[(int64_t)j * ostride] = fmaf(c.x, (float)s_xw, fmaf(c.y, fsx, c3));
+                        if (a.dbg_acc != nullptr) a.dbg_acc[obase + (int64_t)n * ostride] = s_xw;
+                    }
+                }
+            }
+            tc::tc_fence_before_sync();
+            tc::mbar_arrive(&acc_empty[acc]);
+            if (++acc == p.nAcc) { acc = 0; acc_ph ^= 1; }
+        }
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
+}
+
+int sm_count_r()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
+    return sms;
+}
+
+cudaError_t launch_with_scratch(const ConvArgs& c, const ConvI8RPlan& p, void* scratch, cudaStream_t s)
+{
+    uint4* codes = reinterpret_cast<uint4*>(scratch);
+    int* psum = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(scratch) + p.codes_bytes);
+    const unsigned blocks = (unsigned)((p.Pstride + kCodePixels - 1) / kCodePixels);
+    const size_t smem1 = (size_t)p.Cp * 8 + (size_t)kCodeGroups * kCodePixels * 4;
+    conv_codes_kernel<<<blocks, kCodePixels * kCodeGroups, smem1, s>>>(c, p, codes, psum);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(conv_i8r_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(conv_i8r_kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
+                      (const uint4*)codes, (const int*)psum);
+}
+
+}  // namespace
+
+bool conv_i8r_supported(const ConvArgs& c)
+{
+    ConvI8RPlan p;
+    return make_plan_r(c, p, 148);
+}
+
+size_t conv_i8r_scratch_bytes(const ConvArgs& c)
+{
+    ConvI8RPlan p;
+    return make_plan_r(c, p, 148) ? p.scratch_bytes : 0;
+}
+
+// The scratch buffer comes from the stream-ordered allocator and goes back to it right after the two
+// launches, in stream order: no state in the library, safe with several streams, and legal inside a
+// stream capture (the pair becomes allocation and free nodes of the graph).
+cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s)
+{
+    ConvI8RPlan p;
+    if (!make_plan_r(c, p, sm_count_r())) return cudaErrorInvalidConfiguration;
+    void* scratch = nullptr;
+    cudaError_t e = cudaMallocAsync(&scratch, p.scratch_bytes, s);
+    if (e != cudaSuccess) return e;
+    e = launch_with_scratch(c, p, scratch, s);
+    const cudaError_t e2 = cudaFreeAsync(scratch, s);
+    return e != cudaSuccess ? e : e2;
+}
+
+}  // namespace rtn

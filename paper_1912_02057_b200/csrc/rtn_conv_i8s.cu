@@ -240,7 +240,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
         const int tid = (warp - 1) * 32 + lane;
         const bool epi_warp = warp >= kEpiWarp0;
         const int64_t cs = (int64_t)a.H * a.W;
-        const bool per_layer = a.n_thr == 1;
+        const bool per_layer = a.n_thr == 1 && a.C == p.Cp;     // padding channels need their own (infinite) thresholds
         const float lo0 = sLo[0], hi0 = sHi[0];
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
         const int64_t ostride = (int64_t)a.Ho * a.Wo;

@@ -75,10 +75,18 @@ bool conv_i8_supported(const ConvArgs& c);       // filters resident in shared m
 cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s);
 bool conv_i8s_supported(const ConvArgs& c);      // filters streamed (large layers, 1x1 of any stride)
 cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s);
-inline bool conv_i8_any_supported(const ConvArgs& c) { return conv_i8_supported(c) || conv_i8s_supported(c); }
+bool conv_i8r_supported(const ConvArgs& c);      // two kernels: int8 codes in a scratch buffer, filter bank split over CTAs
+size_t conv_i8r_scratch_bytes(const ConvArgs& c);
+cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s);     // scratch from the library's own pool
+inline bool conv_i8_any_supported(const ConvArgs& c)
+{
+    return conv_i8_supported(c) || conv_i8s_supported(c) || conv_i8r_supported(c);
+}
 inline cudaError_t launch_conv_i8_any(const ConvArgs& c, cudaStream_t s)
 {
-    return conv_i8_supported(c) ? launch_conv_i8(c, s) : launch_conv_i8s(c, s);
+    if (conv_i8_supported(c)) return launch_conv_i8(c, s);
+    if (conv_i8s_supported(c)) return launch_conv_i8s(c, s);
+    return launch_conv_i8r(c, s);
 }
 
 // ----------------------------------------------------------------------------------------------

@@ -154,6 +154,18 @@ SMALL_CONVS = [
     (1, 6, 11, 11, 8, 5, 1, 2),
     (1, 300, 6, 6, 16, 3, 1, 1),
     (3, 64, 56, 56, 64, 3, 1, 1),
+    # 256 filters and many channels: the streamed-filter kernel
+    (3, 128, 9, 7, 256, 3, 1, 1),
+    (2, 100, 10, 14, 250, 3, 1, 1),
+    (2, 64, 8, 8, 256, 5, 1, 2),
+    # more than 256 filters: the two-kernel variant (int8 codes in scratch, filter bank split over CTAs)
+    (1, 129, 6, 5, 260, 3, 1, 1),
+    (2, 512, 7, 7, 512, 3, 1, 1),
+    (2, 96, 9, 12, 300, 5, 1, 2),
+    (3, 64, 10, 10, 272, 1, 1, 0),
+    # channel counts that are not multiples of 32 with per-layer thresholds that code 0.0 as -1
+    (2, 40, 8, 12, 24, 3, 1, 1),
+    (2, 100, 8, 8, 256, 1, 1, 0),
 ]
 
 
