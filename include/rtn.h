@@ -135,6 +135,28 @@ rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, i
                               const float* w_scale, const float* w_offset, int64_t n_wparam,
                               float* out, int32_t* dbg_acc, rtn_variant variant, void* stream);
 
+/* Variant of rtn_ternary_conv2d that allocates nothing (the paper has no counterpart; it is for
+ * callers that must not touch an allocator on the hot path).  It always takes the two-kernel
+ * tensor-core path (int8 codes of the input in a scratch buffer, filter bank split over CTAs),
+ * the path rtn_ternary_conv2d chooses for stride-1 layers with more than 256 filters, and gives the
+ * same bits.  The scratch is one array of 16 MiB per device, part of the library's image; the
+ * call performs no cudaMalloc, cudaMallocAsync, cudaFree or other allocating routine.
+ *   - RTN_ERR_UNSUPPORTED: stride != 1, a shape the path does not take, or a layer whose codes
+ *     (about B*(H+2pad)*(W+2pad)*(C rounded up to 32) bytes) exceed the array.
+ *   - The array is shared by every caller on the device: two calls whose kernels may overlap in
+ *     time (different streams, or different host threads on different streams) race on it.
+ *     Issue them on one stream, or order them with events.
+ *   - The first call on a device does set-up (address of the array, kernel attributes) and must come
+ *     before any stream capture; later calls can be captured.
+ * Arguments, layouts and the stream-order rule are those of rtn_ternary_conv2d. */
+rtn_status rtn_ternary_conv2d_noalloc(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
+                              const float* t_lo, const float* t_hi, int64_t n_thr,
+                              const void* w_packed, const int32_t* w_sum,
+                              int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                              rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                              const float* w_scale, const float* w_offset, int64_t n_wparam,
+                              float* out, int32_t* dbg_acc, void* stream);
+
 /* The variant RTN_VARIANT_AUTO resolves to for a shape (never AUTO). */
 rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
 rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,

@@ -64,6 +64,10 @@ def lib():
         L.rtn_ternary_conv2d.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _vp,
                                          _i64, _i64, _i64, _i64, _i64, _int, _f32, _f32,
                                          _vp, _vp, _i64, _vp, _vp, _int, _vp]
+        L.rtn_ternary_conv2d_noalloc.restype = _int
+        L.rtn_ternary_conv2d_noalloc.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _vp,
+                                                 _i64, _i64, _i64, _i64, _i64, _int, _f32, _f32,
+                                                 _vp, _vp, _i64, _vp, _vp, _vp]
         L.rtn_choose_gemm_variant.restype = _int
         L.rtn_choose_gemm_variant.argtypes = [_i64] * 3
         L.rtn_choose_conv_variant.restype = _int
@@ -175,6 +179,21 @@ def rtn_ternary_conv2d(x, t_lo, t_hi, w_packed, w_sum, N, kh, kw, stride, pad, p
         _ptr(w_offset, torch.float32), w_scale.numel(), _ptr(out, torch.float32),
         _ptr(dbg_acc, torch.int32, allow_none=True), int(variant), _stream(stream)),
         "rtn_ternary_conv2d")
+    return out
+
+
+def rtn_ternary_conv2d_noalloc(x, t_lo, t_hi, w_packed, w_sum, N, kh, kw, stride, pad, pad_mode,
+                               a_scale, a_offset, w_scale, w_offset, out, dbg_acc=None, stream=None):
+    """rtn_ternary_conv2d on the two-kernel tensor-core path with the library's static scratch array;
+    ``out`` is the caller's (nothing is allocated here either)."""
+    B, Cin, H, W = x.shape
+    _check(lib().rtn_ternary_conv2d_noalloc(
+        _ptr(x, torch.float32), B, Cin, H, W, _ptr(t_lo, torch.float32), _ptr(t_hi, torch.float32),
+        t_lo.numel(), _ptr(w_packed), _ptr(w_sum, torch.int32), N, kh, kw, stride, pad,
+        int(pad_mode), float(a_scale), float(a_offset), _ptr(w_scale, torch.float32),
+        _ptr(w_offset, torch.float32), w_scale.numel(), _ptr(out, torch.float32),
+        _ptr(dbg_acc, torch.int32, allow_none=True), _stream(stream)),
+        "rtn_ternary_conv2d_noalloc")
     return out
 
 

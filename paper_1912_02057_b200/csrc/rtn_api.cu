@@ -240,6 +240,27 @@ rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, i
     return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
 }
 
+rtn_status rtn_ternary_conv2d_noalloc(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
+                                      const float* t_lo, const float* t_hi, int64_t n_thr,
+                                      const void* w_packed, const int32_t* w_sum,
+                                      int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                                      rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                                      const float* w_scale, const float* w_offset, int64_t n_wparam,
+                                      float* out, int32_t* dbg_acc, void* stream)
+{
+    rtn::ConvArgs c{};
+    rtn_status st = fill_conv_args(c, x, B, C, H, W, t_lo, t_hi, n_thr, w_packed, w_sum, N, kh, kw,
+                                   stride, pad, pad_mode, a_scale, a_offset, w_scale, w_offset,
+                                   n_wparam, out, dbg_acc);
+    if (st != RTN_OK) return st;
+    if (!rtn::conv_i8r_supported(c)) return RTN_ERR_UNSUPPORTED;
+    if (rtn::conv_i8r_scratch_bytes(c) > rtn::conv_i8r_static_scratch_bytes()) return RTN_ERR_UNSUPPORTED;
+    c.status = status_word();
+    if (c.status == nullptr) return RTN_ERR_CUDA;
+    const cudaError_t e = rtn::launch_conv_i8r_static(c, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
 rtn_status rtn_last_device_status(void* stream)
 {
     unsigned* st = status_word();

@@ -484,6 +484,30 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
 }
 
+// Scratch of the variant that allocates nothing: one array per device, part of the module's image.
+// 16 MiB holds the int8 codes of every stride-1 layer of ResNet-18 that this variant takes at batch
+// 128 (512 -> 512, 3x3 on 7x7: 5.4 MB).  Every caller on a device shares it.
+constexpr size_t kStaticScratchBytes = size_t(16) << 20;
+static __device__ __align__(256) uint8_t g_static_scratch[kStaticScratchBytes];
+
+// Address of the array on the current device, looked up once per device.
+void* static_scratch()
+{
+    constexpr int kMaxDevices = 64;
+    static void* addr[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    if (addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        addr[dev] = ptr;
+    }
+    return addr[dev];
+}
+
 int sm_count_r()
 {
     int dev = 0, sms = 0;
@@ -535,5 +559,19 @@ cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s)
     const cudaError_t e2 = cudaFreeAsync(scratch, s);
     return e != cudaSuccess ? e : e2;
 }
+
+// Same two launches with the scratch in the device's static array: no allocating call on this path.
+// cudaErrorInvalidValue: the layer needs more scratch than the array has.
+cudaError_t launch_conv_i8r_static(const ConvArgs& c, cudaStream_t s)
+{
+    ConvI8RPlan p;
+    if (!make_plan_r(c, p, sm_count_r())) return cudaErrorInvalidConfiguration;
+    if (p.scratch_bytes > kStaticScratchBytes) return cudaErrorInvalidValue;
+    void* scratch = static_scratch();
+    if (scratch == nullptr) return cudaErrorInvalidDevicePointer;
+    return launch_with_scratch(c, p, scratch, s);
+}
+
+size_t conv_i8r_static_scratch_bytes() { return kStaticScratchBytes; }
 
 }  // namespace rtn

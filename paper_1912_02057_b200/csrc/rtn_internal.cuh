@@ -77,7 +77,9 @@ bool conv_i8s_supported(const ConvArgs& c);      // filters streamed (large laye
 cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s);
 bool conv_i8r_supported(const ConvArgs& c);      // two kernels: int8 codes in a scratch buffer, filter bank split over CTAs
 size_t conv_i8r_scratch_bytes(const ConvArgs& c);
-cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s);     // scratch from the library's own pool
+cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s);     // scratch from the stream-ordered allocator
+cudaError_t launch_conv_i8r_static(const ConvArgs& c, cudaStream_t s);      // scratch in a static device array
+size_t conv_i8r_static_scratch_bytes();
 inline bool conv_i8_any_supported(const ConvArgs& c)
 {
     return conv_i8_supported(c) || conv_i8s_supported(c) || conv_i8r_supported(c);
