@@ -138,10 +138,10 @@ rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, i
 /* Variant of rtn_ternary_conv2d that allocates nothing (the paper has no counterpart; it is for
  * callers that must not touch an allocator on the hot path).  It always takes the two-kernel
  * tensor-core path (int8 codes of the input in a scratch buffer, filter bank split over CTAs),
- * the path rtn_ternary_conv2d chooses for stride-1 layers with more than 256 filters, and gives the
- * same bits.  The scratch is one array of 16 MiB per device, part of the library's image; the
+ * the path rtn_ternary_conv2d chooses for layers with more than 256 filters and for strided 3x3
+ * layers, and gives the same bits.  The scratch is one array of 16 MiB per device, part of the library's image; the
  * call performs no cudaMalloc, cudaMallocAsync, cudaFree or other allocating routine.
- *   - RTN_ERR_UNSUPPORTED: stride != 1, a shape the path does not take, or a layer whose codes
+ *   - RTN_ERR_UNSUPPORTED: a shape the path does not take (e.g. 3x3 with stride 3), or a layer whose codes
  *     (about B*(H+2pad)*(W+2pad)*(C rounded up to 32) bytes) exceed the array.
  *   - The array is shared by every caller on the device: two calls whose kernels may overlap in
  *     time (different streams, or different host threads on different streams) race on it.

@@ -1,6 +1,6 @@
-// Ternary conv2d, tensor-core variant for stride-1 layers with more than 256 filters or a filter bank
-// the other variants cannot hold (e.g. 512 -> 512, 3x3): two kernels and a scratch buffer of int8
-// codes.  (On 256 -> 256, 3x3 it runs at 44 us against 38 us of the streamed-filter kernel, which
+// Ternary conv2d, tensor-core variant for the layers the other two cannot take: more than 256 filters
+// (e.g. 512 -> 512, 3x3) and strided filters larger than 1x1 (e.g. 3x3 stride 2).  Two kernels and a
+// scratch buffer of int8 codes.  (On 256 -> 256, 3x3 it runs at 44 us against 38 us of the streamed-filter kernel, which
 // therefore keeps that shape.)
 //
 //   conv_codes_kernel   ternarizes the fp32 NCHW input once (Eq. 3) into int8 codes {-1,0,+1} laid out
@@ -19,7 +19,9 @@
 // one 16-channel chunk is one contiguous run of bytes: the producer moves it with one bulk
 // asynchronous copy (cp.async.bulk, completion counted on an mbarrier; no tensor map, no multicast).
 // Shifted-window implicit GEMM as in the other conv kernels: tap (i, j) reads the same rows of
-// shared memory from a start shifted by i*PW + j pixels.  K loop: 32-channel group outer, tap inner;
+// shared memory from a start shifted by i*PW + j pixels.  For stride 2 the code kernel writes the
+// four phase images of the padded input (even/odd rows x even/odd columns) one after the other: tap
+// (i, j) reads phase (i mod 2, j mod 2) shifted by (i div 2, j div 2), a stride-1 window again.  K loop: 32-channel group outer, tap inner;
 // unit of the pipeline = (tile, group) = two chunk windows in one ring slot, 9 MMAs for a 3x3 filter.
 // S_x of a pixel = sum over the taps of the per-pixel code sums (read from the scratch buffer in
 // the epilogue), so all accumulator columns are output channels.
@@ -52,9 +54,11 @@ constexpr int kCodePixels = 64;                        // pixels per block of th
 constexpr int kCodeGroups = 8;                         // 32-channel groups it works on at a time
 
 struct ConvI8RPlan {
-    int PW, PH;            // padded row length / rows per image
-    int Cp, T, halo, RT;   // channels rounded to 32, taps, kh-1, padded rows per tile
-    int ppix;              // pixels of a slot's window: 128 + halo*PW + kw-1, rounded up to 8
+    int PW, PH;            // row length / rows per image of a phase image (the padded image for stride 1)
+    int Cp, T, halo, RT;   // channels rounded to 32, taps, (kh-1)/stride, rows per tile
+    int ppix;              // pixels of a window: 128 + halo*PW + (kw-1)/stride, rounded up to 8
+    int nph;               // phase images some tap reads (1 for stride 1; up to 4 for stride 2)
+    int ph_r[4], ph_c[4];  // their row / column phases
     int total_rows, ntiles;
     int S, Nq;             // filter groups; filters per group (multiple of 16)
     int cpg, grid;         // CTAs per filter group; grid = S * cpg
@@ -67,36 +71,58 @@ struct ConvI8RPlan {
     uint32_t off_w, off_c, off_bar, off_misc, off_slot, slot_bytes;
     size_t smem_bytes;
     size_t codes_bytes, scratch_bytes;     // scratch = codes, then the per-pixel sums
-    uint32_t tap_shift[kMaxTaps];          // i*PW + j
+    uint32_t tap_shift[kMaxTaps];          // start of the tap's A window inside a slot, 16-byte units
+    uint32_t tap_psum[kMaxTaps];           // the tap's offset into the per-pixel sums
 };
 
 bool make_plan_r(const ConvArgs& c, ConvI8RPlan& p, int sms)
 {
-    if (c.stride != 1) return false;
-    if (c.Ho <= 0 || c.Wo <= 0) return false;
+    if (c.stride < 1 || c.Ho <= 0 || c.Wo <= 0) return false;
     p.T = c.kh * c.kw;
     if (p.T > kMaxTaps) return false;
-    p.PW = c.W + 2 * c.pad;
-    p.PH = c.H + 2 * c.pad;
+    // Stride s: the padded image splits into s*s phase images (rows = a mod s, columns = b mod s);
+    // tap (i, j) reads phase (i mod s, j mod s) at the output pixel shifted by (i div s, j div s), so
+    // inside a phase image the convolution has stride 1 and the shifted-window scheme applies.
+    const int st = c.stride;
+    p.nph = 0;
+    int ph_of_tap[kMaxTaps];
+    for (int t = 0; t < p.T; ++t) {
+        const int a = (t / c.kw) % st, b = (t % c.kw) % st;
+        int w = -1;
+        for (int k = 0; k < p.nph; ++k) if (p.ph_r[k] == a && p.ph_c[k] == b) w = k;
+        if (w < 0) {
+            if (p.nph == 4) return false;
+            w = p.nph++;
+            p.ph_r[w] = a; p.ph_c[w] = b;
+        }
+        ph_of_tap[t] = w;
+    }
+    p.PW = (c.W + 2 * c.pad + st - 1) / st;
+    p.PH = (c.H + 2 * c.pad + st - 1) / st;
     if (p.PW > kTileM || p.PH > 2048) return false;
     if ((int64_t)c.B * p.PH > (1 << 20)) return false;
     p.Cp = (c.C + 31) / 32 * 32;
     p.ngroup = p.Cp / 32;
     if (p.ngroup > 16) return false;
-    p.halo = c.kh - 1;
+    p.halo = (c.kh - 1) / st;
     p.RT = kTileM / p.PW;
-    p.ppix = (kTileM + p.halo * p.PW + (c.kw - 1) + 7) / 8 * 8;
+    p.ppix = (kTileM + p.halo * p.PW + (c.kw - 1) / st + 7) / 8 * 8;
     p.total_rows = c.B * p.PH;
     p.ntiles = (p.total_rows + p.RT - 1) / p.RT;
     p.Ptot = (int64_t)p.total_rows * p.PW;
     p.Pstride = p.Ptot + p.ppix;
-    p.gps = (p.ngroup % 2 == 0) ? 2 : 1;
-    p.slot_bytes = (uint32_t)p.gps * 2u * (uint32_t)p.ppix * 16u;
+    if ((int64_t)p.nph * p.Pstride >= (int64_t(1) << 31)) return false;
+    p.gps = (p.ngroup % 2 == 0 && p.nph == 1) ? 2 : 1;
+    p.slot_bytes = (uint32_t)p.nph * (uint32_t)p.gps * 2u * (uint32_t)p.ppix * 16u;
     p.div_pw = make_fastdiv((uint32_t)p.PW);
     p.div_ph = make_fastdiv((uint32_t)p.PH);
     p.div_cw = make_fastdiv((uint32_t)p.ngroup);
-    for (int t = 0; t < p.T; ++t) p.tap_shift[t] = (uint32_t)((t / c.kw) * p.PW + (t % c.kw));
-    // fewest filter groups whose share of the bank leaves room for a ring of at least four slots
+    for (int t = 0; t < p.T; ++t) {
+        const uint32_t shift = (uint32_t)(((t / c.kw) / st) * p.PW + (t % c.kw) / st);
+        p.tap_shift[t] = (uint32_t)ph_of_tap[t] * (uint32_t)(2 * p.gps * p.ppix) + shift;
+        p.tap_psum[t] = (uint32_t)((int64_t)ph_of_tap[t] * p.Pstride) + shift;
+    }
+    // fewest filter groups whose share of the bank leaves room for a ring of at least three slots
     for (p.S = 1; p.S <= kMaxSplit; p.S *= 2) {
         if (p.S > sms) return false;
         p.Nq = ((c.N + p.S - 1) / p.S + 15) / 16 * 16;
@@ -111,7 +137,7 @@ bool make_plan_r(const ConvArgs& c, ConvI8RPlan& p, int sms)
         if (o >= kSmemLimit) continue;
         int ns = (int)((kSmemLimit - o) / p.slot_bytes);
         if (ns > kMaxSlots) ns = kMaxSlots;
-        if (ns < 4) continue;
+        if (ns < 3) continue;
         p.nslots = ns;
         p.smem_bytes = o + (size_t)ns * p.slot_bytes;
         break;
@@ -126,8 +152,8 @@ bool make_plan_r(const ConvArgs& c, ConvI8RPlan& p, int sms)
     uint32_t cols = 32;
     while (cols < (uint32_t)(p.nAcc * p.Nq)) cols *= 2;
     p.tmem_cols = cols;
-    p.codes_bytes = (size_t)(p.Cp / 16) * (size_t)p.Pstride * 16;
-    p.scratch_bytes = p.codes_bytes + ((size_t)p.Pstride * 4 + 255) / 256 * 256;
+    p.codes_bytes = (size_t)p.nph * (size_t)(p.Cp / 16) * (size_t)p.Pstride * 16;
+    p.scratch_bytes = p.codes_bytes + ((size_t)p.nph * (size_t)p.Pstride * 4 + 255) / 256 * 256;
     return true;
 }
 
@@ -155,6 +181,9 @@ conv_codes_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, uint4
     __syncthreads();
     const int px = threadIdx.x % kCodePixels, gi = threadIdx.x / kCodePixels;
     const int64_t P = (int64_t)blockIdx.x * kCodePixels + px;
+    const int w = blockIdx.y;                               // phase image
+    codes += (int64_t)w * (p.Cp / 16) * p.Pstride;
+    psum += (int64_t)w * p.Pstride;
     const bool per_layer = a.n_thr == 1 && a.C == p.Cp;     // padding channels need their own (infinite) thresholds
     const float lo0 = sLo[0], hi0 = sHi[0];
     const int64_t cs = (int64_t)a.H * a.W;
@@ -163,9 +192,9 @@ conv_codes_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, uint4
     const float* src0 = nullptr;
     if (P < p.Ptot) {
         const uint32_t G = fdiv((uint32_t)P, p.div_pw);
-        const int col = (int)((uint32_t)P - G * (uint32_t)p.PW) - a.pad;
+        const int col = (int)((uint32_t)P - G * (uint32_t)p.PW) * a.stride + p.ph_c[w] - a.pad;
         const uint32_t b = fdiv(G, p.div_ph);
-        const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
+        const int r = (int)(G - b * (uint32_t)p.PH) * a.stride + p.ph_r[w] - a.pad;
         inside = r >= 0 && r < a.H && col >= 0 && col < a.W;
         if (inside) src0 = a.x + (((int64_t)b * a.C) * a.H + r) * a.W + col;
     }
@@ -325,10 +354,12 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
                 const int64_t P0 = (int64_t)tile * p.RT * p.PW;
                 for (int h = 0; h < p.ngroup; h += p.gps) {
                     if (!wait_or_die(&slot_empty[s], ph ^ 1, a.status, dead)) { alive = false; break; }
-                    mbar_expect_tx_r(&slot_full[s], (uint32_t)(2 * p.gps) * win_bytes);
+                    mbar_expect_tx_r(&slot_full[s], (uint32_t)(2 * p.gps * p.nph) * win_bytes);
                     const uint32_t dst = ring + s * p.slot_bytes, bar = tc::smem_addr(&slot_full[s]);
-                    for (int c = 0; c < 2 * p.gps; ++c)
-                        bulk_copy_g2s(dst + (uint32_t)c * win_bytes, codes + (int64_t)(2 * h + c) * p.Pstride + P0, win_bytes, bar);
+                    for (int w = 0; w < p.nph; ++w)
+                        for (int c = 0; c < 2 * p.gps; ++c)
+                            bulk_copy_g2s(dst + (uint32_t)(w * 2 * p.gps + c) * win_bytes,
+                                          codes + ((int64_t)w * nchunk + 2 * h + c) * p.Pstride + P0, win_bytes, bar);
                     if (++s == (uint32_t)p.nslots) { s = 0; ph ^= 1; }
                 }
             }
@@ -422,11 +453,11 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
             int n_inside = p.T, s_x = 0;
             if (ok) {
                 const int* ps = psum + (int64_t)g * p.PW + pl;
-                for (int t = 0; t < p.T; ++t) s_x += __ldg(ps + p.tap_shift[t]);
+                for (int t = 0; t < p.T; ++t) s_x += __ldg(ps + p.tap_psum[t]);
                 if (a.pad_mode == RTN_PAD_VALUE_ZERO) {
                     n_inside = 0;
                     for (int t = 0; t < p.T; ++t) {
-                        const int h = ho - a.pad + t / a.kw, v = wo - a.pad + t % a.kw;
+                        const int h = ho * a.stride - a.pad + t / a.kw, v = wo * a.stride - a.pad + t % a.kw;
                         n_inside += (h >= 0 && h < a.H && v >= 0 && v < a.W);
                     }
                 }
@@ -461,7 +492,7 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
                             // value-zero padding at an image border: S_w and K over inside taps only
                             int s_w = 0;
                             for (int t = 0; t < p.T; ++t) {
-                                const int h = ho - a.pad + t / a.kw, vv = wo - a.pad + t % a.kw;
+                                const int h = ho * a.stride - a.pad + t / a.kw, vv = wo * a.stride - a.pad + t % a.kw;
                                 if (h >= 0 && h < a.H && vv >= 0 && vv < a.W) s_w += a.w_sum[(1 + t) * a.N + n];
                             }
                             const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
@@ -520,7 +551,7 @@ cudaError_t launch_with_scratch(const ConvArgs& c, const ConvI8RPlan& p, void* s
 {
     uint4* codes = reinterpret_cast<uint4*>(scratch);
     int* psum = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(scratch) + p.codes_bytes);
-    const unsigned blocks = (unsigned)((p.Pstride + kCodePixels - 1) / kCodePixels);
+    const dim3 blocks((unsigned)((p.Pstride + kCodePixels - 1) / kCodePixels), (unsigned)p.nph);
     const size_t smem1 = (size_t)p.Cp * 8 + (size_t)kCodeGroups * kCodePixels * 4;
     conv_codes_kernel<<<blocks, kCodePixels * kCodeGroups, smem1, s>>>(c, p, codes, psum);
     cudaError_t e = cudaGetLastError();

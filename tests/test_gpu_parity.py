@@ -163,6 +163,11 @@ SMALL_CONVS = [
     (2, 512, 7, 7, 512, 3, 1, 1),
     (2, 96, 9, 12, 300, 5, 1, 2),
     (3, 64, 10, 10, 272, 1, 1, 0),
+    # strided filters: phase images of the two-kernel variant
+    (2, 256, 14, 14, 512, 3, 2, 1),
+    (2, 256, 14, 14, 512, 1, 2, 0),
+    (1, 16, 11, 11, 8, 5, 2, 2),
+    (2, 64, 15, 9, 40, 3, 2, 0),
     # channel counts that are not multiples of 32 with per-layer thresholds that code 0.0 as -1
     (2, 40, 8, 12, 24, 3, 1, 1),
     (2, 100, 8, 8, 256, 1, 1, 0),

@@ -23,7 +23,8 @@ def _args(case):
 
 
 @pytest.mark.parametrize("pad_mode", [rtn.PAD_CODE_ZERO, rtn.PAD_VALUE_ZERO], ids=["codezero", "valuezero"])
-@pytest.mark.parametrize("shape", [(2, 512, 7, 7, 512, 3, 1, 1), (3, 96, 9, 12, 300, 5, 1, 2), (2, 40, 8, 12, 24, 3, 1, 1)],
+@pytest.mark.parametrize("shape", [(2, 512, 7, 7, 512, 3, 1, 1), (3, 96, 9, 12, 300, 5, 1, 2), (2, 40, 8, 12, 24, 3, 1, 1),
+                                   (2, 128, 14, 14, 256, 3, 2, 1)],
                          ids=lambda s: "x".join(map(str, s)))
 def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row(shape, pad_mode):
     B, C, H, W, N, k, stride, pad = shape
@@ -59,9 +60,9 @@ def test_noalloc_rejects_what_does_not_fit_or_is_not_taken():
     with pytest.raises(rtn.RtnError) as e:
         rtn.rtn_ternary_conv2d_noalloc(pad_mode=rtn.PAD_CODE_ZERO, out=out, **a)
     assert e.value.code == 5          # RTN_ERR_UNSUPPORTED
-    strided = inputs.conv_case("noalloc_s2", 2, 64, 12, 12, 32, 3, 2, 1, seed=6, p_zero=0.4, thresholds=(0.3, 1.0))
-    a = _args(strided)
-    out = torch.empty((2, 32, 6, 6), dtype=torch.float32, device="cuda")
+    strided = inputs.conv_case("noalloc_s3", 2, 64, 12, 12, 32, 3, 3, 1, seed=6, p_zero=0.4, thresholds=(0.3, 1.0))
+    a = _args(strided)        # 3x3 with stride 3 reads nine phase images: not taken
+    out = torch.empty((2, 32, 4, 4), dtype=torch.float32, device="cuda")
     with pytest.raises(rtn.RtnError) as e:
         rtn.rtn_ternary_conv2d_noalloc(pad_mode=rtn.PAD_CODE_ZERO, out=out, **a)
     assert e.value.code == 5
