@@ -41,6 +41,9 @@ WORKLOADS = {
     "cfg5_gemm_4096": lambda: inputs.config5(4096),
     "cfg5_gemm_8192": lambda: inputs.config5(8192),
 }
+# every ternary conv layer of ResNet-18 at batch 128 (the layer table of the paper's appendix)
+for _l in inputs.resnet18_ternary_layers():
+    WORKLOADS[f"r18_{_l[0]}_b128"] = (lambda n=_l[0]: inputs.resnet18_layer(n, batch=128))
 DEFAULT_WORKLOAD = "cfg2_conv3x3_c64_56x56_b32"
 
 
@@ -279,7 +282,8 @@ def run_ours(args, case, name):
                 for _ in range(n_sets)]
         variant = rtn.rtn_choose_conv_variant(case.B, case.C, case.H, case.W, case.N, case.kh,
                                               case.kw, case.stride, case.pad)
-        launches_per_step = 1
+        launches_per_step = rtn.rtn_conv_kernel_launches(case.B, case.C, case.H, case.W, case.N, case.kh,
+                                                         case.kw, case.stride, case.pad)
 
         def step(i):
             j = i % n_sets

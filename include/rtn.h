@@ -161,6 +161,10 @@ rtn_status rtn_ternary_conv2d_noalloc(const float* x, int64_t B, int64_t C, int6
 rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
 rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
                                     int64_t kh, int64_t kw, int64_t stride, int64_t pad);
+/* Kernel launches one rtn_ternary_conv2d call with RTN_VARIANT_AUTO makes for a shape: 1, or 2 on the
+ * path that first writes the input's int8 codes to a scratch buffer. */
+int64_t rtn_conv_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
+                                 int64_t kh, int64_t kw, int64_t stride, int64_t pad);
 
 /* Synchronises `stream`, then reads and clears the device status word of the current device.
  * RTN_OK, or RTN_ERR_DEVICE_TIMEOUT if a kernel's bounded wait (on an mbarrier of the

@@ -190,3 +190,12 @@ def resnet18_ternary_layers():
               (f"layer{s}.1.conv1", cout, cout, 3, 1, 1, hout),
               (f"layer{s}.1.conv2", cout, cout, 3, 1, 1, hout)]
     return L
+
+
+def resnet18_layer(name, batch=128, p_zero=0.5):
+    """One of the 19 ternary conv layers of ResNet-18 as a ConvCase (thresholds around the offset)."""
+    for i, (lname, cin, cout, k, stride, pad, hin) in enumerate(resnet18_ternary_layers()):
+        if lname == name:
+            return conv_case(f"r18_{name}_b{batch}", batch, cin, hin, hin, cout, k, stride, pad,
+                             seed=400 + i, p_zero=p_zero)
+    raise KeyError(name)
