@@ -251,6 +251,44 @@ def im2col(x, kh, kw, stride, pad):
     return cols
 
 
+# ----------------------------------------------------------------------------- next layer's input
+def next_layer(pre, relu, skip, t_lo, t_hi):
+    """Eq. 10's phi (ReLU, optional), the block's skip connection (optional), then the next layer's
+    ternarizer (Eq. 3 with that layer's BN folded into per-channel thresholds).
+
+    ``pre`` [B,N,...] double (a conv's affine output); ``skip`` fp32 of the same shape or None.
+    Returns (y double, codes int8, margin double): y = phi(pre) + skip, codes decided on fp32(y),
+    margin = distance of y to the nearer threshold.
+    """
+    pre = _arr(pre, np.float64)
+    B, N = pre.shape[:2]
+    inner = int(np.prod(pre.shape[2:], dtype=np.int64))
+    lo, hi = _param(t_lo), _param(t_hi)
+    assert lo.size == hi.size and lo.size in (1, N)
+    sk = None if skip is None else _arr(skip, np.float32)
+    assert sk is None or sk.shape == pre.shape
+    y = np.empty(pre.shape, np.float64)
+    codes = np.empty(pre.shape, np.int8)
+    margin = np.empty(pre.shape, np.float64)
+    _L().orc_next_layer(_p(pre), _p(sk), C.c_int(1 if relu else 0), _i64(B), _i64(N), _i64(inner),
+                        _p(lo), _p(hi), _i64(lo.size), _p(y), _p(codes), _p(margin))
+    return y, codes, margin
+
+
+def pack_nhwc(codes):
+    """Activation codes [B,C,H,W] -> packed pixel rows [B*H*W, ceil(C/128)*32]: one row of C codes
+    per pixel in the block-plane format (Table 1 planes), pixels in (b, h, w) order."""
+    codes = _arr(codes, np.int8)
+    B, Cc, H, W = codes.shape
+    return pack_rows(np.ascontiguousarray(codes.transpose(0, 2, 3, 1)).reshape(B * H * W, Cc))
+
+
+def unpack_nhwc(packed, B, Cc, H, W):
+    """Inverse of pack_nhwc: packed pixel rows -> codes [B,C,H,W]."""
+    rows = unpack_rows(np.asarray(packed, np.uint8).reshape(B * H * W, packed_row_bytes(Cc)), Cc)
+    return np.ascontiguousarray(rows.reshape(B, H, W, Cc).transpose(0, 3, 1, 2))
+
+
 # ----------------------------------------------------------------------------- tolerance
 REL_TOL = 1e-5
 ABS_TOL = 1e-6

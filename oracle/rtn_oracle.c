@@ -358,3 +358,42 @@ double orc_direct_dot(const int8_t *x, const int8_t *w, int64_t K,
         acc += (a_s * (double)x[k] + a_o) * (w_s * (double)w[k] + w_o);
     return acc;
 }
+
+/* ------------------------------------------------------------------------- */
+/* What a ternary layer hands to the next one.  Eq. 10 wraps the affine form in */
+/* phi (ReLU); the residual block then adds its skip connection; the next       */
+/* layer's BN (placed after the ReLU, section "Activation Ternarization") is    */
+/* folded into a threshold pair per channel and Eq. 3 ternarizes:               */
+/*     y    = phi(pre) + skip          (phi and skip each optional)             */
+/*     code = +1 if y > t_hi[n], -1 if y < t_lo[n], else 0                      */
+/* y is evaluated in double.  The code is decided on y rounded to fp32 with     */
+/* fp32 comparisons, the precision the layer's consumer decides in.  margin is  */
+/* the distance of the double y to the nearer threshold: where it is below the  */
+/* fp32 rounding error of y, the neighbouring code is as valid.                 */
+/* Tensors are [B][N][inner]; thresholds per layer (n_thr == 1) or channel n.   */
+/* ------------------------------------------------------------------------- */
+void orc_next_layer(const double *pre, const float *skip /* nullable */, int relu,
+                    int64_t B, int64_t N, int64_t inner,
+                    const float *t_lo, const float *t_hi, int64_t n_thr,
+                    double *y /* out */, int8_t *codes /* out */, double *margin /* out */)
+{
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t n = 0; n < N; ++n) {
+            const float lo = t_lo[n_thr == 1 ? 0 : n];
+            const float hi = t_hi[n_thr == 1 ? 0 : n];
+            for (int64_t i = 0; i < inner; ++i) {
+                const int64_t idx = (b * N + n) * inner + i;
+                double v = pre[idx];
+                if (relu && !(v > 0.0)) v = 0.0;
+                if (skip) v += (double)skip[idx];
+                y[idx] = v;
+                const float vf = (float)v;
+                int8_t t = 0;
+                if (vf > hi) t = 1;
+                else if (vf < lo) t = -1;
+                codes[idx] = t;
+                const double d_hi = fabs(v - (double)hi), d_lo = fabs(v - (double)lo);
+                margin[idx] = d_hi < d_lo ? d_hi : d_lo;
+            }
+        }
+}

@@ -344,3 +344,113 @@ def test_resnet18_layer_list_matches_the_appendix_table():
     layers = inputs.resnet18_ternary_layers()
     assert sorted(names) == sorted(l[0] for l in layers) and len(layers) == 19
     assert sum(1 for l in layers if l[3] == 3) == 16 and sum(1 for l in layers if l[3] == 1) == 3
+
+
+# ------------------------------------------------------------------ what a layer hands to the next one
+def test_next_layer_hand_case_order_and_ties():
+    # phi acts on the conv output BEFORE the skip connection is added; strict comparisons
+    pre = np.array([[[-1.0, 0.2, 3.0, 0.25, -4.0]]])           # [B=1][N=1][5]
+    skip = np.array([[[0.5, 0.5, -2.0, 0.5, -1.0]]], np.float32)
+    y, codes, margin = oracle.next_layer(pre, True, skip, 0.6, 0.75)
+    assert y.ravel().tolist() == [0.5, 0.7, 1.0, 0.75, -1.0]    # relu(-1)+0.5, ..., relu(-4)-1
+    assert codes.ravel().tolist() == [-1, 0, 1, 0, -1]          # y == t_hi codes to 0
+    assert margin.ravel()[3] == 0.0
+    y2, codes2, _ = oracle.next_layer(pre, False, None, 0.6, 0.75)
+    assert y2.ravel().tolist() == pre.ravel().tolist()
+    assert codes2.ravel().tolist() == [-1, -1, 1, -1, -1]
+
+
+def test_next_layer_relu_is_eq11_folded_form():
+    # Eq. 11: phi(alpha gamma S + C) = alpha * max(0, gamma S + T), T = beta * (1 (x) W^t), alpha > 0
+    g = np.random.default_rng(41)
+    x = inputs.weight_codes(g, (2, 6, 7, 7), 0.3)
+    w = inputs.weight_codes(g, (5, 6, 3, 3), 0.4)
+    gamma, beta = 1.25, -0.375
+    alpha = inputs.uniform(g, 0.5, 1.5, (5,))
+    S, pre, _ = oracle.conv2d(x, w, 1, 1, oracle.PAD_CODE_ZERO, gamma, beta, alpha, np.zeros(5, np.float32))
+    y, _, _ = oracle.next_layer(pre, True, None, 0.0, 0.0)
+    T = beta * w.astype(np.int64).sum(axis=(1, 2, 3))
+    a64 = alpha.astype(np.float64)[None, :, None, None]
+    want = a64 * np.maximum(0.0, gamma * S + T[None, :, None, None])
+    assert np.allclose(y, want, rtol=1e-12, atol=1e-12)
+    assert (y >= 0).all() and (y == 0).any() and (y > 0).any()
+
+
+@pytest.mark.parametrize("relu,with_skip", [(True, True), (True, False), (False, True)])
+def test_next_layer_against_torch_fp64_block(relu, with_skip):
+    # conv on de-quantised values -> ReLU -> + skip -> BN transform (Eq. 2) -> Q of Eq. 1, all in torch fp64
+    g = np.random.default_rng(43)
+    B, C, H, W, N = 2, 5, 8, 8, 6
+    x = inputs.weight_codes(g, (B, C, H, W), 0.3)
+    w = inputs.weight_codes(g, (N, C, 3, 3), 0.4)
+    a_s, a_o = 0.75, 0.125
+    w_s, w_o = inputs.uniform(g, 0.5, 1.5, (N,)), inputs.uniform(g, -0.1, 0.1, (N,))
+    skip = g.standard_normal((B, N, H, W)).astype(np.float32) if with_skip else None
+    k = inputs.uniform(g, 0.2, 0.6, (N,)).astype(np.float64)      # BN scale (k > 0) and shift per channel
+    b = inputs.uniform(g, -1.2, -0.7, (N,)).astype(np.float64)    # t_lo > 0: -1 occurs after a ReLU too
+    t_hi = ((0.5 - b) / k).astype(np.float32)
+    t_lo = (-(0.5 + b) / k).astype(np.float32)
+    _, pre, _ = oracle.conv2d(x, w, 1, 1, oracle.PAD_VALUE_ZERO, a_s, a_o, w_s, w_o)
+    y, codes, margin = oracle.next_layer(pre, relu, skip, t_lo, t_hi)
+
+    xd = _deq(x, a_s, a_o)
+    wd = torch.from_numpy(w_s.astype(np.float64))[:, None, None, None] * torch.from_numpy(
+        w.astype(np.float64)) + torch.from_numpy(w_o.astype(np.float64))[:, None, None, None]
+    ref = F.conv2d(xd, wd, padding=1)
+    if relu:
+        ref = F.relu(ref)
+    if with_skip:
+        ref = ref + torch.from_numpy(skip.astype(np.float64))
+    assert np.allclose(y, ref.numpy(), rtol=1e-12, atol=1e-10)
+    bn = torch.from_numpy(k)[None, :, None, None] * ref + torch.from_numpy(b)[None, :, None, None]
+    q = torch.where(bn.abs() > 0.5, torch.sign(bn), torch.zeros_like(bn)).numpy().astype(np.int8)
+    clear = margin > 1e-5            # fp32 thresholds and fp32(y) move a decision only this close to a threshold
+    assert clear.mean() > 0.99
+    assert np.array_equal(codes[clear], q[clear])
+    assert set(np.unique(codes).tolist()) == {-1, 0, 1}
+
+
+def test_next_layer_per_channel_thresholds_index_axis_1():
+    pre = np.zeros((2, 3, 4))
+    pre[:, 1] = 1.0
+    _, codes, _ = oracle.next_layer(pre, False, None, np.array([-1, 2, -1], np.float32),
+                                    np.array([-0.5, 3, 0.5], np.float32))
+    assert (codes[:, 0] == 1).all() and (codes[:, 1] == -1).all() and (codes[:, 2] == 0).all()
+
+
+def test_pack_nhwc_is_one_packed_row_per_pixel():
+    g = np.random.default_rng(47)
+    B, C, H, W = 2, 70, 3, 5
+    codes = inputs.weight_codes(g, (B, C, H, W), 0.3)
+    packed = oracle.pack_nhwc(codes)
+    assert packed.shape == (B * H * W, 32)
+    # pixel (b=1, h=2, w=3): its row is the pack of its C channel codes
+    row = (1 * H + 2) * W + 3
+    assert np.array_equal(packed[row], oracle.pack_rows(codes[1, :, 2, 3][None, :])[0])
+    # channel 9 of that pixel: bit 1 of byte 1 of plane 1 (non-zero) and of plane 2 (positive)
+    c = int(codes[1, 9, 2, 3])
+    assert (packed[row, 1] >> 1) & 1 == (1 if c != 0 else 0)
+    assert (packed[row, 17] >> 1) & 1 == (1 if c > 0 else 0)
+    assert np.array_equal(oracle.unpack_nhwc(packed, B, C, H, W), codes)
+
+
+def test_two_layer_chain_against_torch_fp64():
+    # layer 1 -> phi -> ternarize -> layer 2: the codes the first layer hands over are the second's input
+    g = np.random.default_rng(53)
+    B, C, H, W, N1, N2 = 1, 4, 6, 6, 5, 3
+    x = inputs.weight_codes(g, (B, C, H, W), 0.3)
+    w1 = inputs.weight_codes(g, (N1, C, 3, 3), 0.4)
+    w2 = inputs.weight_codes(g, (N2, N1, 3, 3), 0.4)
+    ws1, ws2 = inputs.uniform(g, 0.5, 1.5, (N1,)), inputs.uniform(g, 0.5, 1.5, (N2,))
+    zero1, zero2 = np.zeros(N1, np.float32), np.zeros(N2, np.float32)
+    _, pre1, _ = oracle.conv2d(x, w1, 1, 1, oracle.PAD_VALUE_ZERO, 1.0, 0.25, ws1, zero1)
+    _, codes1, margin = oracle.next_layer(pre1, True, None, 0.5, 2.0)
+    assert margin.min() > 1e-6
+    _, pre2, _ = oracle.conv2d(codes1, w2, 1, 1, oracle.PAD_VALUE_ZERO, 0.5, -0.125, ws2, zero2)
+
+    def deq_w(w, s):
+        return torch.from_numpy(s.astype(np.float64))[:, None, None, None] * torch.from_numpy(w.astype(np.float64))
+    h = F.relu(F.conv2d(_deq(x, 1.0, 0.25), deq_w(w1, ws1), padding=1))
+    c = torch.where(h > 2.0, 1.0, torch.where(h < 0.5, -1.0, 0.0)).to(torch.float64)
+    ref = F.conv2d(0.5 * c - 0.125, deq_w(w2, ws2), padding=1).numpy()
+    assert np.allclose(pre2, ref, rtol=1e-12, atol=1e-10)
