@@ -157,6 +157,53 @@ rtn_status rtn_ternary_conv2d_noalloc(const float* x, int64_t B, int64_t C, int6
                               const float* w_scale, const float* w_offset, int64_t n_wparam,
                               float* out, int32_t* dbg_acc, void* stream);
 
+/* Ternary conv2d that hands its result to the next layer from its epilogue (Eq. 10 with its phi;
+ * section "Activation Ternarization": BN sits after the ReLU, so the next layer's BN folds into
+ * that layer's threshold pair of Eq. 3).  Per output value:
+ *     y    = phi(affine form of rtn_ternary_conv2d) + skip      phi = ReLU if relu == 1, else identity
+ *     out        <- y (fp32)                                    if out != NULL
+ *     out_packed <- +1 if y > next_t_hi, -1 if y < next_t_lo, else 0, as a packed pixel row
+ *                                                               if out_packed != NULL
+ * so a layer whose only consumer is the next ternary layer writes 2 bits per value instead of 32.
+ *   x ... n_wparam   as in rtn_ternary_conv2d
+ *   skip        NULL, or fp32 [B][N][Ho][Wo] (the residual block's skip connection), added after phi
+ *   out         NULL, or fp32 [B][N][Ho][Wo]
+ *   next_t_lo, next_t_hi   thresholds of the NEXT layer's ternarizer: n_next_thr = 1 (per layer) or N
+ *               (per channel of this layer's output); strict fp32 comparisons on the fp32 y, +1 first;
+ *               required when out_packed != NULL
+ *   out_packed  NULL, or B*Ho*Wo packed rows of N codes each (rtn_packed_bytes(B*Ho*Wo, N) bytes,
+ *               16-byte aligned): pixel (b, ho, wo) is row (b*Ho + ho)*Wo + wo, channel n is code n of
+ *               the row; canonical zeros, zero fill past N.  This is the x_packed of
+ *               rtn_ternary_conv2d_packed.
+ *   dbg_acc     NULL, or int32 [B][N][Ho][Wo] raw S_xw
+ * At least one of out, out_packed must be given.  Takes the two-kernel tensor-core path (int8 codes in
+ * a scratch buffer from the stream-ordered allocator); RTN_ERR_UNSUPPORTED for shapes that path does
+ * not take (see rtn_ternary_conv2d_noalloc).  Stream-order rule as for rtn_ternary_conv2d; the
+ * next-layer thresholds count as parameters of the layer. */
+rtn_status rtn_ternary_conv2d_fused(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
+                                    const float* t_lo, const float* t_hi, int64_t n_thr,
+                                    const void* w_packed, const int32_t* w_sum,
+                                    int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                                    rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                                    const float* w_scale, const float* w_offset, int64_t n_wparam,
+                                    int relu, const float* skip, float* out,
+                                    const float* next_t_lo, const float* next_t_hi, int64_t n_next_thr,
+                                    void* out_packed, int32_t* dbg_acc, void* stream);
+
+/* The same layer on an input that is already ternary: packed pixel rows (Table 1 planes; A1, A2 of
+ * Eq. 9 with the channel as the fast index), as written by the out_packed of the layer before or by
+ * rtn_ternarize_pack_act on an fp32 [B*H*W][C] (NHWC) matrix.
+ *   x_packed    B*H*W packed rows of C codes: pixel (b, h, w) is row (b*H + h)*W + w; 16-byte aligned
+ * Everything else as in rtn_ternary_conv2d_fused (there are no thresholds for the input: it is codes). */
+rtn_status rtn_ternary_conv2d_packed(const void* x_packed, int64_t B, int64_t C, int64_t H, int64_t W,
+                                     const void* w_packed, const int32_t* w_sum,
+                                     int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                                     rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                                     const float* w_scale, const float* w_offset, int64_t n_wparam,
+                                     int relu, const float* skip, float* out,
+                                     const float* next_t_lo, const float* next_t_hi, int64_t n_next_thr,
+                                     void* out_packed, int32_t* dbg_acc, void* stream);
+
 /* The variant RTN_VARIANT_AUTO resolves to for a shape (never AUTO). */
 rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
 rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,

@@ -68,6 +68,15 @@ def lib():
         L.rtn_ternary_conv2d_noalloc.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _vp,
                                                  _i64, _i64, _i64, _i64, _i64, _int, _f32, _f32,
                                                  _vp, _vp, _i64, _vp, _vp, _vp]
+        _tail = [_int, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp]      # relu ... stream
+        L.rtn_ternary_conv2d_fused.restype = _int
+        L.rtn_ternary_conv2d_fused.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _vp,
+                                               _i64, _i64, _i64, _i64, _i64, _int, _f32, _f32,
+                                               _vp, _vp, _i64] + _tail
+        L.rtn_ternary_conv2d_packed.restype = _int
+        L.rtn_ternary_conv2d_packed.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp, _vp,
+                                                _i64, _i64, _i64, _i64, _i64, _int, _f32, _f32,
+                                                _vp, _vp, _i64] + _tail
         L.rtn_choose_gemm_variant.restype = _int
         L.rtn_choose_gemm_variant.argtypes = [_i64] * 3
         L.rtn_choose_conv_variant.restype = _int
@@ -197,6 +206,45 @@ def rtn_ternary_conv2d_noalloc(x, t_lo, t_hi, w_packed, w_sum, N, kh, kw, stride
         _ptr(dbg_acc, torch.int32, allow_none=True), _stream(stream)),
         "rtn_ternary_conv2d_noalloc")
     return out
+
+
+def _next_tail(relu, skip, out, next_t_lo, next_t_hi, out_packed, dbg_acc, stream):
+    n_next = next_t_lo.numel() if next_t_lo is not None else 1
+    return (int(bool(relu)), _ptr(skip, torch.float32, allow_none=True),
+            _ptr(out, torch.float32, allow_none=True), _ptr(next_t_lo, torch.float32, allow_none=True),
+            _ptr(next_t_hi, torch.float32, allow_none=True), n_next,
+            _ptr(out_packed, torch.uint8, allow_none=True), _ptr(dbg_acc, torch.int32, allow_none=True),
+            _stream(stream))
+
+
+def rtn_ternary_conv2d_fused(x, t_lo, t_hi, w_packed, w_sum, N, kh, kw, stride, pad, pad_mode,
+                             a_scale, a_offset, w_scale, w_offset, relu=False, skip=None, out=None,
+                             next_t_lo=None, next_t_hi=None, out_packed=None, dbg_acc=None, stream=None):
+    """fp32 NCHW input; y = phi(conv) + skip goes to ``out`` (fp32 [B,N,Ho,Wo]) and / or, ternarized
+    against the next layer's thresholds, to ``out_packed`` (uint8 [B*Ho*Wo, row_bytes(N)]).  The
+    caller passes the buffers it wants filled."""
+    B, Cin, H, W = x.shape
+    _check(lib().rtn_ternary_conv2d_fused(
+        _ptr(x, torch.float32), B, Cin, H, W, _ptr(t_lo, torch.float32), _ptr(t_hi, torch.float32),
+        t_lo.numel(), _ptr(w_packed), _ptr(w_sum, torch.int32), N, kh, kw, stride, pad,
+        int(pad_mode), float(a_scale), float(a_offset), _ptr(w_scale, torch.float32),
+        _ptr(w_offset, torch.float32), w_scale.numel(),
+        *_next_tail(relu, skip, out, next_t_lo, next_t_hi, out_packed, dbg_acc, stream)),
+        "rtn_ternary_conv2d_fused")
+    return out, out_packed
+
+
+def rtn_ternary_conv2d_packed(x_packed, B, Cin, H, W, w_packed, w_sum, N, kh, kw, stride, pad, pad_mode,
+                              a_scale, a_offset, w_scale, w_offset, relu=False, skip=None, out=None,
+                              next_t_lo=None, next_t_hi=None, out_packed=None, dbg_acc=None, stream=None):
+    """The same layer on packed pixel rows (uint8 [B*H*W, row_bytes(Cin)])."""
+    _check(lib().rtn_ternary_conv2d_packed(
+        _ptr(x_packed, torch.uint8), B, Cin, H, W, _ptr(w_packed), _ptr(w_sum, torch.int32), N, kh, kw,
+        stride, pad, int(pad_mode), float(a_scale), float(a_offset), _ptr(w_scale, torch.float32),
+        _ptr(w_offset, torch.float32), w_scale.numel(),
+        *_next_tail(relu, skip, out, next_t_lo, next_t_hi, out_packed, dbg_acc, stream)),
+        "rtn_ternary_conv2d_packed")
+    return out, out_packed
 
 
 def rtn_choose_gemm_variant(M, N, K):

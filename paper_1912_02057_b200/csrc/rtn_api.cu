@@ -176,15 +176,17 @@ static rtn_status fill_conv_args(rtn::ConvArgs& c, const float* x, int64_t B, in
                                  const void* w_packed, const int32_t* w_sum, int64_t N, int64_t kh,
                                  int64_t kw, int64_t stride, int64_t pad, rtn_pad_mode pad_mode,
                                  float a_scale, float a_offset, const float* w_scale,
-                                 const float* w_offset, int64_t n_wparam, float* out, int32_t* dbg_acc)
+                                 const float* w_offset, int64_t n_wparam, float* out, int32_t* dbg_acc,
+                                 bool packed_in = false, bool out_optional = false)
 {
-    if (x == nullptr || t_lo == nullptr || t_hi == nullptr || w_packed == nullptr ||
-        w_sum == nullptr || out == nullptr) return RTN_ERR_NULL;
+    // packed_in: the input is packed pixel rows (x is not used, nor are the thresholds)
+    if (w_packed == nullptr || w_sum == nullptr || (out == nullptr && !out_optional)) return RTN_ERR_NULL;
+    if (!packed_in && (x == nullptr || t_lo == nullptr || t_hi == nullptr)) return RTN_ERR_NULL;
     const int64_t lim = 1 << 20;
     if (B <= 0 || C <= 0 || H <= 0 || W <= 0 || N <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0 ||
         B > lim || C > lim || H > lim || W > lim || N > lim || kh > 64 || kw > 64 || stride > 64 ||
         pad > 64) return RTN_ERR_SHAPE;
-    if (n_thr != 1 && n_thr != C) return RTN_ERR_SHAPE;
+    if (!packed_in && n_thr != 1 && n_thr != C) return RTN_ERR_SHAPE;
     const int64_t Ho = rtn_conv_out_dim(H, kh, stride, pad), Wo = rtn_conv_out_dim(W, kw, stride, pad);
     if (Ho <= 0 || Wo <= 0) return RTN_ERR_SHAPE;
     if (rtn_conv_packed_k(C, kh, kw) > kMaxK) return RTN_ERR_SHAPE;
@@ -192,8 +194,9 @@ static rtn_status fill_conv_args(rtn::ConvArgs& c, const float* x, int64_t B, in
     if (pad_mode != RTN_PAD_CODE_ZERO && pad_mode != RTN_PAD_VALUE_ZERO) return RTN_ERR_VALUE;
     rtn_status st = check_params(w_scale, w_offset, n_wparam, N);
     if (st != RTN_OK) return st;
-    if (!aligned16(w_packed) || !aligned4(x) || !aligned4(out) || !aligned4(w_sum) || !aligned4(t_lo) ||
-        !aligned4(t_hi) || (dbg_acc != nullptr && !aligned4(dbg_acc))) return RTN_ERR_ALIGN;
+    if (!aligned16(w_packed) || !aligned4(out) || !aligned4(w_sum) ||
+        (dbg_acc != nullptr && !aligned4(dbg_acc))) return RTN_ERR_ALIGN;
+    if (!packed_in && (!aligned4(x) || !aligned4(t_lo) || !aligned4(t_hi))) return RTN_ERR_ALIGN;
     c.x = x; c.B = (int)B; c.C = (int)C; c.H = (int)H; c.W = (int)W;
     c.t_lo = t_lo; c.t_hi = t_hi; c.n_thr = (int)n_thr;
     c.w_packed = static_cast<const uint8_t*>(w_packed); c.w_sum = w_sum;
@@ -270,6 +273,68 @@ rtn_status rtn_ternary_conv2d_noalloc(const float* x, int64_t B, int64_t C, int6
     if (c.status == nullptr) return RTN_ERR_CUDA;
     const cudaError_t e = rtn::launch_conv_i8r_static(c, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
+// Common tail of the two entry points that hand the result to the next layer.
+static rtn_status conv_next(rtn::ConvArgs& c, const void* x_packed, int relu, const float* skip,
+                            const float* next_t_lo, const float* next_t_hi, int64_t n_next_thr,
+                            void* out_packed, void* stream)
+{
+    if (c.out == nullptr && out_packed == nullptr) return RTN_ERR_NULL;
+    if (relu != 0 && relu != 1) return RTN_ERR_VALUE;
+    if (out_packed != nullptr) {
+        if (next_t_lo == nullptr || next_t_hi == nullptr) return RTN_ERR_NULL;
+        if (n_next_thr != 1 && n_next_thr != c.N) return RTN_ERR_SHAPE;
+        if (!aligned16(out_packed) || !aligned4(next_t_lo) || !aligned4(next_t_hi)) return RTN_ERR_ALIGN;
+    }
+    if ((x_packed != nullptr && !aligned16(x_packed)) || (skip != nullptr && !aligned4(skip))) return RTN_ERR_ALIGN;
+    if (!rtn::conv_i8r_next_supported(c)) return RTN_ERR_UNSUPPORTED;
+    rtn::NextLayerArgs f{};
+    f.x_packed = static_cast<const uint8_t*>(x_packed);
+    f.relu = relu;
+    f.skip = skip;
+    f.next_lo = next_t_lo; f.next_hi = next_t_hi; f.n_next = (int)n_next_thr;
+    f.out_packed = static_cast<uint8_t*>(out_packed);
+    c.status = status_word();
+    if (c.status == nullptr) return RTN_ERR_CUDA;
+    const cudaError_t e = rtn::launch_conv_i8r_next(c, f, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
+rtn_status rtn_ternary_conv2d_fused(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
+                                    const float* t_lo, const float* t_hi, int64_t n_thr,
+                                    const void* w_packed, const int32_t* w_sum,
+                                    int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                                    rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                                    const float* w_scale, const float* w_offset, int64_t n_wparam,
+                                    int relu, const float* skip, float* out,
+                                    const float* next_t_lo, const float* next_t_hi, int64_t n_next_thr,
+                                    void* out_packed, int32_t* dbg_acc, void* stream)
+{
+    rtn::ConvArgs c{};
+    rtn_status st = fill_conv_args(c, x, B, C, H, W, t_lo, t_hi, n_thr, w_packed, w_sum, N, kh, kw,
+                                   stride, pad, pad_mode, a_scale, a_offset, w_scale, w_offset,
+                                   n_wparam, out, dbg_acc, false, true);
+    if (st != RTN_OK) return st;
+    return conv_next(c, nullptr, relu, skip, next_t_lo, next_t_hi, n_next_thr, out_packed, stream);
+}
+
+rtn_status rtn_ternary_conv2d_packed(const void* x_packed, int64_t B, int64_t C, int64_t H, int64_t W,
+                                     const void* w_packed, const int32_t* w_sum,
+                                     int64_t N, int64_t kh, int64_t kw, int64_t stride, int64_t pad,
+                                     rtn_pad_mode pad_mode, float a_scale, float a_offset,
+                                     const float* w_scale, const float* w_offset, int64_t n_wparam,
+                                     int relu, const float* skip, float* out,
+                                     const float* next_t_lo, const float* next_t_hi, int64_t n_next_thr,
+                                     void* out_packed, int32_t* dbg_acc, void* stream)
+{
+    if (x_packed == nullptr) return RTN_ERR_NULL;
+    rtn::ConvArgs c{};
+    rtn_status st = fill_conv_args(c, nullptr, B, C, H, W, nullptr, nullptr, 1, w_packed, w_sum, N, kh, kw,
+                                   stride, pad, pad_mode, a_scale, a_offset, w_scale, w_offset,
+                                   n_wparam, out, dbg_acc, true, true);
+    if (st != RTN_OK) return st;
+    return conv_next(c, x_packed, relu, skip, next_t_lo, next_t_hi, n_next_thr, out_packed, stream);
 }
 
 rtn_status rtn_last_device_status(void* stream)

@@ -68,14 +68,14 @@ struct ConvI8RPlan {
     uint32_t tmem_cols;
     int64_t Ptot, Pstride; // padded pixels of the batch; pixels per chunk row of the scratch (with slack)
     FastDiv div_pw, div_ph, div_nq, div_cw;
-    uint32_t off_w, off_c, off_bar, off_misc, off_slot, slot_bytes;
+    uint32_t off_w, off_c, off_t, off_bar, off_misc, off_slot, slot_bytes;
     size_t smem_bytes;
     size_t codes_bytes, scratch_bytes;     // scratch = codes, then the per-pixel sums
     uint32_t tap_shift[kMaxTaps];          // start of the tap's A window inside a slot, 16-byte units
     uint32_t tap_psum[kMaxTaps];           // the tap's offset into the per-pixel sums
 };
 
-bool make_plan_r(const ConvArgs& c, ConvI8RPlan& p, int sms)
+bool make_plan_r(const ConvArgs& c, ConvI8RPlan& p, int sms, bool fused = false)
 {
     if (c.stride < 1 || c.Ho <= 0 || c.Wo <= 0) return false;
     p.T = c.kh * c.kw;
@@ -130,6 +130,7 @@ bool make_plan_r(const ConvArgs& c, ConvI8RPlan& p, int sms)
         uint32_t o = 0;
         p.off_w = o;    o += (uint32_t)p.T * (uint32_t)(p.Cp / 16) * (uint32_t)p.Nq * 16u;
         p.off_c = o;    o += (uint32_t)p.Nq * 16u;
+        p.off_t = o;    o += fused ? (uint32_t)p.Nq * 8u : 0u;     // next layer's {t_lo, t_hi} per column
         p.off_bar = o;  o += (2 * kMaxSlots + 2 * kMaxAcc + 1) * 8;
         p.off_misc = o; o += 16;
         o = (o + 127) / 128 * 128;
@@ -232,6 +233,58 @@ conv_codes_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, uint4
     }
 }
 
+// Kernel 1 for an input that arrives as packed pixel rows (the layer before wrote them from its
+// epilogue, or rtn_ternarize_pack_act did): bit planes -> the same int8 code layout and per-pixel sums.
+// 0.25 B read and about 1 B written per value.  Same block shape: lanes run along pixels, so the
+// 16-byte code stores of a warp are contiguous; the word loads of a warp touch 32 pixel rows whose
+// other words the block's other channel groups read (served by L1).
+__global__ void __launch_bounds__(kCodePixels * kCodeGroups)
+conv_codes_packed_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p,
+                         const uint8_t* __restrict__ x_packed, uint4* __restrict__ codes, int* __restrict__ psum)
+{
+    __shared__ int sSum[kCodeGroups * kCodePixels];
+    tc::pdl_trigger();
+    const int px = threadIdx.x % kCodePixels, gi = threadIdx.x / kCodePixels;
+    const int64_t P = (int64_t)blockIdx.x * kCodePixels + px;
+    const int w = blockIdx.y;                               // phase image
+    codes += (int64_t)w * (p.Cp / 16) * p.Pstride;
+    psum += (int64_t)w * p.Pstride;
+    const int64_t row_bytes = (int64_t)((a.C + kBlockCodes - 1) / kBlockCodes) * kBlockBytes;
+    const uint32_t* src0 = nullptr;
+    if (P < p.Ptot) {
+        const uint32_t G = fdiv((uint32_t)P, p.div_pw);
+        const int col = (int)((uint32_t)P - G * (uint32_t)p.PW) * a.stride + p.ph_c[w] - a.pad;
+        const uint32_t b = fdiv(G, p.div_ph);
+        const int r = (int)(G - b * (uint32_t)p.PH) * a.stride + p.ph_r[w] - a.pad;
+        if (r >= 0 && r < a.H && col >= 0 && col < a.W)
+            src0 = reinterpret_cast<const uint32_t*>(x_packed + (((int64_t)b * a.H + r) * a.W + col) * row_bytes);
+    }
+    int sum = 0;
+    for (int h = gi; h < p.ngroup; h += kCodeGroups) {
+        uint32_t nz = 0, sg = 0;
+        if (src0 != nullptr) {
+            const uint32_t* blk = src0 + (h >> 2) * 8 + (h & 3);
+            nz = __ldg(blk);
+            sg = __ldg(blk + 4);
+            if (h * 32 + 32 > a.C) nz &= (1u << (a.C - h * 32)) - 1u;      // positions past C code to 0
+        }
+        uint32_t o[8];
+        tc::unpack32(nz, sg, o);
+        sum += __popc(nz & sg) - __popc(nz & ~sg);
+        if (P < p.Pstride) {
+            codes[(int64_t)(2 * h) * p.Pstride + P] = make_uint4(o[0], o[1], o[2], o[3]);
+            codes[(int64_t)(2 * h + 1) * p.Pstride + P] = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+    }
+    sSum[gi * kCodePixels + px] = sum;
+    __syncthreads();
+    if (gi == 0 && P < p.Pstride) {
+        int t = 0;
+        for (int k = 0; k < kCodeGroups; ++k) t += sSum[k * kCodePixels + px];
+        psum[P] = t;
+    }
+}
+
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -252,9 +305,12 @@ __device__ __forceinline__ void role_wait_r(bool leader, uint64_t* bar, uint32_t
 // ------------------------------------------------------------------------------------------------
 // Kernel 2: the contraction and the epilogue.
 // ------------------------------------------------------------------------------------------------
+// kFused: the epilogue also applies phi, adds the skip connection, and hands the result to the next
+// layer as fp32 and / or as packed Eq. 3 codes against that layer's thresholds (NextLayerArgs).
+template <bool kFused>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const uint4* __restrict__ codes,
-                const int* __restrict__ psum)
+                const int* __restrict__ psum, const NextLayerArgs f)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     uint4* sW = reinterpret_cast<uint4*>(smem + p.off_w);        // [T][Cp/16][Nq]
@@ -334,6 +390,17 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
                 c3 = (float)(a_o * (ws * (double)a.w_sum[n] + (double)a.C * p.T * wo));
             }
             sC[r] = make_float4(c1, c2, c3, 0.f);
+        }
+    }
+    if constexpr (kFused) {
+        // the next layer's threshold pair per column (as in the ternarizers: +1 is tested first)
+        float2* sT = reinterpret_cast<float2*>(smem + p.off_t);
+        for (int r = threadIdx.x; r < p.Nq; r += kThreads) {
+            const int n = n_base + r;
+            float2 t = make_float2(-INFINITY, INFINITY);
+            if (f.out_packed != nullptr && n < a.N)
+                t = make_float2(f.next_lo[f.n_next == 1 ? 0 : n], f.next_hi[f.n_next == 1 ? 0 : n]);
+            sT[r] = t;
         }
     }
     tc::fence_smem_to_async_proxy();
@@ -466,6 +533,21 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
             const float fsx = (float)s_x;
             const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.Nq);
             const int64_t obase = (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
+            // packed output: this pixel's row of N codes; positions from N to the end of the last
+            // 128-code block are zero-filled (by the last filter group's first warp set)
+            const int packed_cols = (a.N + kBlockCodes - 1) / kBlockCodes * kBlockCodes;
+            uint8_t* out_row = nullptr;
+            if constexpr (kFused) {
+                if (ok && f.out_packed != nullptr) {
+                    out_row = f.out_packed + (((int64_t)b * a.Ho + ho) * a.Wo + wo) * (int64_t)(packed_cols / 4);
+                    if (fq == p.S - 1 && half == 0)
+                        for (int n0 = p.S * p.Nq; n0 < packed_cols; n0 += 16) {
+                            uint8_t* dst = out_row + (n0 >> 7) * kBlockBytes + ((n0 & 127) >> 3);
+                            *reinterpret_cast<uint16_t*>(dst) = 0;
+                            *reinterpret_cast<uint16_t*>(dst + 16) = 0;
+                        }
+                }
+            }
             for (int blk = blk_begin; blk < blk_end; ++blk) {
                 uint32_t v[16];
                 tc::tmem_ld16(trow + (uint32_t)(blk * 16), v);
@@ -473,6 +555,45 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
                 if (!ok) continue;
                 const int r0 = blk * 16;                   // column of the accumulator = row of the filter group
                 const int n0 = n_base + r0;
+                if constexpr (kFused) {
+                    const float2* sT = reinterpret_cast<const float2*>(smem + p.off_t);
+                    uint32_t nzb = 0, sgb = 0;             // the 16 codes of this block, one bit each per plane
+                    #pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int n = n0 + j;
+                        if (n >= a.N) continue;
+                        const int s_xw = (int)v[j];
+                        const float4 c = sC[r0 + j];
+                        float c3 = c.z;
+                        if (border) {
+                            int s_w = 0;
+                            for (int t = 0; t < p.T; ++t) {
+                                const int h = ho * a.stride - a.pad + t / a.kw, vv = wo * a.stride - a.pad + t % a.kw;
+                                if (h >= 0 && h < a.H && vv >= 0 && vv < a.W) s_w += a.w_sum[(1 + t) * a.N + n];
+                            }
+                            const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
+                            const double wo_ = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
+                            c3 = (float)((double)a.ep.a_offset_val *
+                                         (ws * (double)s_w + (double)a.C * n_inside * wo_));
+                        }
+                        float y = fmaf(c.x, (float)s_xw, fmaf(c.y, fsx, c3));
+                        if (f.relu) y = y > 0.f ? y : 0.f;
+                        const int64_t o = obase + (int64_t)n * ostride;
+                        if (f.skip != nullptr) y += __ldg(f.skip + o);
+                        if (a.out != nullptr) a.out[o] = y;
+                        if (a.dbg_acc != nullptr) a.dbg_acc[o] = s_xw;
+                        const float2 t = sT[r0 + j];
+                        const bool pos = y > t.y, neg = !pos && y < t.x;
+                        nzb |= (uint32_t)(pos || neg) << j;
+                        sgb |= (uint32_t)pos << j;
+                    }
+                    if (f.out_packed != nullptr && n0 < packed_cols) {
+                        uint8_t* dst = out_row + (n0 >> 7) * kBlockBytes + ((n0 & 127) >> 3);
+                        *reinterpret_cast<uint16_t*>(dst) = (uint16_t)nzb;
+                        *reinterpret_cast<uint16_t*>(dst + 16) = (uint16_t)sgb;
+                    }
+                    continue;
+                }
                 float* optr = a.out + obase + (int64_t)n0 * ostride;
                 if (!border && a.dbg_acc == nullptr && n0 + 16 <= a.N) {
                     #pragma unroll
@@ -547,19 +668,30 @@ int sm_count_r()
     return sms;
 }
 
-cudaError_t launch_with_scratch(const ConvArgs& c, const ConvI8RPlan& p, void* scratch, cudaStream_t s)
+cudaError_t launch_with_scratch(const ConvArgs& c, const ConvI8RPlan& p, void* scratch, cudaStream_t s,
+                                const NextLayerArgs* f = nullptr)
 {
     uint4* codes = reinterpret_cast<uint4*>(scratch);
     int* psum = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(scratch) + p.codes_bytes);
     const dim3 blocks((unsigned)((p.Pstride + kCodePixels - 1) / kCodePixels), (unsigned)p.nph);
-    const size_t smem1 = (size_t)p.Cp * 8 + (size_t)kCodeGroups * kCodePixels * 4;
-    conv_codes_kernel<<<blocks, kCodePixels * kCodeGroups, smem1, s>>>(c, p, codes, psum);
+    if (f != nullptr && f->x_packed != nullptr) {
+        conv_codes_packed_kernel<<<blocks, kCodePixels * kCodeGroups, 0, s>>>(c, p, f->x_packed, codes, psum);
+    } else {
+        const size_t smem1 = (size_t)p.Cp * 8 + (size_t)kCodeGroups * kCodePixels * 4;
+        conv_codes_kernel<<<blocks, kCodePixels * kCodeGroups, smem1, s>>>(c, p, codes, psum);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(conv_i8r_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    if (f != nullptr) {
+        e = cudaFuncSetAttribute(conv_i8r_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+        if (e != cudaSuccess) return e;
+        return launch_pdl(conv_i8r_kernel<true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
+                          (const uint4*)codes, (const int*)psum, *f);
+    }
+    e = cudaFuncSetAttribute(conv_i8r_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
-    return launch_pdl(conv_i8r_kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
-                      (const uint4*)codes, (const int*)psum);
+    return launch_pdl(conv_i8r_kernel<false>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
+                      (const uint4*)codes, (const int*)psum, NextLayerArgs{});
 }
 
 }  // namespace
@@ -568,6 +700,12 @@ bool conv_i8r_supported(const ConvArgs& c)
 {
     ConvI8RPlan p;
     return make_plan_r(c, p, 148);
+}
+
+bool conv_i8r_next_supported(const ConvArgs& c)
+{
+    ConvI8RPlan p;
+    return make_plan_r(c, p, 148, true);
 }
 
 size_t conv_i8r_scratch_bytes(const ConvArgs& c)
@@ -604,5 +742,19 @@ cudaError_t launch_conv_i8r_static(const ConvArgs& c, cudaStream_t s)
 }
 
 size_t conv_i8r_static_scratch_bytes() { return kStaticScratchBytes; }
+
+// The two launches with the hand-over to the next layer fused into the second one's epilogue; the
+// first one reads fp32 (Eq. 3 in-kernel) or packed pixel rows.  Scratch as in launch_conv_i8r.
+cudaError_t launch_conv_i8r_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s)
+{
+    ConvI8RPlan p;
+    if (!make_plan_r(c, p, sm_count_r(), true)) return cudaErrorInvalidConfiguration;
+    void* scratch = nullptr;
+    cudaError_t e = cudaMallocAsync(&scratch, p.scratch_bytes, s);
+    if (e != cudaSuccess) return e;
+    e = launch_with_scratch(c, p, scratch, s, &f);
+    const cudaError_t e2 = cudaFreeAsync(scratch, s);
+    return e != cudaSuccess ? e : e2;
+}
 
 }  // namespace rtn

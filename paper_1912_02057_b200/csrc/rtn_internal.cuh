@@ -58,6 +58,20 @@ struct ConvArgs {
     unsigned* status;
 };
 
+// What a conv layer hands to the next one, fused into its epilogue (every member optional):
+//   y = phi(affine form) + skip;  out <- y (fp32);  out_packed <- Eq. 3 codes of y against the
+//   NEXT layer's thresholds, as packed pixel rows.  x_packed != NULL: the layer's own input comes as
+//   packed pixel rows ([B*H*W] rows of C codes) instead of fp32 (ConvArgs::x, t_lo, t_hi unused).
+struct NextLayerArgs {
+    const uint8_t* x_packed;
+    int relu;               // phi of Eq. 10
+    const float* skip;      // fp32 [B][N][Ho][Wo], added after phi
+    const float* next_lo;   // thresholds of the next layer's ternarizer: n_next = 1 or N entries
+    const float* next_hi;
+    int n_next;
+    uint8_t* out_packed;    // [B*Ho*Wo] packed rows of N codes
+};
+
 // Launchers (each returns the cudaError_t of its launch).
 cudaError_t launch_pack_weights(const int8_t* w, int64_t N, int64_t C, int kh, int kw,
                                 uint8_t* packed, int32_t* w_sum, unsigned* status, cudaStream_t s);
@@ -80,6 +94,9 @@ size_t conv_i8r_scratch_bytes(const ConvArgs& c);
 cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s);     // scratch from the stream-ordered allocator
 cudaError_t launch_conv_i8r_static(const ConvArgs& c, cudaStream_t s);      // scratch in a static device array
 size_t conv_i8r_static_scratch_bytes();
+// Two-kernel path with the fused hand-over to the next layer (and, optionally, packed input).
+bool conv_i8r_next_supported(const ConvArgs& c);
+cudaError_t launch_conv_i8r_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s);
 inline bool conv_i8_any_supported(const ConvArgs& c)
 {
     return conv_i8_supported(c) || conv_i8s_supported(c) || conv_i8r_supported(c);
