@@ -45,6 +45,8 @@ WORKLOADS = {
 for _l in inputs.resnet18_ternary_layers():
     WORKLOADS[f"r18_{_l[0]}_b128"] = (lambda n=_l[0]: inputs.resnet18_layer(n, batch=128))
 DEFAULT_WORKLOAD = "cfg2_conv3x3_c64_56x56_b32"
+# --io packed: thresholds of the next layer's ternarizer (per layer), applied to phi(conv output)
+NEXT_THRESHOLDS = (0.5, 2.0)
 
 
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -145,8 +147,17 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def algorithmic_bytes(case):
-    """Bytes the method must move per step: the fp32 input it touches once, fp32 output once, packed weights once."""
+def algorithmic_bytes(case, io="fp32"):
+    """Bytes the method must move per step: the fp32 input it touches once, fp32 output once, packed weights once.
+    io == "packed": input and output are packed pixel rows (2 bits per value, rows of whole 32-byte blocks)."""
+    if isinstance(case, inputs.ConvCase) and io == "packed":
+        M, N, K = case.gemm_mnk
+        kc = case.kh * case.kw * ((case.C + 31) // 32 * 32)
+        rows = {ho * case.stride - case.pad + i for ho in range(case.Ho) for i in range(case.kh)}
+        cols = {wo * case.stride - case.pad + j for wo in range(case.Wo) for j in range(case.kw)}
+        touched = len([r for r in rows if 0 <= r < case.H]) * len([c for c in cols if 0 <= c < case.W])
+        row_bytes = lambda k: (k + 127) // 128 * 32
+        return case.B * touched * row_bytes(case.C) + M * row_bytes(N) + N * row_bytes(kc)
     if isinstance(case, inputs.ConvCase):
         M, N, K = case.gemm_mnk
         kc = case.kh * case.kw * ((case.C + 31) // 32 * 32)
@@ -169,7 +180,7 @@ def ops_of(case):
 # ------------------------------------------------------------------------------------------------
 # CPU oracle leg (reference arm and cpu_baseline)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample(case, budget_s=12.0):
+def oracle_sample(case, budget_s=12.0, io="fp32"):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload.
     Returns (ops per second, seconds, description)."""
     import oracle
@@ -178,8 +189,11 @@ def oracle_sample(case, budget_s=12.0):
             x = case.x[:nb]
             t0 = time.perf_counter()
             codes = oracle.ternarize(x, case.t_lo, case.t_hi, channel_axis=1)
-            oracle.conv2d(codes, case.w_codes, case.stride, case.pad, oracle.PAD_CODE_ZERO,
-                          case.a_scale, case.a_offset, case.w_scale, case.w_offset)
+            _, pre, _ = oracle.conv2d(codes, case.w_codes, case.stride, case.pad, oracle.PAD_CODE_ZERO,
+                                      case.a_scale, case.a_offset, case.w_scale, case.w_offset)
+            if io == "packed":
+                _, nxt, _ = oracle.next_layer(pre, True, None, *NEXT_THRESHOLDS)
+                oracle.pack_nhwc(nxt)
             dt = time.perf_counter() - t0
             M, N, K = case.gemm_mnk
             return 2.0 * (M // case.B * nb) * N * K, dt
@@ -215,10 +229,10 @@ def run_reference(args, case, name):
     per_step_budget = max(0.2, min(12.0, 60.0 / max(1, args.steps + args.warmup)))
     sample = ""
     for _ in range(args.warmup):
-        _, _, sample = oracle_sample(case, per_step_budget)
+        _, _, sample = oracle_sample(case, per_step_budget, args.io)
     rates, secs = [], []
     for _ in range(args.steps):
-        r, dt, sample = oracle_sample(case, per_step_budget)
+        r, dt, sample = oracle_sample(case, per_step_budget, args.io)
         rates.append(r)
         secs.append(dt)
     value = float(np.mean(rates)) / 1e12
@@ -227,7 +241,7 @@ def run_reference(args, case, name):
         "unit": "TOPS", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * float(np.mean(secs)), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": name, "note": "CPU oracle on a bounded sample per step"},
+        "config": {"workload": name, "io": args.io, "note": "CPU oracle on a bounded sample per step"},
         "cpu_baseline": {"value": value, "unit": "TOPS", "cores": oracle.threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -270,13 +284,35 @@ def run_ours(args, case, name):
     is_conv = isinstance(case, inputs.ConvCase)
 
     # resident inputs: enough rotating copies that consecutive steps never find their data in L2
-    step_bytes = algorithmic_bytes(case)
+    packed_io = is_conv and args.io == "packed"
+    step_bytes = algorithmic_bytes(case, args.io if is_conv else "fp32")
     n_sets = max(2, int(np.ceil(2.5 * L2_BYTES / step_bytes)))
     n_sets = min(n_sets, 64)
     w_packed, w_sum = rtn.rtn_pack_weights(dev(case.w_codes))
     w_s, w_o = dev(case.w_scale), dev(case.w_offset)
     t_lo, t_hi = dev(case.t_lo), dev(case.t_hi)
-    if is_conv:
+    if packed_io:
+        # input: packed pixel rows (what the layer before hands over); output: packed rows for the next
+        # layer (phi = ReLU, that layer's thresholds), no fp32 tensor at either end
+        nhwc = dev(np.ascontiguousarray(case.x.transpose(0, 2, 3, 1)).reshape(-1, case.C))
+        x0, _ = rtn.rtn_ternarize_pack_act(nhwc, t_lo, t_hi, want_sum=False)
+        del nhwc
+        xs = [x0.clone() for _ in range(n_sets)]
+        outs = [torch.empty((case.B * case.Ho * case.Wo, rtn.rtn_packed_row_bytes(case.N)), dtype=torch.uint8,
+                            device="cuda") for _ in range(n_sets)]
+        n_lo, n_hi = (dev(np.array([v], np.float32)) for v in NEXT_THRESHOLDS)
+        variant = 2
+        launches_per_step = 2
+
+        def step(i):
+            j = i % n_sets
+            rtn.rtn_ternary_conv2d_packed(xs[j], case.B, case.C, case.H, case.W, w_packed, w_sum, case.N,
+                                          case.kh, case.kw, case.stride, case.pad, rtn.PAD_CODE_ZERO,
+                                          case.a_scale, case.a_offset, w_s, w_o, relu=True,
+                                          next_t_lo=n_lo, next_t_hi=n_hi, out_packed=outs[j])
+            return outs[j]
+        host_in = x0.cpu().pin_memory()
+    elif is_conv:
         xs = [dev(case.x) for _ in range(n_sets)]
         outs = [torch.empty((case.B, case.N, case.Ho, case.Wo), dtype=torch.float32, device="cuda")
                 for _ in range(n_sets)]
@@ -310,7 +346,7 @@ def run_ours(args, case, name):
                                  out=outs[j])
             return outs[j]
         host_in = torch.from_numpy(case.a).pin_memory()
-    host_out = torch.empty(outs[0].shape, dtype=torch.float32).pin_memory()
+    host_out = torch.empty(outs[0].shape, dtype=outs[0].dtype).pin_memory()
 
     def barrier():
         if world > 1:
@@ -421,7 +457,8 @@ def run_ours(args, case, name):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int32 accumulate (int8 / 1-bit-plane operands), fp32 epilogue",
             "data": "synthetic",
-            "config": {"workload": name, "variant": {1: "popc", 2: "i8"}[variant],
+            "config": {"workload": name, "io": args.io if is_conv else "fp32",
+                       "variant": {1: "popc", 2: "i8"}[variant],
                        "l2": f"{n_sets} rotating input/output sets ({n_sets * step_bytes >> 20} MiB) > L2",
                        "thresholds": "t_lo = a_offset - 0.5, t_hi = a_offset + 0.5" if is_conv else
                                      "per layer, as the workload names them",
@@ -430,14 +467,14 @@ def run_ours(args, case, name):
                        "parallelism": "replicas only" if world > 1 else "1 GPU"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": int(host_in.numel() * 4),
-                    "d2h_bytes_per_step": int(host_out.numel() * 4)},
+                    "h2d_bytes_per_step": int(host_in.numel() * host_in.element_size()),
+                    "d2h_bytes_per_step": int(host_out.numel() * host_out.element_size())},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline_of(name, kernel_bytes, ops, kernel_ms),
+            "roofline": roofline_of(name if not packed_io else name + "/packed", kernel_bytes, ops, kernel_ms),
         }
         if not args.no_cpu_baseline and world == 1:
             import oracle
-            rate, dt, sample = oracle_sample(case, 12.0)
+            rate, dt, sample = oracle_sample(case, 12.0, args.io)
             line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TOPS", "cores": oracle.threads(),
                                     "kind": "oracle", "sample": sample, "seconds": dt}
         print(json.dumps(line))
@@ -452,6 +489,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--io", default="fp32", choices=["fp32", "packed"],
+                    help="conv workloads: fp32 NCHW in and out (rtn_ternary_conv2d), or packed pixel rows in and "
+                         "out with the hand-over to the next layer fused (rtn_ternary_conv2d_packed)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true",
                     help="launch the timed steps one by one instead of through a CUDA graph (for profilers)")
