@@ -288,7 +288,8 @@ static rtn_status conv_next(rtn::ConvArgs& c, const void* x_packed, int relu, co
         if (!aligned16(out_packed) || !aligned4(next_t_lo) || !aligned4(next_t_hi)) return RTN_ERR_ALIGN;
     }
     if ((x_packed != nullptr && !aligned16(x_packed)) || (skip != nullptr && !aligned4(skip))) return RTN_ERR_ALIGN;
-    if (!rtn::conv_i8r_next_supported(c)) return RTN_ERR_UNSUPPORTED;
+    const bool one_kernel = rtn::conv_i8_next_supported(c);
+    if (!one_kernel && !rtn::conv_i8r_next_supported(c)) return RTN_ERR_UNSUPPORTED;
     rtn::NextLayerArgs f{};
     f.x_packed = static_cast<const uint8_t*>(x_packed);
     f.relu = relu;
@@ -297,7 +298,8 @@ static rtn_status conv_next(rtn::ConvArgs& c, const void* x_packed, int relu, co
     f.out_packed = static_cast<uint8_t*>(out_packed);
     c.status = status_word();
     if (c.status == nullptr) return RTN_ERR_CUDA;
-    const cudaError_t e = rtn::launch_conv_i8r_next(c, f, static_cast<cudaStream_t>(stream));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const cudaError_t e = one_kernel ? rtn::launch_conv_i8_next(c, f, s) : rtn::launch_conv_i8r_next(c, f, s);
     return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
 }
 

@@ -86,14 +86,14 @@ struct ConvI8Plan {
     uint32_t box_bytes;    // one TMA box: 32 channels x one image row of fp32
     int nslots;            // row slots of the TMA ring
     uint32_t off_stage;
-    uint32_t off_a[2], off_w, off_lo, off_hi, off_c, off_rows, off_bar, off_misc;
+    uint32_t off_a[2], off_w, off_lo, off_hi, off_c, off_t, off_rows, off_bar, off_misc;
     size_t smem_bytes;
     // Per MMA of a sub-tile (tap t, channel group h), in 16-byte units: start of the A window
     // relative to the code buffer, start of the filter slice relative to the filter array.
     uint32_t tab_a[kMaxMma], tab_b[kMaxMma];
 };
 
-bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
+bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms, bool next = false)
 {
     if (c.stride != 1) return false;
     if (c.Ho <= 0 || c.Wo <= 0) return false;
@@ -147,6 +147,7 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms)
     p.off_hi = o;   o += (uint32_t)p.Cp * 4;
     o = (o + 15) / 16 * 16;
     p.off_c = o;    o += (uint32_t)p.Np * 16;           // float4 {c1, c2, c3, 0} per column
+    p.off_t = o;    o += next ? (uint32_t)p.Np * 8 : 0; // float2 {t_lo, t_hi} of the next layer per column
     p.off_rows = o; o += kMaxSlots * 4;                 // producer's row table
     p.off_bar = o;  o += (7 + 2 * kMaxStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] st_full[] st_empty[] a_full[2][groups]
     p.off_misc = o; o += 16;                            // tmem slot, dead flag
@@ -214,8 +215,86 @@ __device__ __forceinline__ void issue_mmas(const ConvI8Plan& p, int i0, uint32_t
     for (int j = 1; j < NB; ++j) tc::mma_i8_ss_acc(d, desc_hi | la[j], desc_hi | lb[j], idesc);
 }
 
+// Hand-over epilogue (NextLayerArgs) of one tile for one warp.  The warp reads TMEM lanes 32 q .. 32 q + 31
+// (pixels).  Unit of work = (sub-tile, block of 128 output channels), dealt to the two warps of a lane quarter
+// in turn: a thread then holds all 128 codes of its pixel and writes each bit plane of the packed row with
+// one 16-byte store.  Constants and the next layer's thresholds come from shared memory.
+__device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const ConvI8Plan& p, const NextLayerArgs& f,
+                                                   const float4* sC, const float2* sT, uint32_t tmem, int buf, int g,
+                                                   int nrows, bool alive, int q, int lane, int half)
+{
+    const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
+    const int64_t ostride = (int64_t)a.Ho * a.Wo;
+    const int nblk16 = (a.N + 15) / 16;
+    const int ncb = (a.N + kBlockCodes - 1) / kBlockCodes;
+    for (int tm = 0; tm < ntm; ++tm) {
+        const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);     // pixel within the tile
+        const uint32_t row = fdiv(pl, p.div_pw);
+        const int wo = (int)(pl - row * (uint32_t)p.PW);
+        const uint32_t G = (uint32_t)g + row;
+        const uint32_t b = fdiv(G, p.div_ph);
+        const int ho = (int)(G - b * (uint32_t)p.PH);
+        const bool ok = alive && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
+        int n_inside = p.T;
+        if (ok && a.pad_mode == RTN_PAD_VALUE_ZERO) {
+            n_inside = 0;
+            for (int t = 0; t < p.T; ++t) {
+                const int h = ho - a.pad + t / a.kw, v = wo - a.pad + t % a.kw;
+                n_inside += (h >= 0 && h < a.H && v >= 0 && v < a.W);
+            }
+        }
+        const bool border = n_inside < p.T;
+        const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + tm) * p.Np);
+        const int64_t obase = (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
+        uint8_t* out_row = nullptr;
+        if (ok && f.out_packed != nullptr)
+            out_row = f.out_packed + (((int64_t)b * a.Ho + ho) * a.Wo + wo) * (int64_t)(ncb * kBlockBytes);
+        // S_x of this pixel: accumulator column N (the all-ones filter row)
+        uint32_t sx_raw;
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
+                     : "=r"(sx_raw) : "r"(trow + (uint32_t)a.N) : "memory");
+        bool sx_ready = false;
+        float fsx = 0.f;
+        for (int cb = 0; cb < ncb; ++cb) {
+            if (((tm * ncb + cb) & 1) != half) continue;
+            uint32_t nzw[4] = {0u, 0u, 0u, 0u}, sgw[4] = {0u, 0u, 0u, 0u};
+            #pragma unroll 1
+            for (int k = 0; k < 8; ++k) {
+                const int n0 = cb * kBlockCodes + k * 16;
+                if (n0 >= nblk16 * 16) break;
+                uint32_t u[16];
+                tc::tmem_ld16(trow + (uint32_t)n0, u);
+                tc::tmem_ld_wait();
+                if (!sx_ready) { fsx = (float)(int)sx_raw; sx_ready = true; }
+                if (!ok) continue;
+                uint32_t nzb, sgb;
+                next_layer_block16(a, f, u, sC + n0, sT + n0, fsx, border, p.T, ho, wo, n_inside, n0,
+                                   obase + (int64_t)n0 * ostride, ostride, out_row != nullptr, nzb, sgb);
+                nzb <<= 16 * (k & 1);
+                sgb <<= 16 * (k & 1);
+                #pragma unroll
+                for (int w = 0; w < 4; ++w) {               // word k/2, without indexing the registers
+                    nzw[w] |= (k >> 1) == w ? nzb : 0u;
+                    sgw[w] |= (k >> 1) == w ? sgb : 0u;
+                }
+            }
+            if (out_row != nullptr) {                       // codes past N are the row's zero fill
+                uint4* dst = reinterpret_cast<uint4*>(out_row + cb * kBlockBytes);
+                dst[0] = make_uint4(nzw[0], nzw[1], nzw[2], nzw[3]);
+                dst[1] = make_uint4(sgw[0], sgw[1], sgw[2], sgw[3]);
+            }
+        }
+        if (!sx_ready) tc::tmem_ld_wait();              // the S_x load still has to land
+    }
+}
+
+// kNext: the layer hands its result to the next one (NextLayerArgs): the input may come as packed pixel
+// rows (the converters then expand bit planes instead of ternarizing fp32), and the epilogue applies
+// phi, adds the skip connection and writes fp32 and / or packed Eq. 3 codes.
+template <bool kNext>
 __global__ void __launch_bounds__(kThreads, 1)
-conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __grid_constant__ CUtensorMap tmap)
+conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __grid_constant__ CUtensorMap tmap,
+               const NextLayerArgs f)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     uint4* sW = reinterpret_cast<uint4*>(smem + p.off_w);        // [T][Cp/16][Np]
@@ -269,8 +348,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         // consecutive lanes take consecutive padded pixels: conflict-free reads of a staged row,
         // coalesced global loads on the direct path, conflict-free 16-byte stores of the codes
         const int tid = conv_warp_index(warp) * 32 + lane;
+        bool packed_in = false;
+        if constexpr (kNext) packed_in = f.x_packed != nullptr;
         // thresholds (their global-load latency overlaps the first TMA loads, already in flight)
-        for (int c = tid; c < p.Cp; c += kConvThreads) {
+        for (int c = tid; c < p.Cp && !packed_in; c += kConvThreads) {
             // channel padding: thresholds that code everything to 0
             float lo = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
             const float hi = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
@@ -305,7 +386,34 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     sA[ch * p.ppix + x] = prev[ch * p.ppix + prev_rows * p.PW + x];
                 }
             }
-            if (p.use_tma) {
+            if (packed_in) {
+                // packed pixel rows: item = (padded pixel, 32-channel group) = one word of each bit plane
+                // -> 32 int8 codes (two 16-byte chunks)
+                if constexpr (kNext) {
+                    const int npix = pp1 - pp0;
+                    const int64_t row_bytes = (int64_t)((a.C + kBlockCodes - 1) / kBlockCodes) * kBlockBytes;
+                    for (int i = tid; i < ngroup * npix; i += kConvThreads) {
+                        const int grp = i / npix, pp = pp0 + (i - grp * npix);
+                        const uint32_t sl = fdiv((uint32_t)pp, p.div_pw);
+                        const int c = (int)((uint32_t)pp - sl * (uint32_t)p.PW) - a.pad;
+                        const uint32_t G = (uint32_t)g + sl;
+                        const uint32_t b = fdiv(G, p.div_ph);
+                        const int r = (int)(G - b * (uint32_t)p.PH) - a.pad;
+                        uint32_t nz = 0, sg = 0;
+                        if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
+                            const uint32_t* blk = reinterpret_cast<const uint32_t*>(
+                                f.x_packed + (((int64_t)b * a.H + r) * a.W + c) * row_bytes) + (grp >> 2) * 8 + (grp & 3);
+                            nz = __ldg(blk);
+                            sg = __ldg(blk + 4);
+                            if (grp * 32 + 32 > a.C) nz &= (1u << (a.C - grp * 32)) - 1u;      // positions past C code to 0
+                        }
+                        uint32_t o[8];
+                        tc::unpack32(nz, sg, o);
+                        sA[(2 * grp) * p.ppix + pp] = make_uint4(o[0], o[1], o[2], o[3]);
+                        sA[(2 * grp + 1) * p.ppix + pp] = make_uint4(o[4], o[5], o[6], o[7]);
+                    }
+                }
+            } else if (p.use_tma) {
                 const int npix = pp1 - pp0;
                 for (int grp = 0; grp < ngroup; ++grp, ++st_count) {
                     const uint32_t s = st_count % (uint32_t)kMaxStages;
@@ -566,6 +674,16 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 }
                 sC[n] = make_float4(c1, c2, c3, 0.f);
             }
+            if constexpr (kNext) {
+                // the next layer's threshold pair per column; columns past N code to 0
+                float2* sT = reinterpret_cast<float2*>(smem + p.off_t);
+                for (int n = etid; n < p.Np; n += kEpiThreads) {
+                    float2 t = make_float2(-INFINITY, INFINITY);
+                    if (f.out_packed != nullptr && n < a.N)
+                        t = make_float2(f.next_lo[f.n_next == 1 ? 0 : n], f.next_hi[f.n_next == 1 ? 0 : n]);
+                    sT[n] = t;
+                }
+            }
         }
         asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible
         tc::pdl_wait();                             // out may still be read by the previous kernel
@@ -578,7 +696,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         // the epilogue then fetches them with tcgen05.ld, which does not compete with the tensor core,
         // the converters and TMA for shared-memory bandwidth as a broadcast shared load per output did.
         const uint32_t cq = tmem + ((uint32_t)(q * 32) << 16) + p.cbase;
-        if (p.const_tmem) {
+        if (p.const_tmem && !kNext) {
             for (int blk = blk_begin; blk < blk_end; ++blk) {
                 uint32_t k1[16], k2[16], k3[16];
                 #pragma unroll
@@ -600,6 +718,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             role_wait(warp == kEpiWarp0, &acc_full[buf], (it >> 1) & 1, a.status, dead, kEpiBarrier, kEpiThreads);
             const bool alive = !*dead;
             tc::tc_fence_after_sync();
+            if constexpr (kNext) {
+                next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, buf, g, nrows,
+                                   alive, q, lane, half);
+            } else
             for (int tm = 0; tm < ntm; ++tm) {
                 const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);     // pixel within the tile
                 const uint32_t row = fdiv(pl, p.div_pw);
@@ -751,12 +873,23 @@ bool conv_i8_supported(const ConvArgs& c)
     return make_plan(c, p, 148);
 }
 
-cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s)
+bool conv_i8_next_supported(const ConvArgs& c)
 {
     ConvI8Plan p;
-    if (!make_plan(c, p, sm_count())) return cudaErrorInvalidConfiguration;
+    return make_plan(c, p, 148, true);
+}
+
+static cudaError_t launch_conv_i8_any_mode(const ConvArgs& c, const NextLayerArgs* f, cudaStream_t s)
+{
+    ConvI8Plan p;
+    if (!make_plan(c, p, sm_count(), f != nullptr)) return cudaErrorInvalidConfiguration;
     CUtensorMap tmap;
     memset(&tmap, 0, sizeof(tmap));
+    if (f != nullptr && f->x_packed != nullptr) {
+        // packed pixel rows are read with plain loads by the converters: no staging ring
+        p.use_tma = 0;
+        p.smem_bytes = p.off_stage;
+    }
     if (p.use_tma) {
         EncodeTiledFn enc = encode_tiled_fn();
         const cuuint64_t dims[4] = {(cuuint64_t)c.W, (cuuint64_t)c.H, (cuuint64_t)c.C, (cuuint64_t)c.B};
@@ -773,10 +906,25 @@ cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s)
             p.smem_bytes = p.off_stage;
         }
     }
-    cudaError_t e = cudaFuncSetAttribute(conv_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (f != nullptr) {
+        cudaError_t e = cudaFuncSetAttribute(conv_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)p.smem_bytes);
+        if (e != cudaSuccess) return e;
+        return launch_pdl(conv_i8_kernel<true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p, tmap, *f);
+    }
+    cudaError_t e = cudaFuncSetAttribute(conv_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
-    return launch_pdl(conv_i8_kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p, tmap);
+    return launch_pdl(conv_i8_kernel<false>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p, tmap,
+                      NextLayerArgs{});
+}
+
+cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s) { return launch_conv_i8_any_mode(c, nullptr, s); }
+
+// The same kernel with the hand-over to the next layer (and, optionally, packed input).
+cudaError_t launch_conv_i8_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s)
+{
+    return launch_conv_i8_any_mode(c, &f, s);
 }
 
 }  // namespace rtn

@@ -66,5 +66,127 @@ __device__ __forceinline__ uint4 codes16(const float (&v)[16], const float* lo, 
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// Epilogue constant c3 of output channel n at a border pixel under value-zero padding: S_w and K
+// run over the taps inside the image only.  Kept out of line: borders are rare, the code is long.  The
+// layer's geometry comes by value: a reference to the kernel's parameter struct would make the compiler
+// keep a copy of it in local memory.
+struct BorderGeom {
+    const int32_t* w_sum;
+    const float* w_scale;
+    const float* w_offset;
+    int n_wparam, N, C, H, W, kw, stride, pad, T;
+    float a_offset;
+};
+__device__ __forceinline__ BorderGeom border_geom(const ConvArgs& a, int T)
+{
+    BorderGeom g;
+    g.w_sum = a.w_sum; g.w_scale = a.ep.w_scale; g.w_offset = a.ep.w_offset; g.n_wparam = (int)a.ep.n_wparam;
+    g.N = a.N; g.C = a.C; g.H = a.H; g.W = a.W; g.kw = a.kw; g.stride = a.stride; g.pad = a.pad; g.T = T;
+    g.a_offset = a.ep.a_offset_val;
+    return g;
+}
+__device__ __noinline__ inline float border_c3_by_value(BorderGeom g, int ho, int wo, int n_inside, int n)
+{
+    int s_w = 0;
+    for (int t = 0; t < g.T; ++t) {
+        const int h = ho * g.stride - g.pad + t / g.kw, v = wo * g.stride - g.pad + t % g.kw;
+        if (h >= 0 && h < g.H && v >= 0 && v < g.W) s_w += g.w_sum[(1 + t) * g.N + n];
+    }
+    const double ws = g.w_scale[g.n_wparam == 1 ? 0 : n];
+    const double wo_ = g.w_offset[g.n_wparam == 1 ? 0 : n];
+    return (float)((double)g.a_offset * (ws * (double)s_w + (double)g.C * n_inside * wo_));
+}
+__device__ __forceinline__ float border_c3(const ConvArgs& a, int T, int ho, int wo, int n_inside, int n)
+{
+    return border_c3_by_value(border_geom(a, T), ho, wo, n_inside, n);
+}
+// Element j (runtime index) of a register array, without sending the array to local memory.
+__device__ __forceinline__ uint32_t pick16(const uint32_t (&v)[16], int j)
+{
+    uint32_t r = v[0];
+    #pragma unroll
+    for (int k = 1; k < 16; ++k) r = (j == k) ? v[k] : r;
+    return r;
+}
+__device__ __forceinline__ void put16(float (&y)[16], int j, float val)
+{
+    #pragma unroll
+    for (int k = 0; k < 16; ++k) y[k] = (j == k) ? val : y[k];
+}
+
+// The hand-over epilogue (NextLayerArgs) for one pixel and one block of 16 output channels n0..n0+15:
+//   y = phi(c1*S_xw + c2*S_x + c3) + skip;  out <- y;  nzb, sgb <- Eq. 3 codes of y (16 bits per plane,
+//   computed when want_codes; the caller assembles them into words of the packed pixel row).
+// v: the block's accumulators; sC: {c1, c2, c3, 0} and sT: {t_lo, t_hi} of the next layer, both for
+// column n0 (columns past N hold zeros and (-inf, +inf): they code to 0).  o0: offset of (b, n0, ho, wo)
+// in the NCHW tensors.  Straight-line over the 16 columns: every load of a step is issued before its
+// first use (the skip values of 16 channels are 16 independent trips to memory).
+__device__ __forceinline__ void next_layer_block16(const ConvArgs& a, const NextLayerArgs& f, const uint32_t (&v)[16],
+                                                   const float4* sC, const float2* sT, float fsx, bool border,
+                                                   int T, int ho, int wo, int n_inside, int n0, int64_t o0,
+                                                   int64_t ostride, bool want_codes, uint32_t& nzb, uint32_t& sgb)
+{
+    const bool full = n0 + 16 <= a.N;
+    float y[16];
+    #pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const float4 c = sC[j];
+        y[j] = fmaf(c.x, (float)(int)v[j], fmaf(c.y, fsx, c.z));
+    }
+    if (border) {
+        // value-zero padding at an image border: S_w and K over inside taps only
+        #pragma unroll 1
+        for (int j = 0; j < 16; ++j) {
+            const int n = n0 + j;
+            if (n >= a.N) break;
+            const float4 c = sC[j];
+            const float c3 = border_c3(a, T, ho, wo, n_inside, n);
+            put16(y, j, fmaf(c.x, (float)(int)pick16(v, j), fmaf(c.y, fsx, c3)));
+        }
+    }
+    if (f.relu) {
+        #pragma unroll
+        for (int j = 0; j < 16; ++j) y[j] = y[j] > 0.f ? y[j] : 0.f;
+    }
+    if (f.skip != nullptr) {
+        float sk[16];
+        #pragma unroll
+        for (int j = 0; j < 16; ++j)
+            sk[j] = (full || n0 + j < a.N) ? __ldg(f.skip + o0 + (int64_t)j * ostride) : 0.f;
+        #pragma unroll
+        for (int j = 0; j < 16; ++j) y[j] += sk[j];
+    }
+    if (a.out != nullptr) {
+        #pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (full || n0 + j < a.N) a.out[o0 + (int64_t)j * ostride] = y[j];
+    }
+    if (a.dbg_acc != nullptr) {
+        #pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (full || n0 + j < a.N) a.dbg_acc[o0 + (int64_t)j * ostride] = (int)v[j];
+    }
+    nzb = 0; sgb = 0;                          // one bit per column and plane
+    if (want_codes) {
+        #pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float2 t = sT[j];
+            const bool pos = y[j] > t.y, neg = !pos && y[j] < t.x;
+            nzb |= (uint32_t)(pos || neg) << j;
+            sgb |= (uint32_t)pos << j;
+        }
+    }
+}
+
+// Zero codes for the columns from n_begin (a multiple of 16) to the end of a packed pixel row.
+__device__ __forceinline__ void zero_fill_packed_row(uint8_t* out_row, int n_begin, int packed_cols)
+{
+    for (int n0 = n_begin; n0 < packed_cols; n0 += 16) {
+        uint8_t* dst = out_row + (n0 >> 7) * kBlockBytes + ((n0 & 127) >> 3);
+        *reinterpret_cast<uint16_t*>(dst) = 0;
+        *reinterpret_cast<uint16_t*>(dst + 16) = 0;
+    }
+}
+
 }  // namespace conv_detail
 }  // namespace rtn

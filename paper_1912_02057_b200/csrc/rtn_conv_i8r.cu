@@ -305,33 +305,6 @@ __device__ __forceinline__ void role_wait_r(bool leader, uint64_t* bar, uint32_t
 // ------------------------------------------------------------------------------------------------
 // Kernel 2: the contraction and the epilogue.
 // ------------------------------------------------------------------------------------------------
-// Epilogue constant c3 of output channel n at a border pixel under value-zero padding: S_w and K
-// run over the taps inside the image only.  Kept out of line: borders are rare, the code is long.
-__device__ __noinline__ float border_c3(const ConvArgs& a, int T, int ho, int wo, int n_inside, int n)
-{
-    int s_w = 0;
-    for (int t = 0; t < T; ++t) {
-        const int h = ho * a.stride - a.pad + t / a.kw, v = wo * a.stride - a.pad + t % a.kw;
-        if (h >= 0 && h < a.H && v >= 0 && v < a.W) s_w += a.w_sum[(1 + t) * a.N + n];
-    }
-    const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
-    const double wo_ = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
-    return (float)((double)a.ep.a_offset_val * (ws * (double)s_w + (double)a.C * n_inside * wo_));
-}
-// Element j (runtime index) of a register array, without sending the array to local memory.
-__device__ __forceinline__ uint32_t pick16(const uint32_t (&v)[16], int j)
-{
-    uint32_t r = v[0];
-    #pragma unroll
-    for (int k = 1; k < 16; ++k) r = (j == k) ? v[k] : r;
-    return r;
-}
-__device__ __forceinline__ void put16(float (&y)[16], int j, float val)
-{
-    #pragma unroll
-    for (int k = 0; k < 16; ++k) y[k] = (j == k) ? val : y[k];
-}
-
 // kFused: the epilogue also applies phi, adds the skip connection, and hands the result to the next
 // layer as fp32 and / or as packed Eq. 3 codes against that layer's thresholds (NextLayerArgs).
 template <bool kFused>
@@ -567,12 +540,7 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
             if constexpr (kFused) {
                 if (ok && f.out_packed != nullptr) {
                     out_row = f.out_packed + (((int64_t)b * a.Ho + ho) * a.Wo + wo) * (int64_t)(packed_cols / 4);
-                    if (fq == p.S - 1 && half == 0)
-                        for (int n0 = p.S * p.Nq; n0 < packed_cols; n0 += 16) {
-                            uint8_t* dst = out_row + (n0 >> 7) * kBlockBytes + ((n0 & 127) >> 3);
-                            *reinterpret_cast<uint16_t*>(dst) = 0;
-                            *reinterpret_cast<uint16_t*>(dst + 16) = 0;
-                        }
+                    if (fq == p.S - 1 && half == 0) zero_fill_packed_row(out_row, p.S * p.Nq, packed_cols);
                 }
             }
             for (int blk = blk_begin; blk < blk_end; ++blk) {
@@ -583,62 +551,11 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
                 const int r0 = blk * 16;                   // column of the accumulator = row of the filter group
                 const int n0 = n_base + r0;
                 if constexpr (kFused) {
-                    // straight-line over the block's 16 columns: every load of a step is issued before
-                    // its first use (the skip values of 16 channels are 16 independent trips to memory)
-                    const float2* sT = reinterpret_cast<const float2*>(smem + p.off_t);
-                    const bool full = n0 + 16 <= a.N;
-                    const int64_t o0 = obase + (int64_t)n0 * ostride;
-                    float y[16];
-                    #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float4 c = sC[r0 + j];
-                        y[j] = fmaf(c.x, (float)(int)v[j], fmaf(c.y, fsx, c.z));
-                    }
-                    if (border) {
-                        // value-zero padding at an image border: S_w and K over inside taps only
-                        #pragma unroll 1
-                        for (int j = 0; j < 16; ++j) {
-                            const int n = n0 + j;
-                            if (n >= a.N) break;
-                            const float4 c = sC[r0 + j];
-                            const float c3 = border_c3(a, p.T, ho, wo, n_inside, n);
-                            const float yb = fmaf(c.x, (float)(int)pick16(v, j), fmaf(c.y, fsx, c3));
-                            put16(y, j, yb);
-                        }
-                    }
-                    if (f.relu) {
-                        #pragma unroll
-                        for (int j = 0; j < 16; ++j) y[j] = y[j] > 0.f ? y[j] : 0.f;
-                    }
-                    if (f.skip != nullptr) {
-                        float sk[16];
-                        #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            sk[j] = (full || n0 + j < a.N) ? __ldg(f.skip + o0 + (int64_t)j * ostride) : 0.f;
-                        #pragma unroll
-                        for (int j = 0; j < 16; ++j) y[j] += sk[j];
-                    }
-                    if (a.out != nullptr) {
-                        #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (full || n0 + j < a.N) a.out[o0 + (int64_t)j * ostride] = y[j];
-                    }
-                    if (a.dbg_acc != nullptr) {
-                        #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (full || n0 + j < a.N) a.dbg_acc[o0 + (int64_t)j * ostride] = (int)v[j];
-                    }
-                    if (f.out_packed != nullptr && n0 < packed_cols) {
-                        // the 16 codes of this block, one bit each per plane; columns past N have the
-                        // thresholds (-inf, +inf) and code to 0
-                        uint32_t nzb = 0, sgb = 0;
-                        #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float2 t = sT[r0 + j];
-                            const bool pos = y[j] > t.y, neg = !pos && y[j] < t.x;
-                            nzb |= (uint32_t)(pos || neg) << j;
-                            sgb |= (uint32_t)pos << j;
-                        }
+                    uint32_t nzb, sgb;
+                    next_layer_block16(a, f, v, sC + r0, reinterpret_cast<const float2*>(smem + p.off_t) + r0, fsx,
+                                       border, p.T, ho, wo, n_inside, n0, obase + (int64_t)n0 * ostride, ostride,
+                                       out_row != nullptr && n0 < packed_cols, nzb, sgb);
+                    if (out_row != nullptr && n0 < packed_cols) {
                         uint8_t* dst = out_row + (n0 >> 7) * kBlockBytes + ((n0 & 127) >> 3);
                         *reinterpret_cast<uint16_t*>(dst) = (uint16_t)nzb;
                         *reinterpret_cast<uint16_t*>(dst + 16) = (uint16_t)sgb;

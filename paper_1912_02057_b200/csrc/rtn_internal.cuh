@@ -95,6 +95,8 @@ cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s);     // scratch f
 cudaError_t launch_conv_i8r_static(const ConvArgs& c, cudaStream_t s);      // scratch in a static device array
 size_t conv_i8r_static_scratch_bytes();
 // Two-kernel path with the fused hand-over to the next layer (and, optionally, packed input).
+bool conv_i8_next_supported(const ConvArgs& c);    // one-kernel variant (filters resident)
+cudaError_t launch_conv_i8_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s);
 bool conv_i8r_next_supported(const ConvArgs& c);
 cudaError_t launch_conv_i8r_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s);
 inline bool conv_i8_any_supported(const ConvArgs& c)
