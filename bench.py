@@ -44,9 +44,22 @@ WORKLOADS = {
 # every ternary conv layer of ResNet-18 at batch 128 (the layer table of the paper's appendix)
 for _l in inputs.resnet18_ternary_layers():
     WORKLOADS[f"r18_{_l[0]}_b128"] = (lambda n=_l[0]: inputs.resnet18_layer(n, batch=128))
+# the 19 ternary layers chained (packed hand-over between layers), batch 64 of 224x224 images (56x56 after the stem)
+WORKLOADS["r18_body_b64"] = lambda: BodyCase(64)
 DEFAULT_WORKLOAD = "cfg2_conv3x3_c64_56x56_b32"
 # --io packed: thresholds of the next layer's ternarizer (per layer), applied to phi(conv output)
 NEXT_THRESHOLDS = (0.5, 2.0)
+
+
+class BodyCase:
+    """The ternary body of ResNet-18 as one workload: random-init layers, thresholds by the recipe of
+    inputs.resnet18_body_blocks, input = max(0, N(0,1)) standing in for the stem's max-pooled output."""
+
+    def __init__(self, batch):
+        self.B = batch
+        self.layers = inputs.resnet18_body(seed=4)
+        self.blocks = inputs.resnet18_body_blocks(self.layers, sigma_in=1.0)
+        self.x = inputs.relu_normal(inputs.rng(44), (batch, 64, 56, 56))
 
 
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -267,6 +280,185 @@ def max_over_ranks(values, world, device):
 def whole_job_tops(ops_per_replica, world, ms):
     """Replicas only: every rank does the same work, so the job's rate is world * ops / slowest time."""
     return world * ops_per_replica / (ms * 1e-3) / 1e12
+
+
+def oracle_body_sample(case, budget_s=12.0):
+    """The CPU oracle on the body's first residual block (two 3x3 layers with the hand-over between
+    them) for as many images as fit the time budget.  Returns (ops per second, seconds, description)."""
+    import oracle
+    c1, c2 = case.blocks[0]["conv1"], case.blocks[0]["conv2"]
+    nxt = case.blocks[1]["conv1"]
+
+    def run(nb):
+        s = case.x[:nb]
+        t0 = time.perf_counter()
+        p = oracle.ternarize(s, c1.t_lo, c1.t_hi)
+        _, pre1, _ = oracle.conv2d(p, c1.w_codes, 1, 1, oracle.PAD_CODE_ZERO, c1.a_scale, c1.a_offset, c1.w_scale, c1.w_offset)
+        _, q, _ = oracle.next_layer(pre1, True, None, c2.t_lo, c2.t_hi)
+        _, pre2, _ = oracle.conv2d(q, c2.w_codes, 1, 1, oracle.PAD_CODE_ZERO, c2.a_scale, c2.a_offset, c2.w_scale, c2.w_offset)
+        oracle.next_layer(pre2, True, s, nxt.t_lo, nxt.t_hi)
+        dt = time.perf_counter() - t0
+        return 2 * 2.0 * nb * 56 * 56 * 64 * 64 * 9, dt
+    ops, dt = run(1)
+    nb = int(max(1, min(case.B, budget_s / max(dt, 1e-6))))
+    if nb > 1:
+        ops, dt = run(nb)
+    return ops / dt, dt, f"first residual block (layer1.0.conv1, conv2 and their hand-over) on {nb} of {case.B} images"
+
+
+def run_body(args, case, name):
+    """Whole-chain workload: a step = the 19 ternary layers of ResNet-18 on one batch."""
+    import torch
+    import torch.distributed as dist
+    import paper_1912_02057_b200 as rtn
+    from paper_1912_02057_b200 import chain
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    n_sets = 2          # two complete sets of activations (input, every intermediate), used in turn
+    bodies = [chain.Body(case.blocks, case.B) for _ in range(n_sets)]
+    xs = [torch.from_numpy(case.x).cuda() for _ in range(n_sets)]
+    host_in = torch.from_numpy(case.x).pin_memory()
+    outs = [None] * n_sets
+
+    def step(i):
+        j = i % n_sets
+        outs[j], _ = bodies[j].forward(xs[j])
+        return outs[j]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    host_out = torch.empty(outs[0].shape, dtype=torch.float32).pin_memory()
+    steps = args.steps
+    chunk = min(steps, 20)
+    n_full, tail = divmod(steps, chunk)
+
+    class Eager:
+        def __init__(self, n):
+            self.n = n
+
+        def replay(self):
+            for i in range(self.n):
+                step(i)
+
+    def capture(n):
+        if args.eager:
+            return Eager(n)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(n):
+                step(i)
+        return g
+    graph = capture(chunk)
+    graph_tail = capture(tail) if tail else None
+    graph.replay()
+    if graph_tail is not None:
+        graph_tail.replay()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(n_full):
+        graph.replay()
+    if graph_tail is not None:
+        graph_tail.replay()
+    t1.record()
+    barrier()
+    total_ms = t0.elapsed_time(t1)
+    if rank == 0 and not args.eager:
+        w0 = time.perf_counter()
+        while time.perf_counter() - w0 < 1.0:
+            graph.replay()
+            torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    if clocks is not None:
+        clocks["window"] = "timed region plus about 1 s of the same launches, untimed"
+    barrier()
+    if rtn.rtn_last_device_status() != 0:
+        raise RuntimeError("device status after the timed region")
+    e2e_steps = max(3, min(steps, 10))
+    for i in range(2):
+        xs[0].copy_(host_in, non_blocking=True)
+        host_out.copy_(step(0), non_blocking=True)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        j = i % n_sets
+        xs[j].copy_(host_in, non_blocking=True)
+        host_out.copy_(step(j), non_blocking=True)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, "cuda")
+    ms_per_step = total_ms / steps
+    ops = bodies[0].ops()
+    launches = bodies[0].kernel_launches()
+    if rank == 0:
+        line = {
+            "metric": "effective ternary TOPS (2MNK/s)", "value": whole_job_tops(ops, world, ms_per_step),
+            "unit": "TOPS", "n_gpus": world, "steps": steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32 accumulate (int8 / 1-bit-plane operands), fp32 epilogue", "data": "synthetic",
+            "config": {"workload": name, "io": "packed rows between layers, fp32 residual stream",
+                       "images_per_s": world * case.B / (ms_per_step * 1e-3),
+                       "layers": 19, "launches_per_step": launches,
+                       "l2": f"{n_sets} complete sets of activations used in turn; a layer's output may still be in L2 "
+                             "when its consumer reads it (part of the chain, not of the timing method)",
+                       "weights": "packed before the timed region (offline step)",
+                       "launch": "eager" if args.eager else f"CUDA graph, {chunk} steps per replay",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "clocks": clocks,
+            "e2e": {"value": whole_job_tops(ops, world, e2e_ms), "unit": "TOPS", "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": int(host_in.numel() * 4), "d2h_bytes_per_step": int(host_out.numel() * 4)},
+            "gpu_launches": launches * steps,
+            "roofline": roofline_of(name, bodies[0].algorithmic_bytes(), ops, ms_per_step),
+        }
+        line["roofline"]["note"] = "whole chain (19 layers) against the binding bound of its summed bytes and operations"
+        if not args.no_cpu_baseline and world == 1:
+            import oracle
+            rate, dt, sample = oracle_body_sample(case, 12.0)
+            line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TOPS", "cores": oracle.threads(),
+                                    "kind": "oracle", "sample": sample, "seconds": dt}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_body_reference(args, case, name):
+    import oracle
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    per_step_budget = max(0.2, min(12.0, 60.0 / max(1, args.steps + args.warmup)))
+    sample = ""
+    for _ in range(args.warmup):
+        _, _, sample = oracle_body_sample(case, per_step_budget)
+    rates, secs = [], []
+    for _ in range(args.steps):
+        r, dt, sample = oracle_body_sample(case, per_step_budget)
+        rates.append(r)
+        secs.append(dt)
+    value = float(np.mean(rates)) / 1e12
+    print(json.dumps({
+        "impl": "reference", "metric": "effective ternary TOPS (2MNK/s)", "value": value, "unit": "TOPS",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(secs)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": name, "note": "CPU oracle on a bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": "TOPS", "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
 
 
 def run_ours(args, case, name):
@@ -499,6 +691,11 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     case = WORKLOADS[args.workload]()
+    if isinstance(case, BodyCase):
+        if args.steps == 2000:          # the default suits 20 us kernels; a chain step is a few milliseconds
+            args.steps = 100
+        (run_body_reference if args.impl == "reference" else run_body)(args, case, args.workload)
+        return
     if args.impl == "reference":
         run_reference(args, case, args.workload)
     else:

@@ -213,6 +213,12 @@ rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, 
 int64_t rtn_conv_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
                                  int64_t kh, int64_t kw, int64_t stride, int64_t pad);
 
+/* Kernel launches of one rtn_ternary_conv2d_fused / rtn_ternary_conv2d_packed call for a shape: 1 (one-kernel
+ * variant with the filters resident in shared memory), 2 (int8 codes in a scratch buffer first), or 0 if
+ * the entry points do not take the shape (they would return RTN_ERR_UNSUPPORTED). */
+int64_t rtn_conv_next_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
+                                      int64_t kh, int64_t kw, int64_t stride, int64_t pad);
+
 /* Synchronises `stream`, then reads and clears the device status word of the current device.
  * RTN_OK, or RTN_ERR_DEVICE_TIMEOUT if a kernel's bounded wait (on an mbarrier of the
  * tensor-core pipeline) ran out since the last call; that kernel's output is then invalid. */

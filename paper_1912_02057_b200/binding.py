@@ -83,6 +83,8 @@ def lib():
         L.rtn_choose_conv_variant.argtypes = [_i64] * 9
         L.rtn_conv_kernel_launches.restype = _i64
         L.rtn_conv_kernel_launches.argtypes = [_i64] * 9
+        L.rtn_conv_next_kernel_launches.restype = _i64
+        L.rtn_conv_next_kernel_launches.argtypes = [_i64] * 9
         L.rtn_last_device_status.restype = _int
         L.rtn_last_device_status.argtypes = [_vp]
         L.rtn_status_string.restype = C.c_char_p
@@ -257,6 +259,10 @@ def rtn_choose_conv_variant(B, Cin, H, W, N, kh, kw, stride, pad):
 
 def rtn_conv_kernel_launches(B, Cin, H, W, N, kh, kw, stride, pad):
     return int(lib().rtn_conv_kernel_launches(B, Cin, H, W, N, kh, kw, stride, pad))
+
+
+def rtn_conv_next_kernel_launches(B, Cin, H, W, N, kh, kw, stride, pad):
+    return int(lib().rtn_conv_next_kernel_launches(B, Cin, H, W, N, kh, kw, stride, pad))
 
 
 def rtn_last_device_status(stream=None):

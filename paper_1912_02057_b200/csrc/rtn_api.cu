@@ -228,6 +228,17 @@ int64_t rtn_conv_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W, int
     return rtn::conv_i8r_supported(c) ? 2 : 1;
 }
 
+int64_t rtn_conv_next_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
+                                      int64_t kh, int64_t kw, int64_t stride, int64_t pad)
+{
+    rtn::ConvArgs c{};
+    c.B = (int)B; c.C = (int)C; c.H = (int)H; c.W = (int)W; c.N = (int)N; c.kh = (int)kh; c.kw = (int)kw;
+    c.stride = (int)stride; c.pad = (int)pad;
+    c.Ho = (int)rtn_conv_out_dim(H, kh, stride, pad); c.Wo = (int)rtn_conv_out_dim(W, kw, stride, pad);
+    if (rtn::conv_i8_next_supported(c)) return 1;
+    return rtn::conv_i8r_next_supported(c) ? 2 : 0;
+}
+
 rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
                               const float* t_lo, const float* t_hi, int64_t n_thr,
                               const void* w_packed, const int32_t* w_sum,

@@ -199,3 +199,88 @@ def resnet18_layer(name, batch=128, p_zero=0.5):
             return conv_case(f"r18_{name}_b{batch}", batch, cin, hin, hin, cout, k, stride, pad,
                              seed=400 + i, p_zero=p_zero)
     raise KeyError(name)
+
+
+# ------------------------------------------------------------------ the ternary body of ResNet-18 as a chain
+@dataclass
+class BodyLayer:
+    """One ternary conv layer of the chain with everything it needs (random init, seeded)."""
+    name: str
+    cin: int
+    cout: int
+    k: int
+    stride: int
+    pad: int
+    hin: int               # input height = width
+    w_codes: np.ndarray    # int8 [cout, cin, k, k]
+    a_scale: float         # gamma, beta of the layer's activation (Eq. 4)
+    a_offset: float
+    w_scale: np.ndarray    # alpha per filter (Eq. 5) and the weight offset the library adds, fp32 [cout]
+    w_offset: np.ndarray
+    t_lo: np.ndarray       # thresholds of the ternarizer in FRONT of this layer (its BN folded, Eq. 3), fp32 [1]
+    t_hi: np.ndarray
+    sigma_out: float       # estimated standard deviation of the layer's conv output (sets the thresholds downstream)
+
+
+def resnet18_body(seed=4, p_zero=0.5, dyadic=False, hin=56):
+    """The 19 ternary conv layers of ResNet-18 (paper's appendix table) with random-init codes and
+    parameters, plus thresholds that keep all three codes in use along the chain.
+
+    Threshold rule: the ternarizer in front of a layer sees y = phi(conv) [+ skip] with standard
+    deviation about sigma (conv: c1 * sqrt(K * q_x * q_w) with q the non-zero fractions, estimated
+    as 0.5; the residual stream adds the variances of its branches); t_lo = 0.3 sigma, t_hi =
+    1.0 sigma, the pair config 1 uses for a unit-scale post-ReLU input.  dyadic=True rounds every
+    parameter to a small multiple of a power of two, so that every product and sum of the
+    epilogues is exact in fp32 and in double (both sides of a parity test then take identical
+    threshold decisions along the whole chain).
+    """
+    g = rng(seed)
+    layers = []
+    size = {1: hin}                                    # input size of each stage's stride-1 layers
+    for st in (2, 3, 4):
+        size[st] = (size[st - 1] + 2 - 3) // 2 + 1     # after the stage's 3x3 stride-2 conv (1x1 stride 2 gives the same)
+    for (name, cin, cout, k, stride, pad, _) in resnet18_ternary_layers():
+        st = int(name[5])
+        h = size[st - 1] if stride == 2 else size[st]
+        w = weight_codes(g, (cout, cin, k, k), p_zero)
+        if dyadic:
+            w_s = (g.integers(2, 7, cout) / 4.0).astype(np.float32)
+            w_o = (g.integers(-2, 3, cout) / 16.0).astype(np.float32)
+            a_s, a_o = 0.75, 0.125
+        else:
+            w_s, w_o = uniform(g, 0.5, 1.5, (cout,)), uniform(g, -0.1, 0.1, (cout,))
+            a_s, a_o = float(uniform(g, 0.5, 1.5)), float(uniform(g, -0.1, 0.1))
+        K = cin * k * k
+        sigma = float(a_s * np.mean(w_s) * np.sqrt(K * 0.5 * (1.0 - p_zero)))
+        layers.append(BodyLayer(name, cin, cout, k, stride, pad, h, w, a_s, a_o, w_s, w_o,
+                                np.zeros(1, np.float32), np.ones(1, np.float32), sigma))
+    return layers
+
+
+def set_thresholds(layer, sigma, dyadic=False):
+    lo, hi = 0.3 * sigma, 1.0 * sigma
+    if dyadic:
+        lo, hi = np.round(lo * 4) / 4, np.round(hi * 4) / 4
+    layer.t_lo = np.array([lo], np.float32)
+    layer.t_hi = np.array([hi], np.float32)
+
+
+def resnet18_body_blocks(layers, sigma_in=1.0, dyadic=False):
+    """Groups the 19 layers into the 8 residual blocks and sets every layer's input thresholds.
+    Returns a list of dicts {conv1, conv2, down (or None)}; sigma_in is the scale of the body's fp32
+    input (the stem's max-pooled output; max(0, N(0,1)) in the synthetic workload)."""
+    by_name = {l.name: l for l in layers}
+    blocks = []
+    sigma_stream = sigma_in
+    for s in (1, 2, 3, 4):
+        for b in (0, 1):
+            c1, c2 = by_name[f"layer{s}.{b}.conv1"], by_name[f"layer{s}.{b}.conv2"]
+            down = by_name.get(f"layer{s}.{b}.downsample.0")
+            set_thresholds(c1, sigma_stream, dyadic)            # ternarizer of the block's input
+            if down is not None:
+                set_thresholds(down, sigma_stream, dyadic)
+            set_thresholds(c2, 0.6 * c1.sigma_out, dyadic)      # input = relu(conv1): about 0.6 sigma
+            skip_sigma = 0.6 * down.sigma_out if down is not None else sigma_stream
+            sigma_stream = float(np.sqrt((0.6 * c2.sigma_out) ** 2 + skip_sigma ** 2))
+            blocks.append({"conv1": c1, "conv2": c2, "down": down})
+    return blocks
