@@ -26,6 +26,7 @@ def _L():
         _lib.orc_conv_out_dim.restype = C.c_int64
         _lib.orc_conv_out_dim.argtypes = [C.c_int64] * 4
         _lib.orc_direct_dot.restype = C.c_double
+        _lib.orc_dot_quaternary_bits.restype = C.c_int64
     return _lib
 
 
@@ -287,6 +288,48 @@ def unpack_nhwc(packed, B, Cc, H, W):
     """Inverse of pack_nhwc: packed pixel rows -> codes [B,C,H,W]."""
     rows = unpack_rows(np.asarray(packed, np.uint8).reshape(B * H * W, packed_row_bytes(Cc)), Cc)
     return np.ascontiguousarray(rows.reshape(B, H, W, Cc).transpose(0, 3, 1, 2))
+
+
+# ----------------------------------------------------------------------------- 2-bit comparison workload
+def quaternary_decode(b1, b2):
+    """Table 1, last column: bits (b1, b2) -> 2*b1 + b2 in {0,1,2,3}."""
+    b1, b2 = _arr(b1, np.uint8), _arr(b2, np.uint8)
+    v = np.empty(b1.shape, np.uint8)
+    _L().orc_quaternary_decode(_p(b1), _p(b2), _i64(b1.size), _p(v))
+    return v
+
+
+def quaternary_encode(values):
+    values = _arr(values, np.uint8)
+    b1, b2 = np.empty(values.shape, np.uint8), np.empty(values.shape, np.uint8)
+    _L().orc_quaternary_encode(_p(values), _i64(values.size), _p(b1), _p(b2))
+    return b1, b2
+
+
+def quaternary_gemm(x, w):
+    """values x [M,K], w [N,K] in {0..3} -> exact int64 dot products [M,N] (the definition)."""
+    x, w = _arr(x, np.uint8), _arr(w, np.uint8)
+    M, K = x.shape
+    N, K2 = w.shape
+    assert K == K2
+    S = np.empty((M, N), np.int64)
+    _L().orc_quaternary_gemm(_p(x), _p(w), _i64(M), _i64(N), _i64(K), _p(S))
+    return S
+
+
+def dot_quaternary_bits(x1, x2, w1, w2):
+    """DoReFa pattern: 4 bC(X1&W1) + 2 bC(X1&W2) + 2 bC(X2&W1) + bC(X2&W2) on one-bit-per-byte vectors."""
+    x1, x2, w1, w2 = (_arr(v, np.uint8) for v in (x1, x2, w1, w2))
+    return int(_L().orc_dot_quaternary_bits(_p(x1), _p(x2), _p(w1), _p(w2), _i64(x1.size)))
+
+
+def pack_quaternary_rows(values):
+    """values [rows, K] in {0..3} -> packed rows: plane 1 = first bit (weight 2), plane 2 = second bit."""
+    values = _arr(values, np.uint8)
+    rows, K = values.shape
+    out = np.empty((rows, packed_row_bytes(K)), np.uint8)
+    _L().orc_pack_quaternary_rows(_p(values), _i64(rows), _i64(K), _p(out))
+    return out
 
 
 # ----------------------------------------------------------------------------- tolerance

@@ -397,3 +397,69 @@ void orc_next_layer(const double *pre, const float *skip /* nullable */, int rel
             }
         }
 }
+
+/* ------------------------------------------------------------------------- */
+/* The paper's comparison workload: 2-bit quaternary weights and activations    */
+/* (Table 1, last column: bits (b1, b2) stand for the value 2*b1 + b2 in        */
+/* {0, 1, 2, 3}), dot product in the DoReFa-Net pattern the section "Efficient  */
+/* Computation Pattern" cites: AND between each bit plane of the two inputs,    */
+/* popcount, power-of-two shifts, four partial sums.                            */
+/* ------------------------------------------------------------------------- */
+void orc_quaternary_decode(const uint8_t *bit1, const uint8_t *bit2, int64_t n, uint8_t *values)
+{
+    for (int64_t i = 0; i < n; ++i) values[i] = (uint8_t)(2 * (bit1[i] != 0) + (bit2[i] != 0));
+}
+
+void orc_quaternary_encode(const uint8_t *values, int64_t n, uint8_t *bit1, uint8_t *bit2)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        bit1[i] = (uint8_t)((values[i] >> 1) & 1);
+        bit2[i] = (uint8_t)(values[i] & 1);
+    }
+}
+
+/* The definition: plain sums of products of the values, int64. */
+void orc_quaternary_gemm(const uint8_t *x, const uint8_t *w, int64_t M, int64_t N, int64_t K,
+                         int64_t *S /* [M][N] */)
+{
+    #pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            int64_t s = 0;
+            for (int64_t k = 0; k < K; ++k) s += (int64_t)x[m * K + k] * (int64_t)w[n * K + k];
+            S[m * N + n] = s;
+        }
+}
+
+/* The bit formula (exists to be pinned against the plain sum):                 */
+/*   x.w = 4 bC(X1&W1) + 2 bC(X1&W2) + 2 bC(X2&W1) + bC(X2&W2)                  */
+int64_t orc_dot_quaternary_bits(const uint8_t *x1, const uint8_t *x2,
+                                const uint8_t *w1, const uint8_t *w2, int64_t n)
+{
+    int64_t c11 = 0, c12 = 0, c21 = 0, c22 = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        c11 += (x1[i] & w1[i]) & 1;
+        c12 += (x1[i] & w2[i]) & 1;
+        c21 += (x2[i] & w1[i]) & 1;
+        c22 += (x2[i] & w2[i]) & 1;
+    }
+    return (c11 << 2) + (c12 << 1) + (c21 << 1) + c22;
+}
+
+/* Packed rows of quaternary values: the library's block-plane format with      */
+/* plane 1 = first bit (weight 2) and plane 2 = second bit (weight 1).          */
+void orc_pack_quaternary_rows(const uint8_t *values, int64_t rows, int64_t K, uint8_t *out)
+{
+    const int64_t rb = orc_packed_row_bytes(K);
+    for (int64_t r = 0; r < rows; ++r) {
+        uint8_t *row = out + r * rb;
+        for (int64_t i = 0; i < rb; ++i) row[i] = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            const uint8_t v = values[r * K + k];
+            uint8_t *blk = row + (k / 128) * 32;
+            const int64_t i = k % 128;
+            if (v & 2) blk[i / 8] |= (uint8_t)(1u << (i % 8));
+            if (v & 1) blk[16 + i / 8] |= (uint8_t)(1u << (i % 8));
+        }
+    }
+}

@@ -454,3 +454,50 @@ def test_two_layer_chain_against_torch_fp64():
     c = torch.where(h > 2.0, 1.0, torch.where(h < 0.5, -1.0, 0.0)).to(torch.float64)
     ref = F.conv2d(0.5 * c - 0.125, deq_w(w2, ws2), padding=1).numpy()
     assert np.allclose(pre2, ref, rtol=1e-12, atol=1e-10)
+
+
+# ------------------------------------------------------------------ the 2-bit comparison workload
+def test_table1_quaternary_column_matches_paper_rows():
+    rows = read_golden("table1_quaternary.txt")
+    assert len(rows) == 4
+    for b1, b2, val in rows:
+        assert int(oracle.quaternary_decode([int(b1)], [int(b2)])[0]) == int(val)
+    v = np.arange(4, dtype=np.uint8)
+    b1, b2 = oracle.quaternary_encode(v)
+    assert b1.tolist() == [0, 0, 1, 1] and b2.tolist() == [0, 1, 0, 1]
+    assert oracle.quaternary_decode(b1, b2).tolist() == [0, 1, 2, 3]
+
+
+def test_quaternary_bit_formula_exhaustive_and_brute_force():
+    for x in range(4):
+        for w in range(4):
+            x1, x2 = oracle.quaternary_encode([x])
+            w1, w2 = oracle.quaternary_encode([w])
+            assert oracle.dot_quaternary_bits(x1, x2, w1, w2) == x * w
+    g = np.random.default_rng(61)
+    for n in (1, 31, 32, 33, 129, 300):
+        x, w = g.integers(0, 4, n).astype(np.uint8), g.integers(0, 4, n).astype(np.uint8)
+        want = sum(int(a) * int(b) for a, b in zip(x.tolist(), w.tolist()))
+        assert oracle.dot_quaternary_bits(*oracle.quaternary_encode(x), *oracle.quaternary_encode(w)) == want
+
+
+def test_quaternary_gemm_against_numpy_and_hand_cases():
+    g = np.random.default_rng(67)
+    x, w = g.integers(0, 4, (7, 45)).astype(np.uint8), g.integers(0, 4, (5, 45)).astype(np.uint8)
+    assert np.array_equal(oracle.quaternary_gemm(x, w), x.astype(np.int64) @ w.astype(np.int64).T)
+    assert oracle.quaternary_gemm(np.full((1, 10), 3, np.uint8), np.full((1, 10), 3, np.uint8))[0, 0] == 90
+    # a transposed operand changes the result
+    sq = g.integers(0, 4, (6, 6)).astype(np.uint8)
+    y = g.integers(0, 4, (6, 6)).astype(np.uint8)
+    assert not np.array_equal(oracle.quaternary_gemm(sq, y), oracle.quaternary_gemm(sq, y.T.copy()))
+
+
+def test_pack_quaternary_rows_planes():
+    v = np.zeros((1, 130), np.uint8)
+    v[0, 0], v[0, 9], v[0, 129] = 3, 2, 1
+    p = oracle.pack_quaternary_rows(v)
+    assert p.shape == (1, 64)
+    assert p[0, 0] == 1 and p[0, 16] == 1              # value 3 at position 0: both planes
+    assert p[0, 1] == 2 and p[0, 17] == 0              # value 2 at position 9: first-bit plane only
+    assert p[0, 32] == 0 and p[0, 48] == 2             # value 1 at position 129: second-bit plane of block 1
+    assert p.sum() == 1 + 1 + 2 + 2
