@@ -46,6 +46,8 @@ for _l in inputs.resnet18_ternary_layers():
     WORKLOADS[f"r18_{_l[0]}_b128"] = (lambda n=_l[0]: inputs.resnet18_layer(n, batch=128))
 # the 19 ternary layers chained (packed hand-over between layers), batch 64 of 224x224 images (56x56 after the stem)
 WORKLOADS["r18_body_b64"] = lambda: BodyCase(64)
+# the paper's comparison: 2-bit quaternary against ternary, both with the bit-plane (AND / popcount) pattern
+WORKLOADS["quaternary_vs_ternary_popc_gemm_2048"] = lambda: QuaternaryCase(2048)
 DEFAULT_WORKLOAD = "cfg2_conv3x3_c64_56x56_b32"
 # --io packed: thresholds of the next layer's ternarizer (per layer), applied to phi(conv output)
 NEXT_THRESHOLDS = (0.5, 2.0)
@@ -60,6 +62,19 @@ class BodyCase:
         self.layers = inputs.resnet18_body(seed=4)
         self.blocks = inputs.resnet18_body_blocks(self.layers, sigma_in=1.0)
         self.x = inputs.relu_normal(inputs.rng(44), (batch, 64, 56, 56))
+
+
+class QuaternaryCase:
+    """Square GEMM on 2-bit quaternary values (uniform over {0,1,2,3}) and, for the ratio the paper's
+    hardware section argues about, the same-size ternary GEMM on the bit-plane kernel."""
+
+    def __init__(self, n):
+        self.n = n
+        g = inputs.rng(6)
+        self.x = g.integers(0, 4, (n, n)).astype(np.uint8)
+        self.w = g.integers(0, 4, (n, n)).astype(np.uint8)
+        self.ternary = inputs.gemm_case(f"ternary_{n}", n, n, n, seed=6, p_zero=1.0 / 3.0, act="uniform3",
+                                        thresholds=(-0.5, 0.5))
 
 
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -461,6 +476,106 @@ def run_body_reference(args, case, name):
         "gpu_launches": 0}))
 
 
+POPC_LANES_PER_CLK_SM = 16      # popcount issue rate per SM and clock (quarter rate)
+SMS = 148
+
+
+def run_quaternary(args, case, name):
+    """rtn_quaternary_gemm against rtn_ternary_gemm's bit-plane variant at the same size."""
+    import torch
+    import paper_1912_02057_b200 as rtn
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1 and int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    n = case.n
+    n_sets = 8                      # 8 x (2 x 1 MiB packed + 16 MiB out) > L2
+    xq = [rtn.rtn_pack_quaternary(dev(case.x)) for _ in range(n_sets)]
+    wq = rtn.rtn_pack_quaternary(dev(case.w))
+    outs = [torch.empty((n, n), dtype=torch.int32, device="cuda") for _ in range(n_sets)]
+    t = case.ternary
+    w_packed, w_sum = rtn.rtn_pack_weights(dev(t.w_codes))
+    packs = [rtn.rtn_ternarize_pack_act(dev(t.a), dev(t.t_lo), dev(t.t_hi)) for _ in range(n_sets)]
+    a_s, a_o, w_s, w_o = dev(t.a_scale), dev(t.a_offset), dev(t.w_scale), dev(t.w_offset)
+    fouts = [torch.empty((n, n), dtype=torch.float32, device="cuda") for _ in range(n_sets)]
+    steps = min(args.steps, 200)
+
+    def q_step(i):
+        j = i % n_sets
+        return rtn.rtn_quaternary_gemm(xq[j], wq, n, n, n, out=outs[j])
+
+    def t_step(i):
+        j = i % n_sets
+        return rtn.rtn_ternary_gemm(packs[j][0], packs[j][1], w_packed, w_sum[0], n, n, n, a_s, a_o, w_s, w_o,
+                                    out=fouts[j], variant=rtn.VARIANT_POPC)
+
+    def timed(fn):
+        for i in range(max(args.warmup, 3)):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    t_ms = timed(t_step)
+    q_ms = timed(q_step)
+    clocks = sampler.stop()
+    host_in = torch.from_numpy(case.x).pin_memory()
+    dx = torch.empty((n, n), dtype=torch.uint8, device="cuda")
+    host_out = torch.empty((n, n), dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = 5
+    e0.record()
+    for i in range(e2e_steps):
+        dx.copy_(host_in, non_blocking=True)
+        host_out.copy_(rtn.rtn_quaternary_gemm(rtn.rtn_pack_quaternary(dx), wq, n, n, n, out=outs[0]), non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    ops = 2.0 * n * n * n
+    mhz = clocks.get("sm_mhz") or 1965.0
+    # four popcounts per 32 multiply-accumulates at 16 lanes per clock and SM
+    peak = 2.0 * 32 * POPC_LANES_PER_CLK_SM * SMS * mhz * 1e6 / 4 / 1e12
+    achieved = ops / (q_ms * 1e-3) / 1e12
+    line = {
+        "metric": "effective 2-bit TOPS (2MNK/s)", "value": achieved, "unit": "TOPS", "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": q_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int32 accumulate (1-bit-plane operands)", "data": "synthetic",
+        "config": {"workload": name, "ternary_popc_ms": t_ms, "ternary_popc_tops": ops / (t_ms * 1e-3) / 1e12,
+                   "quaternary_over_ternary_time": q_ms / t_ms,
+                   "note": "same tiling for both; per 32 values and output 4 popcounts (quaternary) against 2 (ternary, Eq. 9)",
+                   "l2": f"{n_sets} rotating operand/output sets > L2", "launch": "eager", "parallelism": "1 GPU"},
+        "clocks": clocks,
+        "e2e": {"value": ops / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(host_in.numel()), "d2h_bytes_per_step": int(host_out.numel() * 4)},
+        "gpu_launches": steps,
+        "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
+                     "traffic": None,
+                     "peak_source": f"derived: 16 popcount lanes per clock and SM x {SMS} SMs x {mhz:.0f} MHz (median sampled), "
+                                    "4 popcounts per 32 multiply-accumulates",
+                     "kernel_ms": q_ms},
+    }
+    if not args.no_cpu_baseline:
+        import oracle
+        rows = 16
+        t0 = time.perf_counter()
+        oracle.quaternary_gemm(case.x[:rows], case.w)
+        dt = time.perf_counter() - t0
+        rows2 = int(max(rows, min(n, rows * 12.0 / max(dt, 1e-6))))
+        t0 = time.perf_counter()
+        oracle.quaternary_gemm(case.x[:rows2], case.w)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": 2.0 * rows2 * n * n / dt / 1e12, "unit": "TOPS", "cores": oracle.threads(),
+                                "kind": "oracle", "sample": f"first {rows2} of {n} rows, all columns", "seconds": dt}
+    print(json.dumps(line))
+
+
 def run_ours(args, case, name):
     import torch
     import torch.distributed as dist
@@ -691,6 +806,26 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     case = WORKLOADS[args.workload]()
+    if isinstance(case, QuaternaryCase):
+        if args.impl == "reference":
+            import oracle
+            if int(os.environ.get("RANK", "0")) == 0:
+                t0 = time.perf_counter()
+                rows = 64
+                oracle.quaternary_gemm(case.x[:rows], case.w)
+                dt = time.perf_counter() - t0
+                v = 2.0 * rows * case.n * case.n / dt / 1e12
+                print(json.dumps({"impl": "reference", "metric": "effective 2-bit TOPS (2MNK/s)", "value": v, "unit": "TOPS",
+                                  "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt,
+                                  "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+                                  "data": "synthetic", "config": {"workload": args.workload},
+                                  "cpu_baseline": {"value": v, "unit": "TOPS", "cores": oracle.threads(), "kind": "oracle",
+                                                   "sample": f"first {rows} of {case.n} rows, all columns"},
+                                  "e2e": {"value": v, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                                  "gpu_launches": 0}))
+        else:
+            run_quaternary(args, case, args.workload)
+        return
     if isinstance(case, BodyCase):
         if args.steps == 2000:          # the default suits 20 us kernels; a chain step is a few milliseconds
             args.steps = 100

@@ -204,6 +204,19 @@ rtn_status rtn_ternary_conv2d_packed(const void* x_packed, int64_t B, int64_t C,
                                      const float* next_t_lo, const float* next_t_hi, int64_t n_next_thr,
                                      void* out_packed, int32_t* dbg_acc, void* stream);
 
+/* The paper's comparison workload (section "Efficient Computation Pattern", Table 1's last column and the
+ * DoReFa-Net pattern it cites): 2-bit quaternary values q = 2*b1 + b2 in {0,1,2,3}, dot products by AND
+ * between each bit plane of the two inputs, popcount, power-of-two shifts and four partial sums:
+ *     x.w = 4 bC(X1&W1) + 2 bC(X1&W2) + 2 bC(X2&W1) + bC(X2&W2).
+ * Same packed operand format, with plane 1 = first bit (weight 2) and plane 2 = second bit (weight 1).
+ *
+ * rtn_pack_quaternary: q_values uint8 [rows][K] in {0..3} -> packed rows (16-byte aligned).  Synchronises
+ *   `stream`; RTN_ERR_VALUE if a value is above 3 (output then unspecified).
+ * rtn_quaternary_gemm: out[m][n] = sum_k x[m][k] * w[n][k], exact int32 ([M][N] row-major; <= 9 K). */
+rtn_status rtn_pack_quaternary(const uint8_t* q_values, int64_t rows, int64_t K, void* packed, void* stream);
+rtn_status rtn_quaternary_gemm(const void* a_packed, const void* w_packed, int64_t M, int64_t N, int64_t K,
+                               int32_t* out, void* stream);
+
 /* The variant RTN_VARIANT_AUTO resolves to for a shape (never AUTO). */
 rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
 rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,

@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     RtnError, lib, lib_path,
     rtn_packed_row_bytes, rtn_packed_bytes, rtn_conv_packed_k, rtn_conv_out_dim,
     rtn_pack_weights, rtn_ternarize_pack_act, rtn_ternary_gemm, rtn_ternary_conv2d,
+    rtn_pack_quaternary, rtn_quaternary_gemm,
     rtn_ternary_conv2d_noalloc, rtn_ternary_conv2d_fused, rtn_ternary_conv2d_packed,
     rtn_last_device_status, rtn_choose_gemm_variant, rtn_choose_conv_variant, rtn_conv_kernel_launches, rtn_conv_next_kernel_launches,
     PAD_CODE_ZERO, PAD_VALUE_ZERO, VARIANT_AUTO, VARIANT_POPC, VARIANT_I8,

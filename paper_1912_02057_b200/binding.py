@@ -77,6 +77,10 @@ def lib():
         L.rtn_ternary_conv2d_packed.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp, _vp,
                                                 _i64, _i64, _i64, _i64, _i64, _int, _f32, _f32,
                                                 _vp, _vp, _i64] + _tail
+        L.rtn_pack_quaternary.restype = _int
+        L.rtn_pack_quaternary.argtypes = [_vp, _i64, _i64, _vp, _vp]
+        L.rtn_quaternary_gemm.restype = _int
+        L.rtn_quaternary_gemm.argtypes = [_vp, _vp, _i64, _i64, _i64, _vp, _vp]
         L.rtn_choose_gemm_variant.restype = _int
         L.rtn_choose_gemm_variant.argtypes = [_i64] * 3
         L.rtn_choose_conv_variant.restype = _int
@@ -247,6 +251,24 @@ def rtn_ternary_conv2d_packed(x_packed, B, Cin, H, W, w_packed, w_sum, N, kh, kw
         *_next_tail(relu, skip, out, next_t_lo, next_t_hi, out_packed, dbg_acc, stream)),
         "rtn_ternary_conv2d_packed")
     return out, out_packed
+
+
+def rtn_pack_quaternary(q_values, stream=None):
+    """uint8 values [rows,K] in {0..3} on the device -> packed rows uint8 [rows, row_bytes]."""
+    rows, K = q_values.shape
+    packed = torch.empty((rows, rtn_packed_row_bytes(K)), dtype=torch.uint8, device=q_values.device)
+    _check(lib().rtn_pack_quaternary(_ptr(q_values, torch.uint8), rows, K, _ptr(packed), _stream(stream)),
+           "rtn_pack_quaternary")
+    return packed
+
+
+def rtn_quaternary_gemm(a_packed, w_packed, M, N, K, out=None, stream=None):
+    """Packed 2-bit x 2-bit GEMM (the paper's comparison workload) -> exact int32 [M,N]."""
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.int32, device=a_packed.device)
+    _check(lib().rtn_quaternary_gemm(_ptr(a_packed), _ptr(w_packed), M, N, K, _ptr(out, torch.int32),
+                                     _stream(stream)), "rtn_quaternary_gemm")
+    return out
 
 
 def rtn_choose_gemm_variant(M, N, K):

@@ -350,6 +350,41 @@ rtn_status rtn_ternary_conv2d_packed(const void* x_packed, int64_t B, int64_t C,
     return conv_next(c, x_packed, relu, skip, next_t_lo, next_t_hi, n_next_thr, out_packed, stream);
 }
 
+rtn_status rtn_pack_quaternary(const uint8_t* q_values, int64_t rows, int64_t K, void* packed, void* stream)
+{
+    if (q_values == nullptr || packed == nullptr) return RTN_ERR_NULL;
+    if (rows <= 0 || K <= 0 || rows >= kMaxDim || K > kMaxK) return RTN_ERR_SHAPE;
+    if (!aligned16(packed)) return RTN_ERR_ALIGN;
+    unsigned* st = status_word();
+    if (st == nullptr) return RTN_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (rtn::launch_pack_quaternary(q_values, rows, K, static_cast<uint8_t*>(packed), st, s) != cudaSuccess)
+        return RTN_ERR_CUDA;
+    unsigned h = 0;
+    if (cudaMemcpyAsync(&h, st, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return RTN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return RTN_ERR_CUDA;
+    if (h & rtn::kStatusBadWeightCode) {
+        const unsigned keep = h & ~rtn::kStatusBadWeightCode;
+        cudaMemcpyAsync(st, &keep, sizeof(keep), cudaMemcpyHostToDevice, s);
+        cudaStreamSynchronize(s);
+        return RTN_ERR_VALUE;
+    }
+    return RTN_OK;
+}
+
+rtn_status rtn_quaternary_gemm(const void* a_packed, const void* w_packed, int64_t M, int64_t N, int64_t K,
+                               int32_t* out, void* stream)
+{
+    if (a_packed == nullptr || w_packed == nullptr || out == nullptr) return RTN_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || M >= kMaxDim || N >= kMaxDim || K > kMaxK) return RTN_ERR_SHAPE;
+    if (!aligned16(a_packed) || !aligned16(w_packed) || !aligned4(out)) return RTN_ERR_ALIGN;
+    if ((M + 15) / 16 > INT_MAX || (N + 15) / 16 > 65535) return RTN_ERR_UNSUPPORTED;
+    const cudaError_t e = rtn::launch_gemm_quaternary(static_cast<const uint8_t*>(a_packed),
+                                                      static_cast<const uint8_t*>(w_packed), M, N, K, out,
+                                                      static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
 rtn_status rtn_last_device_status(void* stream)
 {
     unsigned* st = status_word();

@@ -82,6 +82,12 @@ cudaError_t launch_gemm_popc(const GemmArgs& g, cudaStream_t s);
 bool conv_popc_supported(const ConvArgs& c);
 cudaError_t launch_conv_popc(const ConvArgs& c, cudaStream_t s);
 
+// The paper's 2-bit quaternary comparison workload (AND / popcount / shift pattern).
+cudaError_t launch_pack_quaternary(const uint8_t* q, int64_t rows, int64_t K, uint8_t* packed, unsigned* status,
+                                   cudaStream_t s);
+cudaError_t launch_gemm_quaternary(const uint8_t* a, const uint8_t* w, int64_t M, int64_t N, int64_t K, int32_t* out,
+                                   cudaStream_t s);
+
 // Tensor-core (tcgen05 kind::i8) variants; *_supported say whether a shape can run there.
 bool gemm_i8_supported(int64_t M, int64_t N, int64_t K);
 cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s);
