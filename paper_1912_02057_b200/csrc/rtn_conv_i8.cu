@@ -721,6 +721,73 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             if constexpr (kNext) {
                 next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, buf, g, nrows,
                                    alive, q, lane, half);
+            } else if (p.const_tmem && a.dbg_acc == nullptr && ntm == 2 && a.pad_mode == RTN_PAD_CODE_ZERO) {
+                // Full tile, constants in tensor memory, no border classes: the thread's pixels of both
+                // sub-tiles go through the channel blocks together, so that one fetch of a block's
+                // constants serves two pixels and the epilogue waits for tensor memory half as often
+                // (the wait for a tcgen05.ld, several hundred cycles while the tensor core works on the next
+                // tile, is what this epilogue's time is made of).
+                float* optr2[2];
+                bool ok2[2];
+                uint32_t trow2[2], sx2[2];
+                #pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const uint32_t pl = (uint32_t)(t * kTileM + q * 32 + lane);
+                    const uint32_t row = fdiv(pl, p.div_pw);
+                    const int wo = (int)(pl - row * (uint32_t)p.PW);
+                    const uint32_t G = (uint32_t)g + row;
+                    const uint32_t b = fdiv(G, p.div_ph);
+                    const int ho = (int)(G - b * (uint32_t)p.PH);
+                    ok2[t] = alive && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
+                    trow2[t] = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + t) * p.Np);
+                    optr2[t] = a.out + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
+                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
+                                 : "=r"(sx2[t]) : "r"(trow2[t] + (uint32_t)a.N) : "memory");
+                }
+                tc::tmem_ld_wait();
+                const float fsx0 = (float)(int)sx2[0], fsx1 = (float)(int)sx2[1];
+                for (int blk = blk_begin; blk < blk_end; ++blk) {
+                    const int n0 = blk * 16;
+                    if (n0 + 16 <= a.N) {
+                        #pragma unroll
+                        for (int h8 = 0; h8 < 16; h8 += 8) {
+                            uint32_t u0[8], u1[8], k1[8], k2[8], k3[8];
+                            tc::tmem_ld8(trow2[0] + (uint32_t)(n0 + h8), u0);
+                            tc::tmem_ld8(trow2[1] + (uint32_t)(n0 + h8), u1);
+                            tc::tmem_ld8(cq + (uint32_t)(n0 + h8), k1);
+                            tc::tmem_ld8(cq + p.Nc + (uint32_t)(n0 + h8), k2);
+                            tc::tmem_ld8(cq + 2 * p.Nc + (uint32_t)(n0 + h8), k3);
+                            tc::tmem_ld_wait();
+                            if (ok2[0]) {
+                                #pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    optr2[0][(int64_t)(n0 + h8 + j) * ostride] =
+                                        fmaf(__uint_as_float(k1[j]), (float)(int)u0[j],
+                                             fmaf(__uint_as_float(k2[j]), fsx0, __uint_as_float(k3[j])));
+                            }
+                            if (ok2[1]) {
+                                #pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    optr2[1][(int64_t)(n0 + h8 + j) * ostride] =
+                                        fmaf(__uint_as_float(k1[j]), (float)(int)u1[j],
+                                             fmaf(__uint_as_float(k2[j]), fsx1, __uint_as_float(k3[j])));
+                            }
+                        }
+                    } else {
+                        // the last, ragged block: constants from shared memory
+                        uint32_t u0[16], u1[16];
+                        tc::tmem_ld16(trow2[0] + (uint32_t)n0, u0);
+                        tc::tmem_ld16(trow2[1] + (uint32_t)n0, u1);
+                        tc::tmem_ld_wait();
+                        #pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (n0 + j >= a.N) continue;
+                            const float4 c = sC[n0 + j];
+                            if (ok2[0]) optr2[0][(int64_t)(n0 + j) * ostride] = fmaf(c.x, (float)(int)u0[j], fmaf(c.y, fsx0, c.z));
+                            if (ok2[1]) optr2[1][(int64_t)(n0 + j) * ostride] = fmaf(c.x, (float)(int)u1[j], fmaf(c.y, fsx1, c.z));
+                        }
+                    }
+                }
             } else
             for (int tm = 0; tm < ntm; ++tm) {
                 const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);     // pixel within the tile
