@@ -37,6 +37,9 @@ WORKLOADS = {
     "cfg3a_conv3x3_c256_14x14_b128": lambda: inputs.config3a(0.5, batch=128),
     "cfg3b_conv1x1s2_c128_28x28_b128": lambda: inputs.config3b(0.5, batch=128),
     "cfg1_gemm_64x64x576": inputs.config1,
+    # a batch of 16 samples through a wide linear layer (K cut into slices by the bit-plane kernel)
+    "linear_m16_n256_k9216": lambda: inputs.gemm_case("linear_m16_n256_k9216", 16, 256, 9216, seed=9, p_zero=0.5,
+                                                      thresholds=(0.3, 1.0)),
     "cfg5_gemm_2048": lambda: inputs.config5(2048),
     "cfg5_gemm_4096": lambda: inputs.config5(4096),
     "cfg5_gemm_8192": lambda: inputs.config5(8192),
@@ -644,7 +647,7 @@ def run_ours(args, case, name):
         sums = [torch.empty((M,), dtype=torch.int32, device="cuda") for _ in range(n_sets)]
         outs = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _ in range(n_sets)]
         variant = rtn.rtn_choose_gemm_variant(M, N, K)
-        launches_per_step = 2
+        launches_per_step = 2 if rtn.rtn_gemm_k_slices(M, N, K) <= 1 else 4        # sliced K: memset + 2 kernels
 
         def step(i):
             j = i % n_sets

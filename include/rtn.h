@@ -219,6 +219,12 @@ rtn_status rtn_quaternary_gemm(const void* a_packed, const void* w_packed, int64
 
 /* The variant RTN_VARIANT_AUTO resolves to for a shape (never AUTO). */
 rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
+/* Slices of K that RTN_VARIANT_AUTO cuts a GEMM shape into (1 = none).  A linear layer with few rows and
+ * columns and a long K (the paper's "both convolution and linear layers", section "Efficient Computation
+ * Pattern") has too few output tiles to fill the GPU: the bit-plane kernel then works on slices of K in
+ * parallel, adds their exact integer parts into the output buffer and applies the affine form in place
+ * (3 launches instead of 1; the integers do not depend on the order of the additions). */
+int64_t rtn_gemm_k_slices(int64_t M, int64_t N, int64_t K);
 rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
                                     int64_t kh, int64_t kw, int64_t stride, int64_t pad);
 /* Kernel launches one rtn_ternary_conv2d call with RTN_VARIANT_AUTO makes for a shape: 1, or 2 on the

@@ -128,7 +128,16 @@ rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K)
     // Tiny problems finish inside one wave of the bit-plane kernel before the tensor-core
     // pipeline has filled; everything else is far faster on the tensor cores.
     if (M * N <= 128 * 128 && K <= 1024) return RTN_VARIANT_POPC;
+    // A linear layer with few rows and columns and a long K is one or two tiles for the tensor-core
+    // kernel, whose single CTA then walks all of K; the bit-plane kernel cuts K into slices instead.
+    if (M * N <= 64 * 256 && rtn::gemm_popc_slices(M, N, K) > 1) return RTN_VARIANT_POPC;
     return RTN_VARIANT_I8;
+}
+
+int64_t rtn_gemm_k_slices(int64_t M, int64_t N, int64_t K)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    return rtn_choose_gemm_variant(M, N, K) == RTN_VARIANT_POPC ? rtn::gemm_popc_slices(M, N, K) : 1;
 }
 
 rtn_status rtn_ternary_gemm(const void* a_packed, const int32_t* a_sum,

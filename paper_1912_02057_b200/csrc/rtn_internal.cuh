@@ -79,6 +79,7 @@ cudaError_t launch_ternarize_pack(const float* a, int64_t M, int64_t K, const fl
                                   const float* t_hi, int64_t n_thr, uint8_t* packed, int32_t* a_sum,
                                   cudaStream_t s);
 cudaError_t launch_gemm_popc(const GemmArgs& g, cudaStream_t s);
+int gemm_popc_slices(int64_t M, int64_t N, int64_t K);     // K slices the bit-plane GEMM cuts a shape into (1 = none)
 bool conv_popc_supported(const ConvArgs& c);
 cudaError_t launch_conv_popc(const ConvArgs& c, cudaStream_t s);
 

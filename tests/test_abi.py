@@ -69,3 +69,11 @@ def test_argument_errors_come_back_as_codes_without_a_gpu():
     assert conv(4, 3, 1, 1, 0, nthr=3) == 2
     assert conv(4, 3, 1, 1, 7) == 4
     assert rtn.lib().rtn_status_string(2).startswith(b"RTN_ERR_SHAPE")
+
+
+def test_k_slices_only_for_small_outputs_with_a_long_k():
+    assert rtn.rtn_gemm_k_slices(64, 64, 576) == 1            # config 1: one launch
+    assert rtn.rtn_gemm_k_slices(4096, 4096, 4096) == 1       # tensor-core kernel
+    assert rtn.rtn_gemm_k_slices(16, 256, 9216) > 1
+    assert rtn.rtn_gemm_k_slices(64, 4096, 9216) == 1         # enough output tiles without slicing
+    assert rtn.rtn_gemm_k_slices(0, 4, 4) == 0

@@ -83,6 +83,19 @@ def test_gemm_ragged_shapes(M, N, K, variant):
     run_or_skip_unsupported(lambda: gemm_parity(case, variant), variant)
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 1000, 4608), (8, 40, 9000), (64, 64, 16384), (16, 256, 9216), (33, 17, 1025)])
+def test_linear_layer_with_few_rows_is_cut_along_k(M, N, K):
+    """A batch of a few samples through a wide linear layer: AUTO resolves to the bit-plane kernel with K
+    cut into slices (integer parts added atomically into the output buffer, affine form in place); the
+    integers and the fp32 outputs meet the same bar as everywhere."""
+    assert rtn.rtn_choose_gemm_variant(M, N, K) == rtn.VARIANT_POPC
+    assert rtn.rtn_gemm_k_slices(M, N, K) > 1
+    case = inputs.gemm_case(f"linear_{M}x{N}x{K}", M, N, K, seed=M + N + K, p_zero=0.35, act="uniform3",
+                            thresholds=(-0.5, 0.5), per_row_act_params=(M % 2 == 1))
+    gemm_parity(case, rtn.VARIANT_AUTO)
+    gemm_parity(case, rtn.VARIANT_AUTO)          # a second call starts from a used output buffer
+
+
 @pytest.mark.parametrize("variant", VARIANTS)
 def test_gemm_degenerate_codes(variant):
     # all-zero codes -> K*a_o*w_o; all +1 against all -1 -> S_xw = -K
