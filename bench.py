@@ -88,7 +88,8 @@ INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
 NCU_TRAFFIC_BYTES = {
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch; a kernel's fp32 output is still in L2
     # when the kernel ends, so the write-back of most of it falls outside the capture window
-    "cfg2_conv3x3_c64_56x56_b32": 25_796_096 + 29_184,
+    "cfg2_conv3x3_c64_56x56_b32": 25_799_424 + 11_008,
+    "cfg2_conv3x3_c64_56x56_b32/packed": 3_311_872 + 0,
     "cfg3a_conv3x3_c256_14x14_b128": 26_113_280 + 195_840,
     "cfg3b_conv1x1s2_c128_28x28_b128": 51_698_432 + 2_256_896,
     "cfg5_gemm_4096": 8_664_832 + 15_990_016,
