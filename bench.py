@@ -212,9 +212,10 @@ def ops_of(case):
 # ------------------------------------------------------------------------------------------------
 # CPU oracle leg (reference arm and cpu_baseline)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample(case, budget_s=12.0, io="fp32"):
+def oracle_sample(case, budget_s=12.0, io="fp32", fill_budget=False):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload.
-    Returns (ops per second, seconds, description)."""
+    Returns (ops per second, seconds, description).  fill_budget: when the whole batch takes a small part
+    of the budget, run it several times in a row so that the figure rests on about budget_s of CPU work."""
     import oracle
     if isinstance(case, inputs.ConvCase):
         def run(nb):
@@ -233,7 +234,16 @@ def oracle_sample(case, budget_s=12.0, io="fp32"):
         nb = int(max(1, min(case.B, budget_s / max(dt, 1e-6))))
         if nb > 1:
             ops, dt = run(nb)
-        return ops / dt, dt, f"first {nb} of {case.B} images, all output channels (ternarize + conv2d + epilogue)"
+        what = f"first {nb} of {case.B} images, all output channels (ternarize + conv2d + epilogue)"
+        if fill_budget and nb == case.B and dt < budget_s / 3:
+            reps = int(min(40, budget_s / max(dt, 1e-6)))
+            tot_ops, tot_dt = 0.0, 0.0
+            for _ in range(reps):
+                o, d = run(nb)
+                tot_ops, tot_dt = tot_ops + o, tot_dt + d
+            ops, dt = tot_ops, tot_dt
+            what = f"the whole batch of {case.B} images {reps} times in a row, all output channels (ternarize + conv2d + epilogue)"
+        return ops / dt, dt, what
 
     def run(rows):
         a = case.a[:rows]
@@ -785,7 +795,7 @@ def run_ours(args, case, name):
         }
         if not args.no_cpu_baseline and world == 1:
             import oracle
-            rate, dt, sample = oracle_sample(case, 12.0, args.io)
+            rate, dt, sample = oracle_sample(case, 12.0, args.io, fill_budget=True)
             line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TOPS", "cores": oracle.threads(),
                                     "kind": "oracle", "sample": sample, "seconds": dt}
         print(json.dumps(line))
