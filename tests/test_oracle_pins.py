@@ -501,3 +501,30 @@ def test_pack_quaternary_rows_planes():
     assert p[0, 1] == 2 and p[0, 17] == 0              # value 2 at position 9: first-bit plane only
     assert p[0, 32] == 0 and p[0, 48] == 2             # value 1 at position 129: second-bit plane of block 1
     assert p.sum() == 1 + 1 + 2 + 2
+
+
+# ------------------------------------------------------------------ the chain's recipe (host logic, no arithmetic of the method)
+@pytest.mark.parametrize("hin", [56, 28, 16])
+def test_resnet18_body_recipe_is_a_consistent_chain(hin):
+    layers = inputs.resnet18_body(seed=4, hin=hin)
+    assert [l.name for l in layers] == [l[0] for l in inputs.resnet18_ternary_layers()]
+    blocks = inputs.resnet18_body_blocks(layers)
+    assert len(blocks) == 8 and sum(b["down"] is not None for b in blocks) == 3
+    size, chans = hin, 64
+    for blk in blocks:
+        c1, c2, down = blk["conv1"], blk["conv2"], blk["down"]
+        assert c1.cin == chans and c1.hin == size
+        out = oracle.conv_out_dim(c1.hin, c1.k, c1.stride, c1.pad)
+        assert c2.cin == c1.cout and c2.hin == out and c2.stride == 1
+        assert oracle.conv_out_dim(c2.hin, c2.k, 1, c2.pad) == out
+        if down is not None:
+            assert (down.cin, down.cout, down.hin) == (c1.cin, c2.cout, c1.hin)
+            assert oracle.conv_out_dim(down.hin, down.k, down.stride, down.pad) == out
+        else:
+            assert c1.stride == 1 and c1.cin == c2.cout      # the skip is the block's input itself
+        for l in (c1, c2, down):
+            if l is not None:
+                assert 0 < float(l.t_lo[0]) < float(l.t_hi[0])
+        size, chans = out, c2.cout
+    if hin == 56:
+        assert (size, chans) == (7, 512)
