@@ -241,3 +241,43 @@ def test_next_layer_argument_errors():
         rtn.rtn_ternary_conv2d_fused(*args, out_packed=outp, next_t_lo=dev(np.zeros(3, np.float32)),
                                      next_t_hi=dev(np.ones(3, np.float32)))
     assert e.value.code == 2
+
+
+@pytest.mark.parametrize("name,maker", [
+    ("cfg2", lambda: inputs.config2(batch=32, thresholds=(0.3, 1.0))),          # one-kernel variant
+    ("cfg3a", lambda: inputs.config3a(0.5, batch=128)),                          # two-kernel variant
+])
+def test_next_layer_full_size_sampled(name, maker):
+    """The benchmark's shapes at full batch, in the launch configuration bench.py times (packed rows in, ReLU,
+    skip, fp32 and packed rows out): sampled outputs against the oracle point by point, the four image corners
+    and the last channel included."""
+    case = maker()
+    g = inputs.rng(91)
+    B, C, H, W, N, Ho, Wo = case.B, case.C, case.H, case.W, case.N, case.Ho, case.Wo
+    codes_in = oracle.ternarize(case.x, case.t_lo, case.t_hi, channel_axis=1)
+    skip = g.standard_normal((B, N, Ho, Wo)).astype(np.float32)
+    nlo, nhi = next_thresholds(g, N, True, lo=2.0, hi=12.0)
+    acc, y, packed = run_layer(case, codes_in, True, oracle.PAD_CODE_ZERO, True, skip, True, nlo, nhi)
+    n_pts = 6000
+    pts = np.stack([g.integers(0, B, n_pts), g.integers(0, N, n_pts), g.integers(0, Ho, n_pts),
+                    g.integers(0, Wo, n_pts)], 1)
+    corners = [(b, n, h, v) for b in (0, B - 1) for n in (0, N - 1) for h in (0, Ho - 1) for v in (0, Wo - 1)]
+    pts = np.concatenate([pts, np.array(corners, np.int64)], 0)
+    S, pre, mag = oracle.conv2d_points(codes_in, case.w_codes, case.stride, case.pad, oracle.PAD_CODE_ZERO,
+                                       case.a_scale, case.a_offset, case.w_scale, case.w_offset, pts)
+    ix = tuple(pts.T)
+    assert np.array_equal(acc[ix].astype(np.int64), S), f"{name}: sampled accumulators differ"
+    # the hand-over step at the sampled points: one "image" of len(pts) channels-by-1 values, thresholds per point
+    sk = skip[ix]
+    y_ref, codes_ref, margin = oracle.next_layer(pre.reshape(1, -1, 1), True, sk.reshape(1, -1, 1),
+                                                 nlo[pts[:, 1]], nhi[pts[:, 1]])
+    y_ref, codes_ref, margin = y_ref.ravel(), codes_ref.ravel(), margin.ravel()
+    mag_y = mag + np.abs(sk.astype(np.float64))
+    check_fp32(y[ix], y_ref, mag_y, name + " y (sampled)")
+    got = oracle.unpack_nhwc(packed, B, N, Ho, Wo)[ix]
+    clear = margin > np.maximum(oracle.REL_TOL * np.abs(y_ref), oracle.ABS_TOL * np.maximum(1.0, mag_y))
+    assert clear.mean() > 0.999
+    assert np.array_equal(got[clear], codes_ref[clear]), f"{name}: sampled codes differ away from the thresholds"
+    assert set(np.unique(got).tolist()) == {-1, 0, 1}
+    # every packed row is canonical (00 zeros, zero fill past N)
+    assert np.array_equal(packed, oracle.pack_nhwc(oracle.unpack_nhwc(packed, B, N, Ho, Wo)))
