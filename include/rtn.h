@@ -7,8 +7,11 @@
  *
  * Conventions
  *   - Every data pointer is a DEVICE pointer unless its comment says "host".  The caller owns
- *     every buffer; the library allocates no memory and keeps no state besides one device
- *     status word (see rtn_last_device_status).
+ *     every input and output buffer.  The library keeps no state besides one device status word (see
+ *     rtn_last_device_status) and, per device, the fixed scratch array of rtn_ternary_conv2d_noalloc.
+ *     Convolutions that take the two-kernel path (rtn_conv_kernel_launches / rtn_conv_next_kernel_launches
+ *     say which) borrow a scratch buffer from the stream-ordered allocator for the duration of the call
+ *     (cudaMallocAsync / cudaFreeAsync on `stream`); nothing else is allocated.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
  *     enqueue work and return without synchronising, except rtn_pack_weights and
  *     rtn_last_device_status, which synchronise the stream.
