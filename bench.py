@@ -90,7 +90,7 @@ NCU_TRAFFIC_BYTES = {
     # when the kernel ends, so the write-back of most of it falls outside the capture window
     "cfg2_conv3x3_c64_56x56_b32": 25_799_424 + 11_008,
     "cfg2_conv3x3_c64_56x56_b32/packed": 3_311_872 + 0,
-    "cfg3a_conv3x3_c256_14x14_b128": 26_113_280 + 195_840,
+    "cfg3a_conv3x3_c256_14x14_b128": 26_533_888 + 196_096,
     "cfg3b_conv1x1s2_c128_28x28_b128": 51_698_432 + 2_256_896,
     "cfg5_gemm_4096": 8_664_832 + 15_990_016,
 }

@@ -233,7 +233,8 @@ int64_t rtn_conv_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W, int
     c.B = (int)B; c.C = (int)C; c.H = (int)H; c.W = (int)W; c.N = (int)N; c.kh = (int)kh; c.kw = (int)kw;
     c.stride = (int)stride; c.pad = (int)pad;
     c.Ho = (int)rtn_conv_out_dim(H, kh, stride, pad); c.Wo = (int)rtn_conv_out_dim(W, kw, stride, pad);
-    if (rtn::conv_i8_supported(c) || rtn::conv_i8s_supported(c)) return 1;
+    if (rtn::conv_i8_supported(c)) return 1;
+    if (rtn::conv_i8s_supported(c)) return rtn::conv_i8s_launches(c);
     return rtn::conv_i8r_supported(c) ? 2 : 1;
 }
 

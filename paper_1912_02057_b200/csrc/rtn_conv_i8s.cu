@@ -16,7 +16,13 @@
 //   * S_x comes from per-pixel code sums the ternarizer leaves in shared memory (summed over the
 //     taps in the epilogue), so all 256 accumulator columns are free for output channels;
 //   * a 1x1 convolution (any stride, no padding) uses the same code with "rows" = output rows and a
-//     strided pixel gather in the ternarizer (no halo, one tap).
+//     strided pixel gather in the ternarizer (no halo, one tap);
+//   * for a long filter stream (four stages or more) every CTA expanding the whole bank again is the
+//     kernel's largest cost (cfg3a: 18 stages of about 1 us each per tile against 9 us of MMAs), so
+//     the bank is expanded ONCE, by a small kernel of its own, into a scratch buffer laid out stage by
+//     stage as the ring wants it; one thread of the contraction kernel then fills the ring with bulk
+//     asynchronous copies (one 32 KB run per stage, served by L2) and the expander warps have
+//     nothing to do.
 //
 // Warp roles: warp 0 issues MMAs (one thread); warps 12..19 expand filters; warps 4..11 ternarize
 // tile i+1 and then run the epilogue of tile i; warps 1..3 only ternarize.  One or two code buffers
@@ -64,6 +70,7 @@ struct ConvI8SPlan {
     uint32_t off_a[2], off_w, off_psum, off_lo, off_hi, off_c, off_bar, off_misc;
     size_t smem_bytes;
     int blocks_major;      // stage order: 128-channel block outer, tap inner (else the packed order)
+    int pre;               // filters expanded beforehand into scratch, slices in (32-channel group, tap) order
     uint32_t tab_a[kMaxK]; // per slice of the stage order: start of the A window in 16-byte units of
                            // the code buffer (bits 0..23) and its 32-channel group (bits 24..27);
                            // 0xFFFFFFFF for the padding slices of the last packed block
@@ -108,7 +115,19 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
     p.nK = nblocks * kSlices;
     if (p.nK > kMaxK) return false;
     p.blocks_major = (cwords % kSlices == 0) ? 1 : 0;
-    for (int st = 0; st < nblocks; ++st) {
+    // A long filter stream is expanded beforehand into scratch, and the order of its K = 32 slices is then
+    // free: 32-channel group outer, tap inner, so that the tensor core starts on a tile as soon as the
+    // first 32 channels are ternarized and follows the ternarizers group by group.
+    p.pre = nblocks >= 4 ? 1 : 0;
+    for (int i = 0; p.pre && i < p.nK; ++i) {
+        uint32_t e = 0xFFFFFFFFu;
+        if (i < nwords) {
+            const int h = i / p.T, t = i % p.T;
+            e = ((uint32_t)(2 * h) * p.ppix + (uint32_t)((t / c.kw) * p.PW + (t % c.kw))) | ((uint32_t)h << 24);
+        }
+        p.tab_a[i] = e;
+    }
+    for (int st = 0; !p.pre && st < nblocks; ++st) {
         // packed block of stage st
         const int blk = p.blocks_major ? (st % p.T) * (cwords / kSlices) + st / p.T : st;
         for (int j = 0; j < kSlices; ++j) {
@@ -162,8 +181,43 @@ __device__ __forceinline__ void role_wait(bool leader, uint64_t* bar, uint32_t p
     asm volatile("bar.sync %0, %1;" ::"r"(barrier_id), "r"(nthreads) : "memory");
 }
 
+// The filter bank expanded once: wexp[stage][16-byte k chunk (8)][filter row (Np)][16 B], the bytes a ring
+// stage holds, in the slice order of the plan (32-channel group outer, tap inner).  Thread = (stage, filter row).
+__global__ void __launch_bounds__(256)
+conv_expand_filters_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, uint4* __restrict__ wexp)
+{
+    tc::pdl_trigger();          // the contraction kernel may start its set-up (it reads no expanded filters there)
+    const int nstages = p.nK / kSlices;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)nstages * p.Np) return;
+    const int st = (int)(i / p.Np), row = (int)(i % p.Np);
+    const int cwords = p.Cp / 32, nwords = p.T * cwords;
+    const int64_t row_blocks = ((int64_t)p.T * cwords + 3) / 4;
+    const uint32_t* Wrow = reinterpret_cast<const uint32_t*>(a.w_packed) + (int64_t)row * row_blocks * 8;
+    uint4* dst = wexp + (int64_t)st * kSlices * 2 * p.Np + row;
+    #pragma unroll
+    for (int j = 0; j < kSlices; ++j) {
+        // slice st*4 + j of the stream = (32-channel group h, tap t) = word t*cwords + h of the packed row
+        const int s = st * kSlices + j;
+        uint32_t nz = 0, sg = 0;
+        if (s < nwords && row < a.N) {
+            const int h = s / p.T, t = s - h * p.T;
+            const int word = t * cwords + h;
+            nz = __ldg(Wrow + (word >> 2) * 8 + (word & 3));
+            sg = __ldg(Wrow + (word >> 2) * 8 + 4 + (word & 3));
+        }
+        uint32_t o[8];
+        tc::unpack32(nz, sg, o);
+        dst[(2 * j) * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[(2 * j + 1) * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
+// kPre: the filter stages come from the scratch buffer conv_expand_filters_kernel wrote (bulk copies by
+// one thread) instead of being expanded by warps 12..19.
+template <bool kPre>
 __global__ void __launch_bounds__(kThreads, 1)
-conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
+conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const uint4* __restrict__ wexp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     uint4* sWr = reinterpret_cast<uint4*>(smem + p.off_w);       // [nW][kSlices][2][Np]
@@ -198,7 +252,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
             tc::mbar_init(&acc_full[i], 1);
             tc::mbar_init(&acc_empty[i], kEpiThreads);
         }
-        for (int i = 0; i < kMaxWStages; ++i) { tc::mbar_init(&w_full[i], kExpWarps); tc::mbar_init(&w_empty[i], 1); }
+        for (int i = 0; i < kMaxWStages; ++i) { tc::mbar_init(&w_full[i], kPre ? 1 : kExpWarps); tc::mbar_init(&w_empty[i], 1); }
         for (int i = 0; i < 2 * kMaxGroups; ++i) tc::mbar_init(&a_full[i], kTernThreads);
         tc::mbar_init_fence();
         *dead = 0;
@@ -378,6 +432,22 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
         // ------------------------------------------------------------ filter expanders
         // thread = filter row; a stage = one packed block of the row (four K = 32 slices).  The
         // planes of the next two stages are in flight while this one expands.
+        if constexpr (kPre) {
+            // one thread streams the expanded stages into the ring
+            if (warp == kExpWarp0 && lane == 0) {
+                const uint32_t stage_bytes = (uint32_t)p.Np * 32u * kSlices;
+                const uint32_t ring = tc::smem_addr(sWr);
+                uint32_t wcount = 0;
+                bool alive = true;
+                for (int it = 0; it < ntile && alive; ++it)
+                    for (int s = 0; s < nstages; ++s, ++wcount) {
+                        const uint32_t st = wcount % (uint32_t)p.nW;
+                        if (!wait_or_die(&w_empty[st], ((wcount / (uint32_t)p.nW) & 1) ^ 1, a.status, dead)) { alive = false; break; }
+                        tc::mbar_arrive_expect_tx(&w_full[st], stage_bytes);
+                        tc::bulk_copy_g2s(ring + st * stage_bytes, wexp + (size_t)s * (stage_bytes / 16), stage_bytes, &w_full[st]);
+                    }
+            }
+        } else {
         const int tid = threadIdx.x - kExpWarp0 * 32;
         const int cwords = p.Cp / 32;
         const int64_t row_blocks = ((int64_t)p.T * cwords + 3) / 4;
@@ -427,6 +497,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p)
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&w_full[st]);
             }
+        }
         }
     } else if (warp == 0) {
         // ------------------------------------------------------------ MMA issue (one thread)
@@ -516,14 +587,43 @@ bool conv_i8s_supported(const ConvArgs& c)
     return make_plan_s(c, p, 148);
 }
 
+// A filter stream of four stages or more is expanded once into scratch (an extra small kernel).
+static bool pre_expand(const ConvI8SPlan& p) { return p.pre != 0; }
+
+int conv_i8s_launches(const ConvArgs& c)
+{
+    ConvI8SPlan p;
+    if (!make_plan_s(c, p, 148)) return 0;
+    return pre_expand(p) ? 2 : 1;
+}
+
 cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s)
 {
     ConvI8SPlan p;
     if (!make_plan_s(c, p, sm_count_s())) return cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaFuncSetAttribute(conv_i8s_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)p.smem_bytes);
+    if (!pre_expand(p)) {
+        cudaError_t e = cudaFuncSetAttribute(conv_i8s_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)p.smem_bytes);
+        if (e != cudaSuccess) return e;
+        return launch_pdl(conv_i8s_kernel<false>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
+                          (const uint4*)nullptr);
+    }
+    // scratch from the stream-ordered allocator, given back right after the two launches, in stream order
+    const int nstages = p.nK / kSlices;
+    const size_t bytes = (size_t)nstages * p.Np * 32 * kSlices;
+    void* scratch = nullptr;
+    cudaError_t e = cudaMallocAsync(&scratch, bytes, s);
     if (e != cudaSuccess) return e;
-    return launch_pdl(conv_i8s_kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p);
+    const int64_t items = (int64_t)nstages * p.Np;
+    conv_expand_filters_kernel<<<(unsigned)((items + 255) / 256), 256, 0, s>>>(c, p, reinterpret_cast<uint4*>(scratch));
+    e = cudaGetLastError();
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(conv_i8s_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    if (e == cudaSuccess)
+        e = launch_pdl(conv_i8s_kernel<true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
+                       (const uint4*)scratch);
+    const cudaError_t e2 = cudaFreeAsync(scratch, s);
+    return e != cudaSuccess ? e : e2;
 }
 
 }  // namespace rtn

@@ -96,6 +96,7 @@ bool conv_i8_supported(const ConvArgs& c);       // filters resident in shared m
 cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s);
 bool conv_i8s_supported(const ConvArgs& c);      // filters streamed (large layers, 1x1 of any stride)
 cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s);
+int conv_i8s_launches(const ConvArgs& c);       // 1, or 2 when the filter bank is expanded into scratch first (0: not taken)
 bool conv_i8r_supported(const ConvArgs& c);      // two kernels: int8 codes in a scratch buffer, filter bank split over CTAs
 size_t conv_i8r_scratch_bytes(const ConvArgs& c);
 cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s);     // scratch from the stream-ordered allocator

@@ -68,6 +68,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
     return false;
 }
 
+// ------------------------------------------------------------------------------------ bulk copies
+// One contiguous run of global memory -> shared memory, asynchronously; completion is counted in bytes
+// on `bar` (no tensor map, no multicast).  Both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// One arrival on `bar` that also announces `bytes` of asynchronous copies to come.
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+
 // ------------------------------------------------------------------------------------ launch overlap
 // Programmatic dependent launch.  The kernel is launched so that its CTAs may start while the
 // previous kernel of the stream is still draining: every access to tensors that kernel may write or read sits behind
