@@ -64,6 +64,7 @@ struct ConvI8SPlan {
     int nK;                // K = 32 slices per tile in stage order, padded to whole packed blocks
     int nW;                // filter ring depth
     int nAcc;              // accumulator sets (1 or 2)
+    int npass, NpP;        // passes over the output channels (2 when N > 256) and columns per pass
     int nA;                // code buffers (1 or 2)
     uint32_t tmem_cols;
     FastDiv div_pw, div_ph, div_T;   // div_T: stage -> (128-channel block, tap)
@@ -91,20 +92,25 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
     if ((int64_t)c.B * p.PH > (1 << 20)) return false;
     p.Cp = (c.C + 31) / 32 * 32;
     p.Np = (c.N + 15) / 16 * 16;
-    if (p.Np > 256) return false;
+    // More than 256 filters: two passes over the tile's codes, 256 output channels each; a pass is to the
+    // accumulator sets and their barriers what a tile is, so with two sets the first pass's epilogue runs
+    // under the second pass's MMAs.  Only with the filters expanded beforehand (checked below).
+    if (p.Np > 512) return false;
+    p.npass = p.Np > 256 ? 2 : 1;
+    p.NpP = p.npass == 2 ? 256 : p.Np;
     if (p.Cp / 32 > kMaxGroups) return false;
     p.total_rows = c.B * p.PH;
     p.grid = p.total_rows < sms ? p.total_rows : sms;
     // 256-pixel tiles whenever a CTA's strip has more than 128 pixels: a tile's filter stream costs
     // the same whatever its size
     const int strip_rows = (p.total_rows + p.grid - 1) / p.grid;
-    p.TM = (2 * p.Np <= 512 && strip_rows * p.PW > kTileM) ? 2 : 1;
-    p.nAcc = (2 * p.TM * p.Np <= 512) ? 2 : 1;
+    p.TM = (2 * p.NpP <= 512 && strip_rows * p.PW > kTileM) ? 2 : 1;
+    p.nAcc = (2 * p.TM * p.NpP <= 512) ? 2 : 1;
     p.RT = p.TM * kTileM / p.PW;
     if (p.RT < 1) return false;
     p.ppix = (p.TM * kTileM + p.halo * p.PW + (c.kw - 1) + 7) / 8 * 8;
     uint32_t cols = 32;
-    while (cols < (uint32_t)(p.nAcc * p.TM * p.Np)) cols *= 2;
+    while (cols < (uint32_t)(p.nAcc * p.TM * p.NpP)) cols *= 2;
     p.tmem_cols = cols;
     p.div_pw = make_fastdiv((uint32_t)p.PW);
     p.div_ph = make_fastdiv((uint32_t)p.PH);
@@ -119,6 +125,7 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
     // free: 32-channel group outer, tap inner, so that the tensor core starts on a tile as soon as the
     // first 32 channels are ternarized and follows the ternarizers group by group.
     p.pre = nblocks >= 4 ? 1 : 0;
+    if (p.npass > 1 && !p.pre) return false;
     for (int i = 0; p.pre && i < p.nK; ++i) {
         uint32_t e = 0xFFFFFFFFu;
         if (i < nwords) {
@@ -141,7 +148,7 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
         }
     }
     const uint32_t a_bytes = (uint32_t)(p.Cp / 16) * p.ppix * 16;
-    const uint32_t stage = (uint32_t)p.Np * 32 * kSlices;
+    const uint32_t stage = (uint32_t)p.NpP * 32 * kSlices;
     const int nstages = p.nK / kSlices;
     // two code buffers when they leave room for a filter ring of four stages (or all of them)
     for (p.nA = 2; p.nA >= 1; --p.nA) {
@@ -181,7 +188,7 @@ __device__ __forceinline__ void role_wait(bool leader, uint64_t* bar, uint32_t p
     asm volatile("bar.sync %0, %1;" ::"r"(barrier_id), "r"(nthreads) : "memory");
 }
 
-// The filter bank expanded once: wexp[stage][16-byte k chunk (8)][filter row (Np)][16 B], the bytes a ring
+// The filter bank expanded once: wexp[pass][stage][16-byte k chunk (8)][filter row of the pass][16 B], the bytes a ring
 // stage holds, in the slice order of the plan (32-channel group outer, tap inner).  Thread = (stage, filter row).
 __global__ void __launch_bounds__(256)
 conv_expand_filters_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, uint4* __restrict__ wexp)
@@ -189,16 +196,18 @@ conv_expand_filters_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan
     tc::pdl_trigger();          // the contraction kernel may start its set-up (it reads no expanded filters there)
     const int nstages = p.nK / kSlices;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= (int64_t)nstages * p.Np) return;
-    const int st = (int)(i / p.Np), row = (int)(i % p.Np);
+    if (i >= (int64_t)p.npass * nstages * p.NpP) return;
+    const int st = (int)(i / p.NpP);                        // pass * nstages + stage of the pass
+    const int row = (int)(i % p.NpP) + (st / nstages) * p.NpP;      // filter
+    const int stage_of_pass = st % nstages;
     const int cwords = p.Cp / 32, nwords = p.T * cwords;
     const int64_t row_blocks = ((int64_t)p.T * cwords + 3) / 4;
     const uint32_t* Wrow = reinterpret_cast<const uint32_t*>(a.w_packed) + (int64_t)row * row_blocks * 8;
-    uint4* dst = wexp + (int64_t)st * kSlices * 2 * p.Np + row;
+    uint4* dst = wexp + (int64_t)st * kSlices * 2 * p.NpP + (i % p.NpP);
     #pragma unroll
     for (int j = 0; j < kSlices; ++j) {
-        // slice st*4 + j of the stream = (32-channel group h, tap t) = word t*cwords + h of the packed row
-        const int s = st * kSlices + j;
+        // slice stage*4 + j of the stream = (32-channel group h, tap t) = word t*cwords + h of the packed row
+        const int s = stage_of_pass * kSlices + j;
         uint32_t nz = 0, sg = 0;
         if (s < nwords && row < a.N) {
             const int h = s / p.T, t = s - h * p.T;
@@ -208,8 +217,8 @@ conv_expand_filters_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan
         }
         uint32_t o[8];
         tc::unpack32(nz, sg, o);
-        dst[(2 * j) * p.Np] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[(2 * j + 1) * p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
+        dst[(2 * j) * p.NpP] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[(2 * j + 1) * p.NpP] = make_uint4(o[4], o[5], o[6], o[7]);
     }
 }
 
@@ -299,8 +308,6 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
         const int64_t ostride = (int64_t)a.Ho * a.Wo;
         const int nblk16 = (a.N + 15) / 16;
-        const int blk_begin = half == 0 ? 0 : (nblk16 + 1) / 2;
-        const int blk_end = half == 0 ? (nblk16 + 1) / 2 : nblk16;
         for (int step = 0; step <= ntile; ++step) {
             if (step < ntile) {
                 const int it = step, g = s0 + it * rt;
@@ -355,13 +362,19 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             if (step >= 1 && epi_warp) {
                 const int it = step - 1, g = s0 + it * rt;
                 const int nrows = min(rt, s1 - g);
-            const int acc = p.nAcc == 2 ? (it & 1) : 0;
-            const uint32_t acc_ph = p.nAcc == 2 ? ((it >> 1) & 1) : (it & 1);
             const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
             const int* psum = sPsum + (it & (kPsumRing - 1)) * p.ppix;
-            role_wait(warp == kEpiWarp0, &acc_full[acc], acc_ph, a.status, dead, kEpiBarrier, kEpiThreads);
+          for (int pass = 0; pass < p.npass; ++pass) {
+            const int vt = it * p.npass + pass;             // the accumulators go round per (tile, pass)
+            const int acc = p.nAcc == 2 ? (vt & 1) : 0;
+            const uint32_t acc_ph = p.nAcc == 2 ? ((vt >> 1) & 1) : (vt & 1);
+            const int slot_acc = acc;
+            role_wait(warp == kEpiWarp0, &acc_full[slot_acc], acc_ph, a.status, dead, kEpiBarrier, kEpiThreads);
             const bool alive = !*dead;
             tc::tc_fence_after_sync();
+            const int pass_blocks = p.npass == 2 ? min(p.NpP / 16, nblk16 - pass * (p.NpP / 16)) : nblk16;
+            const int pb_begin = half == 0 ? 0 : (pass_blocks + 1) / 2;
+            const int pb_end = half == 0 ? (pass_blocks + 1) / 2 : pass_blocks;
             for (int tm = 0; tm < ntm; ++tm) {
                 const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);
                 const uint32_t row = fdiv(pl, p.div_pw);
@@ -383,15 +396,15 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                 }
                 const bool border = n_inside < p.T;
                 const float fsx = (float)s_x;
-                const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((acc * p.TM + tm) * p.Np);
+                const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((slot_acc * p.TM + tm) * p.NpP);
                 float* optr = a.out + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
                 int32_t* dptr = a.dbg_acc ? a.dbg_acc + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo : nullptr;
-                for (int blk = blk_begin; blk < blk_end; ++blk) {
+                for (int blk = pb_begin; blk < pb_end; ++blk) {
                     uint32_t v[16];
                     tc::tmem_ld16(trow + (uint32_t)(blk * 16), v);
                     tc::tmem_ld_wait();
                     if (!ok) continue;
-                    const int n0 = blk * 16;
+                    const int n0 = pass * p.NpP + blk * 16;
                     if (!border && dptr == nullptr && n0 + 16 <= a.N) {
                         #pragma unroll
                         for (int j = 0; j < 16; ++j) {
@@ -426,6 +439,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[acc]);
+          }
             }
         }
     } else if (warp >= kExpWarp0 && warp < kExpWarp0 + kExpWarps) {
@@ -435,12 +449,12 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
         if constexpr (kPre) {
             // one thread streams the expanded stages into the ring
             if (warp == kExpWarp0 && lane == 0) {
-                const uint32_t stage_bytes = (uint32_t)p.Np * 32u * kSlices;
+                const uint32_t stage_bytes = (uint32_t)p.NpP * 32u * kSlices;
                 const uint32_t ring = tc::smem_addr(sWr);
                 uint32_t wcount = 0;
                 bool alive = true;
                 for (int it = 0; it < ntile && alive; ++it)
-                    for (int s = 0; s < nstages; ++s, ++wcount) {
+                    for (int s = 0; s < p.npass * nstages; ++s, ++wcount) {      // pass after pass
                         const uint32_t st = wcount % (uint32_t)p.nW;
                         if (!wait_or_die(&w_empty[st], ((wcount / (uint32_t)p.nW) & 1) ^ 1, a.status, dead)) { alive = false; break; }
                         tc::mbar_arrive_expect_tx(&w_full[st], stage_bytes);
@@ -504,11 +518,11 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
         // The tensor core's queue is short, so whatever the issuing thread does between two MMAs is
         // tensor-core idle time: the A offsets of a stage are fetched one stage ahead.
         if (lane == 0) {
-            const uint32_t idesc = tc::idesc_i8(kTileM, (uint32_t)p.Np);
+            const uint32_t idesc = tc::idesc_i8(kTileM, (uint32_t)p.NpP);
             const uint64_t desc_hi = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
             const uint32_t a_lbo_field = (((uint32_t)p.ppix * 16) >> 4) << 16;
-            const uint32_t w16 = (tc::smem_addr(sWr) >> 4) + ((((uint32_t)p.Np * 16) >> 4) << 16);
-            const uint32_t wslice16 = ((uint32_t)p.Np * 32) >> 4;
+            const uint32_t w16 = (tc::smem_addr(sWr) >> 4) + ((((uint32_t)p.NpP * 16) >> 4) << 16);
+            const uint32_t wslice16 = ((uint32_t)p.NpP * 32) >> 4;
             const uint32_t wstage16 = wslice16 * kSlices;
             uint32_t wcount = 0;
             int it = 0;
@@ -516,18 +530,20 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             for (int g = s0; g < s1 && alive; g += rt, ++it) {
                 const int buf = p.nA == 2 ? (it & 1) : 0;
                 const uint32_t use_ph = p.nA == 2 ? ((it >> 1) & 1) : (it & 1);
-                const int acc = p.nAcc == 2 ? (it & 1) : 0;
-                const uint32_t acc_ph = p.nAcc == 2 ? ((it >> 1) & 1) : (it & 1);
                 const int nrows = min(rt, s1 - g);
                 const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
                 const uint32_t a16 = (tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4) + a_lbo_field;
                 uint64_t* full = &a_full[buf * kMaxGroups];
-                alive = wait_or_die(&acc_empty[acc], acc_ph ^ 1, a.status, dead);
+                uint32_t ready = 0;             // 32-channel groups whose codes are known to be written
+              for (int pass = 0; pass < p.npass && alive; ++pass) {
+                const int vt = it * p.npass + pass;
+                const int slot_acc = p.nAcc == 2 ? (vt & 1) : 0;
+                const uint32_t acc_ph = p.nAcc == 2 ? ((vt >> 1) & 1) : (vt & 1);
+                alive = wait_or_die(&acc_empty[slot_acc], acc_ph ^ 1, a.status, dead);
                 if (!alive) break;
                 uint32_t ta[kSlices], tn[kSlices];
                 #pragma unroll
                 for (int j = 0; j < kSlices; ++j) tn[j] = p.tab_a[j];
-                uint32_t ready = 0;             // 32-channel groups whose codes are known to be written
                 bool accum = false;
                 for (int s = 0; s < nstages && alive; ++s, ++wcount) {
                     #pragma unroll
@@ -550,9 +566,9 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                             if (alive) {
                                 const uint64_t bd = desc_hi | (uint64_t)(w16 + st * wstage16 + (uint32_t)j * wslice16);
                                 const uint32_t aw = a16 + (ta[j] & 0xFFFFFFu);
-                                tc::mma_i8_ss(tmem + (uint32_t)((acc * p.TM) * p.Np), desc_hi | (uint64_t)aw, bd, idesc, accum);
+                                tc::mma_i8_ss(tmem + (uint32_t)((slot_acc * p.TM) * p.NpP), desc_hi | (uint64_t)aw, bd, idesc, accum);
                                 if (ntm == 2)
-                                    tc::mma_i8_ss(tmem + (uint32_t)((acc * p.TM + 1) * p.Np),
+                                    tc::mma_i8_ss(tmem + (uint32_t)((slot_acc * p.TM + 1) * p.NpP),
                                                   desc_hi | (uint64_t)(aw + (uint32_t)kTileM), bd, idesc, accum);
                                 accum = true;
                             }
@@ -560,9 +576,10 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                     }
                     if (alive) tc::mma_commit(&w_empty[st]);
                 }
+                if (alive) tc::mma_commit(&acc_full[slot_acc]);      // this pass's accumulators are complete
+              }
                 if (!alive) break;
                 tc::mma_commit(&a_empty[buf]);
-                tc::mma_commit(&acc_full[acc]);
             }
         }
     }
@@ -610,11 +627,11 @@ cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s)
     }
     // scratch from the stream-ordered allocator, given back right after the two launches, in stream order
     const int nstages = p.nK / kSlices;
-    const size_t bytes = (size_t)nstages * p.Np * 32 * kSlices;
+    const size_t bytes = (size_t)p.npass * nstages * p.NpP * 32 * kSlices;
     void* scratch = nullptr;
     cudaError_t e = cudaMallocAsync(&scratch, bytes, s);
     if (e != cudaSuccess) return e;
-    const int64_t items = (int64_t)nstages * p.Np;
+    const int64_t items = (int64_t)p.npass * nstages * p.NpP;
     conv_expand_filters_kernel<<<(unsigned)((items + 255) / 256), 256, 0, s>>>(c, p, reinterpret_cast<uint4*>(scratch));
     e = cudaGetLastError();
     if (e == cudaSuccess)

@@ -171,9 +171,11 @@ SMALL_CONVS = [
     (3, 128, 9, 7, 256, 3, 1, 1),
     (2, 100, 10, 14, 250, 3, 1, 1),
     (2, 64, 8, 8, 256, 5, 1, 2),
-    # more than 256 filters: the two-kernel variant (int8 codes in scratch, filter bank split over CTAs)
+    # more than 256 filters: two passes of the streamed-filter kernel over the tile's codes (3x3, 5x5), the
+    # two-kernel variant with the filter bank split over CTAs where the filter stream is short (1x1)
     (1, 129, 6, 5, 260, 3, 1, 1),
     (2, 512, 7, 7, 512, 3, 1, 1),
+    (5, 256, 14, 14, 400, 3, 1, 1),
     (2, 96, 9, 12, 300, 5, 1, 2),
     (3, 64, 10, 10, 272, 1, 1, 0),
     # strided filters: phase images of the two-kernel variant
