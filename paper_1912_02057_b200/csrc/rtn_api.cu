@@ -234,7 +234,8 @@ int64_t rtn_conv_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W, int
     c.stride = (int)stride; c.pad = (int)pad;
     c.Ho = (int)rtn_conv_out_dim(H, kh, stride, pad); c.Wo = (int)rtn_conv_out_dim(W, kw, stride, pad);
     if (rtn::conv_i8_supported(c)) return 1;
-    if (rtn::conv_i8s_supported(c)) return rtn::conv_i8s_launches(c);
+    if (rtn::conv_i8s_supported(c) && (!rtn::conv_i8r_supported(c) || rtn::conv_prefers_streamed(c)))
+        return rtn::conv_i8s_launches(c);
     return rtn::conv_i8r_supported(c) ? 2 : 1;
 }
 
@@ -246,6 +247,8 @@ int64_t rtn_conv_next_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W
     c.stride = (int)stride; c.pad = (int)pad;
     c.Ho = (int)rtn_conv_out_dim(H, kh, stride, pad); c.Wo = (int)rtn_conv_out_dim(W, kw, stride, pad);
     if (rtn::conv_i8_next_supported(c)) return 1;
+    if (rtn::conv_i8s_next_supported(c) && (!rtn::conv_i8r_next_supported(c) || rtn::conv_prefers_streamed(c)))
+        return rtn::conv_i8s_next_launches(c);
     return rtn::conv_i8r_next_supported(c) ? 2 : 0;
 }
 
@@ -310,7 +313,9 @@ static rtn_status conv_next(rtn::ConvArgs& c, const void* x_packed, int relu, co
     }
     if ((x_packed != nullptr && !aligned16(x_packed)) || (skip != nullptr && !aligned4(skip))) return RTN_ERR_ALIGN;
     const bool one_kernel = rtn::conv_i8_next_supported(c);
-    if (!one_kernel && !rtn::conv_i8r_next_supported(c)) return RTN_ERR_UNSUPPORTED;
+    const bool streamed = !one_kernel && rtn::conv_i8s_next_supported(c) &&
+                          (!rtn::conv_i8r_next_supported(c) || rtn::conv_prefers_streamed(c));
+    if (!one_kernel && !streamed && !rtn::conv_i8r_next_supported(c)) return RTN_ERR_UNSUPPORTED;
     rtn::NextLayerArgs f{};
     f.x_packed = static_cast<const uint8_t*>(x_packed);
     f.relu = relu;
@@ -320,7 +325,8 @@ static rtn_status conv_next(rtn::ConvArgs& c, const void* x_packed, int relu, co
     c.status = status_word();
     if (c.status == nullptr) return RTN_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const cudaError_t e = one_kernel ? rtn::launch_conv_i8_next(c, f, s) : rtn::launch_conv_i8r_next(c, f, s);
+    const cudaError_t e = one_kernel ? rtn::launch_conv_i8_next(c, f, s)
+                        : streamed ? rtn::launch_conv_i8s_next(c, f, s) : rtn::launch_conv_i8r_next(c, f, s);
     return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
 }
 

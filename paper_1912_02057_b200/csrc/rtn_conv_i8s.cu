@@ -68,7 +68,7 @@ struct ConvI8SPlan {
     int nA;                // code buffers (1 or 2)
     uint32_t tmem_cols;
     FastDiv div_pw, div_ph, div_T;   // div_T: stage -> (128-channel block, tap)
-    uint32_t off_a[2], off_w, off_psum, off_lo, off_hi, off_c, off_bar, off_misc;
+    uint32_t off_a[2], off_w, off_psum, off_lo, off_hi, off_c, off_t, off_bar, off_misc;
     size_t smem_bytes;
     int blocks_major;      // stage order: 128-channel block outer, tap inner (else the packed order)
     int pre;               // filters expanded beforehand into scratch, slices in (32-channel group, tap) order
@@ -77,7 +77,7 @@ struct ConvI8SPlan {
                            // 0xFFFFFFFF for the padding slices of the last packed block
 };
 
-bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
+bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
 {
     if (c.Ho <= 0 || c.Wo <= 0) return false;
     p.T = c.kh * c.kw;
@@ -160,6 +160,7 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms)
         p.off_hi = o;   o += (uint32_t)p.Cp * 4;
         o = (o + 15) / 16 * 16;
         p.off_c = o;    o += (uint32_t)p.Np * 16;
+        p.off_t = o;    o += next ? (uint32_t)p.Np * 8 : 0;     // float2 {t_lo, t_hi} of the next layer per column
         p.off_bar = o;  o += (6 + 2 * kMaxWStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] w_full[] w_empty[] a_full[2][]
         p.off_misc = o; o += 16;
         o = (o + 127) / 128 * 128;
@@ -224,9 +225,13 @@ conv_expand_filters_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan
 
 // kPre: the filter stages come from the scratch buffer conv_expand_filters_kernel wrote (bulk copies by
 // one thread) instead of being expanded by warps 12..19.
-template <bool kPre>
+// kNext: the layer hands its result to the next one (NextLayerArgs): the input may come as packed pixel
+// rows (the ternarizers then expand bit planes), and the epilogue applies phi, adds the skip connection and
+// writes fp32 and / or packed Eq. 3 codes against the next layer's thresholds.
+template <bool kPre, bool kNext>
 __global__ void __launch_bounds__(kThreads, 1)
-conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const uint4* __restrict__ wexp)
+conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const uint4* __restrict__ wexp,
+                const NextLayerArgs f)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     uint4* sWr = reinterpret_cast<uint4*>(smem + p.off_w);       // [nW][kSlices][2][Np]
@@ -266,7 +271,19 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
         tc::mbar_init_fence();
         *dead = 0;
     }
-    for (int c = threadIdx.x; c < p.Cp; c += kThreads) {
+    bool packed_in = false;
+    if constexpr (kNext) packed_in = f.x_packed != nullptr;
+    if constexpr (kNext) {
+        // the next layer's threshold pair per column; columns past N code to 0
+        float2* sT = reinterpret_cast<float2*>(smem + p.off_t);
+        for (int n = threadIdx.x; n < p.Np; n += kThreads) {
+            float2 t = make_float2(-INFINITY, INFINITY);
+            if (f.out_packed != nullptr && n < a.N)
+                t = make_float2(f.next_lo[f.n_next == 1 ? 0 : n], f.next_hi[f.n_next == 1 ? 0 : n]);
+            sT[n] = t;
+        }
+    }
+    for (int c = threadIdx.x; c < p.Cp && !packed_in; c += kThreads) {
         float lo = c < a.C ? a.t_lo[a.n_thr == 1 ? 0 : c] : -INFINITY;
         const float hi = c < a.C ? a.t_hi[a.n_thr == 1 ? 0 : c] : INFINITY;
         if (lo > hi) lo = nextafterf(hi, INFINITY);      // v < lo  <=>  v <= hi: -1 unless +1
@@ -304,7 +321,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
         const bool epi_warp = warp >= kEpiWarp0;
         const int64_t cs = (int64_t)a.H * a.W;
         const bool per_layer = a.n_thr == 1 && a.C == p.Cp;     // padding channels need their own (infinite) thresholds
-        const float lo0 = sLo[0], hi0 = sHi[0];
+        const float lo0 = packed_in ? 0.f : sLo[0], hi0 = packed_in ? 0.f : sHi[0];
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
         const int64_t ostride = (int64_t)a.Ho * a.Wo;
         const int nblk16 = (a.N + 15) / 16;
@@ -331,6 +348,25 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                 const uint32_t b = fdiv(G, p.div_ph);
                 const int r = (int)(G - b * (uint32_t)p.PH) * p.istride - p.ipad;
                 uint4 w0 = make_uint4(0, 0, 0, 0), w1 = make_uint4(0, 0, 0, 0);
+                if (packed_in) {
+                    // packed pixel rows: one word of each bit plane = the 32 codes of this (pixel, group)
+                    if constexpr (kNext) {
+                        if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
+                            const int64_t row_bytes = (int64_t)((a.C + kBlockCodes - 1) / kBlockCodes) * kBlockBytes;
+                            const uint32_t* blk = reinterpret_cast<const uint32_t*>(
+                                f.x_packed + (((int64_t)b * a.H + r) * a.W + c) * row_bytes) + (h >> 2) * 8 + (h & 3);
+                            uint32_t nz = __ldg(blk);
+                            const uint32_t sg = __ldg(blk + 4);
+                            if (h * 32 + 32 > a.C) nz &= (1u << (a.C - h * 32)) - 1u;      // positions past C code to 0
+                            uint32_t o[8];
+                            tc::unpack32(nz, sg, o);
+                            w0 = make_uint4(o[0], o[1], o[2], o[3]);
+                            w1 = make_uint4(o[4], o[5], o[6], o[7]);
+                            const int sm = __popc(nz & sg) - __popc(nz & ~sg);
+                            if (sm != 0) atomicAdd(&psum[pp], sm);
+                        }
+                    }
+                } else
                 if (b < (uint32_t)a.B && r >= 0 && r < a.H && c >= 0 && c < a.W) {
                     const float* src = a.x + (((int64_t)b * a.C + h * 32) * a.H + r) * a.W + c;
                     float v0[16], v1[16];
@@ -399,12 +435,36 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                 const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((slot_acc * p.TM + tm) * p.NpP);
                 float* optr = a.out + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
                 int32_t* dptr = a.dbg_acc ? a.dbg_acc + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo : nullptr;
+                // packed output: this pixel's row of N codes; the positions from the last computed block to the
+                // end of the last 128-code block are zero-filled (first warp set, last pass)
+                const int packed_cols = (a.N + kBlockCodes - 1) / kBlockCodes * kBlockCodes;
+                uint8_t* out_row = nullptr;
+                if constexpr (kNext) {
+                    if (ok && f.out_packed != nullptr) {
+                        out_row = f.out_packed + (((int64_t)b * a.Ho + ho) * a.Wo + wo) * (int64_t)(packed_cols / 4);
+                        if (half == 0 && pass == p.npass - 1) zero_fill_packed_row(out_row, nblk16 * 16, packed_cols);
+                    }
+                }
                 for (int blk = pb_begin; blk < pb_end; ++blk) {
                     uint32_t v[16];
                     tc::tmem_ld16(trow + (uint32_t)(blk * 16), v);
                     tc::tmem_ld_wait();
                     if (!ok) continue;
                     const int n0 = pass * p.NpP + blk * 16;
+                    if constexpr (kNext) {
+                        uint32_t nzb, sgb;
+                        const bool codes = out_row != nullptr && n0 < packed_cols;
+                        next_layer_block16(a, f, v, sC + n0, reinterpret_cast<const float2*>(smem + p.off_t) + n0, fsx,
+                                           border, p.T, ho, wo, n_inside, n0,
+                                           (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo + (int64_t)n0 * ostride, ostride,
+                                           codes, nzb, sgb);
+                        if (codes) {
+                            uint8_t* dst = out_row + (n0 >> 7) * kBlockBytes + ((n0 & 127) >> 3);
+                            *reinterpret_cast<uint16_t*>(dst) = (uint16_t)nzb;
+                            *reinterpret_cast<uint16_t*>(dst + 16) = (uint16_t)sgb;
+                        }
+                        continue;
+                    }
                     if (!border && dptr == nullptr && n0 + 16 <= a.N) {
                         #pragma unroll
                         for (int j = 0; j < 16; ++j) {
@@ -614,16 +674,17 @@ int conv_i8s_launches(const ConvArgs& c)
     return pre_expand(p) ? 2 : 1;
 }
 
-cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s)
+template <bool kNext>
+static cudaError_t launch_i8s_mode(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s)
 {
     ConvI8SPlan p;
-    if (!make_plan_s(c, p, sm_count_s())) return cudaErrorInvalidConfiguration;
+    if (!make_plan_s(c, p, sm_count_s(), kNext)) return cudaErrorInvalidConfiguration;
     if (!pre_expand(p)) {
-        cudaError_t e = cudaFuncSetAttribute(conv_i8s_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(conv_i8s_kernel<false, kNext>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)p.smem_bytes);
         if (e != cudaSuccess) return e;
-        return launch_pdl(conv_i8s_kernel<false>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
-                          (const uint4*)nullptr);
+        return launch_pdl(conv_i8s_kernel<false, kNext>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
+                          (const uint4*)nullptr, f);
     }
     // scratch from the stream-ordered allocator, given back right after the two launches, in stream order
     const int nstages = p.nK / kSlices;
@@ -635,12 +696,46 @@ cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s)
     conv_expand_filters_kernel<<<(unsigned)((items + 255) / 256), 256, 0, s>>>(c, p, reinterpret_cast<uint4*>(scratch));
     e = cudaGetLastError();
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(conv_i8s_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+        e = cudaFuncSetAttribute(conv_i8s_kernel<true, kNext>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)p.smem_bytes);
     if (e == cudaSuccess)
-        e = launch_pdl(conv_i8s_kernel<true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
-                       (const uint4*)scratch);
+        e = launch_pdl(conv_i8s_kernel<true, kNext>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p,
+                       (const uint4*)scratch, f);
     const cudaError_t e2 = cudaFreeAsync(scratch, s);
     return e != cudaSuccess ? e : e2;
+}
+
+cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s) { return launch_i8s_mode<false>(c, NextLayerArgs{}, s); }
+
+// Rough time of this variant for a shape, in microseconds (negative: not taken), for the choice between it
+// and the variant that splits the filter bank over CTAs.  Measured on B200: a CTA's time is the filter stream of
+// its tiles, about 0.75 us per 32 KB stage from scratch (1 us when the stage is expanded in the kernel),
+// whatever the batch, plus about 13 us of ternarizing, epilogue and launch.
+double conv_i8s_estimate_us(const ConvArgs& c)
+{
+    ConvI8SPlan p;
+    if (!make_plan_s(c, p, 148)) return -1.0;
+    const int strip_rows = (p.total_rows + p.grid - 1) / p.grid;
+    const int tiles = (strip_rows + p.RT - 1) / p.RT;
+    const double stage_us = (p.pre ? 0.75 : 1.0) * (double)p.NpP / 256.0;
+    return 13.0 + (double)tiles * p.npass * (p.nK / kSlices) * stage_us;
+}
+
+// The same kernels with the hand-over to the next layer (and, optionally, packed input).
+bool conv_i8s_next_supported(const ConvArgs& c)
+{
+    ConvI8SPlan p;
+    return make_plan_s(c, p, 148, true);
+}
+int conv_i8s_next_launches(const ConvArgs& c)
+{
+    ConvI8SPlan p;
+    if (!make_plan_s(c, p, 148, true)) return 0;
+    return pre_expand(p) ? 2 : 1;
+}
+cudaError_t launch_conv_i8s_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s)
+{
+    return launch_i8s_mode<true>(c, f, s);
 }
 
 }  // namespace rtn

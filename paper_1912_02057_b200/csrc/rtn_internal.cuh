@@ -105,16 +105,29 @@ size_t conv_i8r_static_scratch_bytes();
 // Two-kernel path with the fused hand-over to the next layer (and, optionally, packed input).
 bool conv_i8_next_supported(const ConvArgs& c);    // one-kernel variant (filters resident)
 cudaError_t launch_conv_i8_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s);
+bool conv_i8s_next_supported(const ConvArgs& c);   // streamed-filter variant
+int conv_i8s_next_launches(const ConvArgs& c);
+cudaError_t launch_conv_i8s_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s);
 bool conv_i8r_next_supported(const ConvArgs& c);
 cudaError_t launch_conv_i8r_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s);
 inline bool conv_i8_any_supported(const ConvArgs& c)
 {
     return conv_i8_supported(c) || conv_i8s_supported(c) || conv_i8r_supported(c);
 }
+// Rough times (us; negative: shape not taken) behind the choice between the streamed-filter variant, whose
+// time is set by the filter stream and hardly moves with the batch, and the split-bank variant, whose time
+// grows with the pixels.
+double conv_i8s_estimate_us(const ConvArgs& c);
+double conv_i8r_estimate_us(const ConvArgs& c);
+inline bool conv_prefers_streamed(const ConvArgs& c)
+{
+    const double ts = conv_i8s_estimate_us(c), tr = conv_i8r_estimate_us(c);
+    return ts >= 0.0 && (tr < 0.0 || ts <= 0.9 * tr);      // the estimates are rough: a tie goes to the split bank
+}
 inline cudaError_t launch_conv_i8_any(const ConvArgs& c, cudaStream_t s)
 {
     if (conv_i8_supported(c)) return launch_conv_i8(c, s);
-    if (conv_i8s_supported(c)) return launch_conv_i8s(c, s);
+    if (conv_i8s_supported(c) && (!conv_i8r_supported(c) || conv_prefers_streamed(c))) return launch_conv_i8s(c, s);
     return launch_conv_i8r(c, s);
 }
 
