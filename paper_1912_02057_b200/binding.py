@@ -83,6 +83,8 @@ def lib():
         L.rtn_quaternary_gemm.argtypes = [_vp, _vp, _i64, _i64, _i64, _vp, _vp]
         L.rtn_choose_gemm_variant.restype = _int
         L.rtn_choose_gemm_variant.argtypes = [_i64] * 3
+        L.rtn_gemm_kernel_launches.restype = _i64
+        L.rtn_gemm_kernel_launches.argtypes = [_i64] * 3
         L.rtn_gemm_k_slices.restype = _i64
         L.rtn_gemm_k_slices.argtypes = [_i64] * 3
         L.rtn_choose_conv_variant.restype = _int
@@ -275,6 +277,10 @@ def rtn_quaternary_gemm(a_packed, w_packed, M, N, K, out=None, stream=None):
 
 def rtn_choose_gemm_variant(M, N, K):
     return int(lib().rtn_choose_gemm_variant(M, N, K))
+
+
+def rtn_gemm_kernel_launches(M, N, K):
+    return int(lib().rtn_gemm_kernel_launches(M, N, K))
 
 
 def rtn_gemm_k_slices(M, N, K):

@@ -140,6 +140,13 @@ int64_t rtn_gemm_k_slices(int64_t M, int64_t N, int64_t K)
     return rtn_choose_gemm_variant(M, N, K) == RTN_VARIANT_POPC ? rtn::gemm_popc_slices(M, N, K) : 1;
 }
 
+int64_t rtn_gemm_kernel_launches(int64_t M, int64_t N, int64_t K)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    if (rtn_choose_gemm_variant(M, N, K) == RTN_VARIANT_I8) return rtn::gemm_i8_launches(M, N, K);
+    return rtn::gemm_popc_slices(M, N, K) > 1 ? 2 : 1;
+}
+
 rtn_status rtn_ternary_gemm(const void* a_packed, const int32_t* a_sum,
                             const void* w_packed, const int32_t* w_sum,
                             int64_t M, int64_t N, int64_t K,

@@ -92,8 +92,46 @@ bool make_gemm_plan(int64_t M, int64_t N, int64_t K, GemmI8Plan& p, int sms)
     return true;
 }
 
+// The weight operand expanded once: wexp[column tile][packed block of K][16-byte k chunk (8)][row of the
+// tile (BN)][16 B], the bytes the weight part of a ring stage holds.  Thread = (tile, block, row).
+__global__ void __launch_bounds__(256)
+gemm_expand_weights_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, uint4* __restrict__ wexp)
+{
+    tc::pdl_trigger();
+    const int64_t nblk = (g.K + kBlockCodes - 1) / kBlockCodes;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.tiles_n * nblk * p.BN) return;
+    const int r = (int)(i % p.BN);
+    const int64_t tk = i / p.BN, kb = tk % nblk, tn = tk / nblk;
+    const int64_t n = tn * p.BN + r;
+    uint4 nz = make_uint4(0, 0, 0, 0), sg = nz;
+    if (n < g.N) {
+        const uint4* src = reinterpret_cast<const uint4*>(g.w_packed + (n * nblk + kb) * kBlockBytes);
+        nz = __ldg(src);
+        sg = __ldg(src + 1);
+    }
+    uint4* dst = wexp + tk * 8 * p.BN + r;
+    uint32_t o[8];
+    tc::unpack32(nz.x, sg.x, o);
+    dst[0 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+    tc::unpack32(nz.y, sg.y, o);
+    dst[2 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[3 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+    tc::unpack32(nz.z, sg.z, o);
+    dst[4 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[5 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+    tc::unpack32(nz.w, sg.w, o);
+    dst[6 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[7 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
+// kPreW: the weight part of every stage comes from the scratch buffer gemm_expand_weights_kernel wrote (one
+// bulk asynchronous copy per stage, issued by a thread of warp 1), so the expander warps expand only the
+// activation rows: half of the integer work that paces the kernel.
+template <bool kPreW>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p)
+gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uint4* __restrict__ wexp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     float4* sC = reinterpret_cast<float4*>(smem + p.off_c);
@@ -112,7 +150,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p)
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
         for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kEpiThreads); }
-        for (int i = 0; i < kMaxStages; ++i) { tc::mbar_init(&full[i], kExpWarps); tc::mbar_init(&empty[i], 1); }
+        for (int i = 0; i < kMaxStages; ++i) { tc::mbar_init(&full[i], kExpWarps + (kPreW ? 1 : 0)); tc::mbar_init(&empty[i], 1); }
         tc::mbar_init_fence();
         *dead = 0;
     }
@@ -120,6 +158,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p)
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
+    if constexpr (kPreW) tc::pdl_wait();           // the expanded weights come from the kernel before
 
     if (warp >= kExpWarp0) {
         // ------------------------------------------------------------ expanders
@@ -135,7 +174,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p)
             for (int k = 0; k < 2; ++k) {
                 const int r = tid + k * kExpThreads;
                 src[k] = nullptr; dst_off[k] = nullptr; stride[k] = 0;
-                if (r < p.rows) {
+                if (r < (kPreW ? rowsA : p.rows)) {
                     const bool isA = r < rowsA;
                     const int64_t grow = isA ? m0 + r : n0 + (r - rowsA);
                     if (grow < (isA ? g.M : g.N))
@@ -190,6 +229,24 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p)
                 tc::fence_smem_to_async_proxy();
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&full[s]);
+            }
+        }
+    } else if (kPreW && warp == 1) {
+        // ------------------------------------------------------------ weight stages from scratch (one thread)
+        if (lane == 0) {
+            const uint32_t w_bytes = (uint32_t)p.BN * 128u;
+            const uint32_t w_off = (uint32_t)rowsA * 128u;            // the weight block follows the activation block
+            uint32_t count = 0;
+            bool alive = true;
+            for (int64_t tile = blockIdx.x; tile < p.tiles && alive; tile += gridDim.x) {
+                const int64_t tn = tile % p.tiles_n;
+                for (int64_t kb = 0; kb < nblk; ++kb, ++count) {
+                    const uint32_t s = count % (uint32_t)p.stages;
+                    if (!wait_or_die(&empty[s], ((count / (uint32_t)p.stages) & 1) ^ 1, g.status, dead)) { alive = false; break; }
+                    tc::mbar_arrive_expect_tx(&full[s], w_bytes);
+                    tc::bulk_copy_g2s(tc::smem_addr(smem + p.off_stage + s * p.stage_bytes + w_off),
+                                      wexp + (tn * nblk + kb) * (w_bytes / 16), w_bytes, &full[s]);
+                }
             }
         }
     } else if (warp == 0) {
@@ -325,14 +382,40 @@ bool gemm_i8_supported(int64_t M, int64_t N, int64_t K)
     return make_gemm_plan(M, N, K, p, 148);
 }
 
+int gemm_i8_launches(int64_t M, int64_t N, int64_t K)
+{
+    GemmI8Plan p;
+    if (!make_gemm_plan(M, N, K, p, 148)) return 0;
+    return p.tiles_m < 2 ? 1 : 2;
+}
+
 cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s)
 {
     GemmI8Plan p;
     if (!make_gemm_plan(g.M, g.N, g.K, p, sm_count_g())) return cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    // Every tile of a column re-expands that column's weights: with two or more row tiles the weights are
+    // expanded once into scratch instead (stream-ordered allocation, N rounded up to tiles x K bytes).
+    const int64_t nblk = (g.K + kBlockCodes - 1) / kBlockCodes;
+    const size_t wbytes = (size_t)p.tiles_n * nblk * p.BN * 128;
+    if (p.tiles_m < 2 || wbytes > (size_t(1) << 31)) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+        if (e != cudaSuccess) return e;
+        gemm_i8_kernel<false><<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(g, p, nullptr);
+        return cudaGetLastError();
+    }
+    void* scratch = nullptr;
+    cudaError_t e = cudaMallocAsync(&scratch, wbytes, s);
     if (e != cudaSuccess) return e;
-    gemm_i8_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(g, p);
-    return cudaGetLastError();
+    const int64_t items = p.tiles_n * nblk * p.BN;
+    gemm_expand_weights_kernel<<<(unsigned)((items + 255) / 256), 256, 0, s>>>(g, p, reinterpret_cast<uint4*>(scratch));
+    e = cudaGetLastError();
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    if (e == cudaSuccess)
+        e = launch_pdl(gemm_i8_kernel<true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, g, p,
+                       (const uint4*)scratch);
+    const cudaError_t e2 = cudaFreeAsync(scratch, s);
+    return e != cudaSuccess ? e : e2;
 }
 
 }  // namespace rtn

@@ -92,6 +92,7 @@ cudaError_t launch_gemm_quaternary(const uint8_t* a, const uint8_t* w, int64_t M
 // Tensor-core (tcgen05 kind::i8) variants; *_supported say whether a shape can run there.
 bool gemm_i8_supported(int64_t M, int64_t N, int64_t K);
 cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s);
+int gemm_i8_launches(int64_t M, int64_t N, int64_t K);     // 1, or 2 when the weights are expanded into scratch first
 bool conv_i8_supported(const ConvArgs& c);       // filters resident in shared memory (stride 1)
 cudaError_t launch_conv_i8(const ConvArgs& c, cudaStream_t s);
 bool conv_i8s_supported(const ConvArgs& c);      // filters streamed (large layers, 1x1 of any stride)
