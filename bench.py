@@ -92,7 +92,7 @@ NCU_TRAFFIC_BYTES = {
     "cfg2_conv3x3_c64_56x56_b32/packed": 3_311_872 + 0,
     "cfg3a_conv3x3_c256_14x14_b128": 26_533_888 + 196_096,
     "cfg3b_conv1x1s2_c128_28x28_b128": 51_397_888 + 51_456 + 3_419_648 + 256,    # both kernels of a step
-    "cfg5_gemm_4096": 21_263_104 + 16_880_128,
+    "cfg5_gemm_4096": 36_865_280 + 20_435_200,
 }
 
 

@@ -12,7 +12,7 @@
  *     Convolutions that take the two-kernel path (rtn_conv_kernel_launches / rtn_conv_next_kernel_launches
  *     say which) borrow a scratch buffer from the stream-ordered allocator for the duration of the call
  *     (cudaMallocAsync / cudaFreeAsync on `stream`), and so does the tensor-core GEMM for its expanded
- *     weights (rtn_gemm_kernel_launches); nothing else is allocated.
+ *     operands (rtn_gemm_kernel_launches); nothing else is allocated.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
  *     enqueue work and return without synchronising, except rtn_pack_weights and
  *     rtn_last_device_status, which synchronise the stream.
@@ -231,7 +231,8 @@ rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
 int64_t rtn_gemm_k_slices(int64_t M, int64_t N, int64_t K);
 /* Kernel launches of one rtn_ternary_gemm call with RTN_VARIANT_AUTO: 1; 2 when the tensor-core kernel first
  * expands the weight operand into a scratch buffer (stream-ordered allocation of about N*K bytes; shapes with
- * two or more row tiles) or when K is cut into slices (plus a memset). */
+ * two or more row tiles; with two or more column tiles as well the activations too, M*K bytes more) or when K
+ * is cut into slices (plus a memset). */
 int64_t rtn_gemm_kernel_launches(int64_t M, int64_t N, int64_t K);
 rtn_variant rtn_choose_conv_variant(int64_t B, int64_t C, int64_t H, int64_t W, int64_t N,
                                     int64_t kh, int64_t kw, int64_t stride, int64_t pad);

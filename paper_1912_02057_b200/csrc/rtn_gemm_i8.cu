@@ -31,8 +31,13 @@ constexpr int kExpWarps = 8;
 constexpr int kExpThreads = kExpWarps * 32;
 constexpr int kThreads = (kExpWarp0 + kExpWarps) * 32;
 constexpr int kMaxStages = 6;
-constexpr size_t kSmemLimit = 220 * 1024;
+constexpr size_t kSmemLimit = 226 * 1024;
 constexpr int kEpiBarrier = 3;
+// Output staging of the epilogue: per warp 32 rows x 8 columns of fp32, rows 48 bytes apart (32 + 16: both the
+// row-wise writes and the 8-rows-by-one-chunk reads of a quarter warp then fall on distinct banks).
+constexpr int kStageRow = 48;
+constexpr int kStageWarp = 32 * kStageRow;
+constexpr int kMaxEpiWarps = kEpiWarps + kExpWarps;     // with both operands expanded ahead the expander warps join
 
 struct GemmI8Plan {
     int TM;                 // 128-row sub-tiles per tile
@@ -43,7 +48,7 @@ struct GemmI8Plan {
     int64_t tiles_m, tiles_n, tiles;
     int grid;
     uint32_t tmem_cols;
-    uint32_t stage_bytes, off_stage, off_c, off_bar, off_misc;
+    uint32_t stage_bytes, off_stage, off_c, off_bar, off_misc, off_t;
     size_t smem_bytes;
 };
 
@@ -82,6 +87,7 @@ bool make_gemm_plan(int64_t M, int64_t N, int64_t K, GemmI8Plan& p, int sms)
     p.off_c = o;    o += (uint32_t)p.BN * 16;                  // float4 {p1, p2, p3, 0} per column
     p.off_bar = o;  o += (4 + 2 * kMaxStages) * 8;             // acc_full[2] acc_empty[2] full[] empty[]
     p.off_misc = o; o += 16;
+    p.off_t = o;    o += kMaxEpiWarps * kStageWarp;             // 16-byte aligned: every term above is
     o = (o + 127) / 128 * 128;
     p.off_stage = o;
     int ns = (int)((kSmemLimit - o) / p.stage_bytes);
@@ -92,46 +98,54 @@ bool make_gemm_plan(int64_t M, int64_t N, int64_t K, GemmI8Plan& p, int sms)
     return true;
 }
 
-// The weight operand expanded once: wexp[column tile][packed block of K][16-byte k chunk (8)][row of the
-// tile (BN)][16 B], the bytes the weight part of a ring stage holds.  Thread = (tile, block, row).
+// Operands expanded once: wexp[column tile][packed block of K][16-byte k chunk (8)][row of the tile (BN)][16 B]
+// and, when aexp is not null, aexp[row tile][block][chunk][row of the tile (128 TM)][16 B]: the bytes the weight
+// and the activation part of a ring stage hold.  Thread = (operand, tile, block, row).
 __global__ void __launch_bounds__(256)
-gemm_expand_weights_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, uint4* __restrict__ wexp)
+gemm_expand_operands_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, uint4* __restrict__ wexp,
+                            uint4* __restrict__ aexp)
 {
     tc::pdl_trigger();
     const int64_t nblk = (g.K + kBlockCodes - 1) / kBlockCodes;
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= p.tiles_n * nblk * p.BN) return;
-    const int r = (int)(i % p.BN);
-    const int64_t tk = i / p.BN, kb = tk % nblk, tn = tk / nblk;
-    const int64_t n = tn * p.BN + r;
+    const int64_t items_w = p.tiles_n * nblk * p.BN;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool isA = i >= items_w;
+    if (isA) i -= items_w;
+    const int R = isA ? p.TM * 128 : p.BN;                  // rows of a tile of this operand
+    if (isA && (aexp == nullptr || i >= p.tiles_m * nblk * R)) return;
+    const int r = (int)(i % R);
+    const int64_t tk = i / R, kb = tk % nblk, t = tk / nblk;
+    const int64_t row = t * R + r;
     uint4 nz = make_uint4(0, 0, 0, 0), sg = nz;
-    if (n < g.N) {
-        const uint4* src = reinterpret_cast<const uint4*>(g.w_packed + (n * nblk + kb) * kBlockBytes);
+    if (row < (isA ? g.M : g.N)) {
+        const uint4* src = reinterpret_cast<const uint4*>((isA ? g.a_packed : g.w_packed) + (row * nblk + kb) * kBlockBytes);
         nz = __ldg(src);
         sg = __ldg(src + 1);
     }
-    uint4* dst = wexp + tk * 8 * p.BN + r;
+    uint4* dst = (isA ? aexp : wexp) + tk * 8 * R + r;
     uint32_t o[8];
     tc::unpack32(nz.x, sg.x, o);
-    dst[0 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
-    dst[1 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+    dst[0 * R] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1 * R] = make_uint4(o[4], o[5], o[6], o[7]);
     tc::unpack32(nz.y, sg.y, o);
-    dst[2 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
-    dst[3 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+    dst[2 * R] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[3 * R] = make_uint4(o[4], o[5], o[6], o[7]);
     tc::unpack32(nz.z, sg.z, o);
-    dst[4 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
-    dst[5 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+    dst[4 * R] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[5 * R] = make_uint4(o[4], o[5], o[6], o[7]);
     tc::unpack32(nz.w, sg.w, o);
-    dst[6 * p.BN] = make_uint4(o[0], o[1], o[2], o[3]);
-    dst[7 * p.BN] = make_uint4(o[4], o[5], o[6], o[7]);
+    dst[6 * R] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[7 * R] = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
-// kPreW: the weight part of every stage comes from the scratch buffer gemm_expand_weights_kernel wrote (one
+// kPreW: the weight part of every stage comes from the scratch buffer gemm_expand_operands_kernel wrote (one
 // bulk asynchronous copy per stage, issued by a thread of warp 1), so the expander warps expand only the
-// activation rows: half of the integer work that paces the kernel.
-template <bool kPreW>
+// activation rows: half of the integer work that paces the kernel.  kPreA (only with kPreW): the activation
+// part too; the expander warps then have nothing to do and the ring is paced by the copies and the MMAs.
+template <bool kPreW, bool kPreA>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uint4* __restrict__ wexp)
+gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uint4* __restrict__ wexp,
+               const uint4* __restrict__ aexp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     float4* sC = reinterpret_cast<float4*>(smem + p.off_c);
@@ -149,8 +163,8 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
 
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
-        for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kEpiThreads); }
-        for (int i = 0; i < kMaxStages; ++i) { tc::mbar_init(&full[i], kExpWarps + (kPreW ? 1 : 0)); tc::mbar_init(&empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kPreA ? kMaxEpiWarps * 32 : kEpiThreads); }
+        for (int i = 0; i < kMaxStages; ++i) { tc::mbar_init(&full[i], kPreA ? 1 : kExpWarps + (kPreW ? 1 : 0)); tc::mbar_init(&empty[i], 1); }
         tc::mbar_init_fence();
         *dead = 0;
     }
@@ -160,8 +174,9 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
     const uint32_t tmem = *slot;
     if constexpr (kPreW) tc::pdl_wait();           // the expanded weights come from the kernel before
 
-    if (warp >= kExpWarp0) {
+    if (!kPreA && warp >= kExpWarp0) {
         // ------------------------------------------------------------ expanders
+        {
         const int tid = threadIdx.x - kExpWarp0 * 32;
         uint32_t count = 0;                                   // stages produced so far
         for (int64_t tile = blockIdx.x; tile < p.tiles; tile += gridDim.x) {
@@ -231,19 +246,24 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
                 if (lane == 0) tc::mbar_arrive(&full[s]);
             }
         }
+        }
     } else if (kPreW && warp == 1) {
         // ------------------------------------------------------------ weight stages from scratch (one thread)
         if (lane == 0) {
             const uint32_t w_bytes = (uint32_t)p.BN * 128u;
             const uint32_t w_off = (uint32_t)rowsA * 128u;            // the weight block follows the activation block
+            const uint32_t a_bytes = kPreA ? w_off : 0u;
             uint32_t count = 0;
             bool alive = true;
             for (int64_t tile = blockIdx.x; tile < p.tiles && alive; tile += gridDim.x) {
-                const int64_t tn = tile % p.tiles_n;
+                const int64_t tn = tile % p.tiles_n, tm = tile / p.tiles_n;
                 for (int64_t kb = 0; kb < nblk; ++kb, ++count) {
                     const uint32_t s = count % (uint32_t)p.stages;
                     if (!wait_or_die(&empty[s], ((count / (uint32_t)p.stages) & 1) ^ 1, g.status, dead)) { alive = false; break; }
-                    tc::mbar_arrive_expect_tx(&full[s], w_bytes);
+                    tc::mbar_arrive_expect_tx(&full[s], w_bytes + a_bytes);
+                    if constexpr (kPreA)
+                        tc::bulk_copy_g2s(tc::smem_addr(smem + p.off_stage + s * p.stage_bytes),
+                                          aexp + (tm * nblk + kb) * (a_bytes / 16), a_bytes, &full[s]);
                     tc::bulk_copy_g2s(tc::smem_addr(smem + p.off_stage + s * p.stage_bytes + w_off),
                                       wexp + (tn * nblk + kb) * (w_bytes / 16), w_bytes, &full[s]);
                 }
@@ -288,11 +308,17 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
                 if (alive) tc::mma_commit(&acc_full[acc]);
             }
         }
-    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
+    } else if (warp >= kEpiWarp0) {
         // ------------------------------------------------------------ epilogue
         //   out = a_s * (p1*S_xw + p2*S_x) + a_o * p3,  p1 = w_s, p2 = w_o, p3 = w_s*S_w + K*w_o
-        const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;
+        // (kPreA: all sixteen warps from kEpiWarp0 on; else the eight epilogue warps, the rest being expanders)
+        constexpr int nEpiThreads = kPreA ? kMaxEpiWarps * 32 : kEpiThreads;
+        constexpr int nParts = nEpiThreads / 128;              // column ranges; the four warps of a range take 32 rows each
+        const int q = warp & 3, part = (warp - kEpiWarp0) >> 2;
         const int etid = threadIdx.x - kEpiWarp0 * 32;
+        uint8_t* sT = smem + p.off_t + (warp - kEpiWarp0) * kStageWarp;
+        // whole-row float4 stores need every row start on a 16-byte boundary (the same for all lanes)
+        const bool vec_ok = g.dbg_acc == nullptr && (g.N & 3) == 0 && (((uintptr_t)g.out) & 15) == 0;
         uint32_t tc_ = 0;
         for (int64_t tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++tc_) {
             const int acc = p.nAcc == 2 ? (tc_ & 1) : 0;
@@ -300,8 +326,8 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
             const int64_t m0 = (tile / p.tiles_n) * rowsA, n0 = (tile % p.tiles_n) * p.BN;
             // per-column constants of this tile, in double, rounded once (the previous tile's readers
             // are past them: same warps, program order + barrier)
-            asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");
-            for (int j = etid; j < p.BN; j += kEpiThreads) {
+            asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(nEpiThreads) : "memory");
+            for (int j = etid; j < p.BN; j += nEpiThreads) {
                 const int64_t n = n0 + j;
                 float p1 = 0.f, p2 = 0.f, p3 = 0.f;
                 if (n < g.N) {
@@ -312,12 +338,12 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
                 }
                 sC[j] = make_float4(p1, p2, p3, 0.f);
             }
-            asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");
+            asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(nEpiThreads) : "memory");
             const bool alive = wait_or_die(&acc_full[acc], acc_ph, g.status, dead);
             tc::tc_fence_after_sync();
-            const int cols_half = p.BN / 2;                       // BN is a multiple of 16; halves of >= 8
-            const int c_begin = half == 0 ? 0 : (cols_half + 15) / 16 * 16;
-            const int c_end = half == 0 ? ((cols_half + 15) / 16 * 16 < p.BN ? (cols_half + 15) / 16 * 16 : p.BN) : p.BN;
+            const int per = ((p.BN + nParts - 1) / nParts + 15) / 16 * 16;     // columns per range, whole blocks of 16
+            const int c_begin = part * per < p.BN ? part * per : p.BN;
+            const int c_end = c_begin + per < p.BN ? c_begin + per : p.BN;
             for (int tm = 0; tm < p.TM; ++tm) {
                 const int64_t m = m0 + tm * 128 + q * 32 + lane;
                 const bool row_ok = alive && m < g.M;
@@ -328,24 +354,41 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
                     s_x = (float)g.a_sum[m];
                 }
                 const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((acc * p.TM + tm) * p.BN);
+                const int64_t mbase = m0 + tm * 128 + q * 32;
+                // write-out of a staged block: lane -> rows rr and rr + 16, 16-byte chunk ch
+                const int rr = (lane & 7) + 8 * (lane >> 4), ch = (lane >> 3) & 1;
                 for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                     uint32_t v[16];
                     tc::tmem_ld16(trow + (uint32_t)c0, v);
                     tc::tmem_ld_wait();
-                    if (!row_ok) continue;
-                    float* orow = g.out + m * g.N + n0 + c0;
-                    if (n0 + c0 + 16 <= g.N && g.dbg_acc == nullptr && (((uintptr_t)orow) & 15) == 0) {
+                    if (vec_ok && n0 + c0 + 16 <= g.N) {
+                        // A lane holds 16 columns of ONE row; stored as is, a warp store would touch 32 rows
+                        // with 16 bytes each.  Through the staging block (8 columns at a time) a store covers
+                        // 16 rows x 32 bytes: whole sectors.
                         #pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            float r[4];
+                        for (int h = 0; h < 16; h += 8) {
                             #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float4 c = sC[c0 + j + e];
-                                r[e] = fmaf(a_s, fmaf(c.x, (float)(int)v[j + e], c.y * s_x), a_o * c.z);
+                            for (int j = 0; j < 8; j += 4) {
+                                float r[4];
+                                #pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float4 c = sC[c0 + h + j + e];
+                                    r[e] = fmaf(a_s, fmaf(c.x, (float)(int)v[h + j + e], c.y * s_x), a_o * c.z);
+                                }
+                                *reinterpret_cast<float4*>(sT + lane * kStageRow + j * 4) = make_float4(r[0], r[1], r[2], r[3]);
                             }
-                            *reinterpret_cast<float4*>(orow + j) = make_float4(r[0], r[1], r[2], r[3]);
+                            __syncwarp();
+                            #pragma unroll
+                            for (int i = 0; i < 32; i += 16) {
+                                const float4 t = *reinterpret_cast<const float4*>(sT + (rr + i) * kStageRow + ch * 16);
+                                const int64_t mt = mbase + rr + i;
+                                if (alive && mt < g.M)
+                                    *reinterpret_cast<float4*>(g.out + mt * g.N + n0 + c0 + h + ch * 4) = t;
+                            }
+                            __syncwarp();
                         }
-                    } else {
+                    } else if (row_ok) {
+                        float* orow = g.out + m * g.N + n0 + c0;
                         #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             if (n0 + c0 + j >= g.N) continue;
@@ -374,6 +417,18 @@ int sm_count_g()
     return sms;
 }
 
+// Pre-expansion mode of a plan: 0 = both operands expanded inside the kernel (one row tile: every weight row
+// is expanded once anyway), 1 = weights expanded ahead (several row tiles, one column tile), 2 = both ahead
+// (several tiles each way: every row of either operand would be expanded once per tile it takes part in).
+int gemm_pre_mode(const GemmI8Plan& p, int64_t K)
+{
+    const int64_t nblk = (K + kBlockCodes - 1) / kBlockCodes;
+    const size_t wbytes = (size_t)p.tiles_n * nblk * p.BN * 128, abytes = (size_t)p.tiles_m * nblk * p.TM * 128 * 128;
+    if (p.tiles_m < 2 || wbytes > (size_t(1) << 31)) return 0;
+    if (p.tiles_n < 2 || wbytes + abytes > (size_t(1) << 31)) return 1;
+    return 2;
+}
+
 }  // namespace
 
 bool gemm_i8_supported(int64_t M, int64_t N, int64_t K)
@@ -386,34 +441,41 @@ int gemm_i8_launches(int64_t M, int64_t N, int64_t K)
 {
     GemmI8Plan p;
     if (!make_gemm_plan(M, N, K, p, 148)) return 0;
-    return p.tiles_m < 2 ? 1 : 2;
+    return gemm_pre_mode(p, K) == 0 ? 1 : 2;
 }
 
 cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s)
 {
     GemmI8Plan p;
     if (!make_gemm_plan(g.M, g.N, g.K, p, sm_count_g())) return cudaErrorInvalidConfiguration;
-    // Every tile of a column re-expands that column's weights: with two or more row tiles the weights are
-    // expanded once into scratch instead (stream-ordered allocation, N rounded up to tiles x K bytes).
-    const int64_t nblk = (g.K + kBlockCodes - 1) / kBlockCodes;
-    const size_t wbytes = (size_t)p.tiles_n * nblk * p.BN * 128;
-    if (p.tiles_m < 2 || wbytes > (size_t(1) << 31)) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    const int mode = gemm_pre_mode(p, g.K);
+    if (mode == 0) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
         if (e != cudaSuccess) return e;
-        gemm_i8_kernel<false><<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(g, p, nullptr);
+        gemm_i8_kernel<false, false><<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(g, p, nullptr, nullptr);
         return cudaGetLastError();
     }
+    // scratch from the stream-ordered allocator: N (and M) rounded up to tiles, times K rounded up to blocks, bytes
+    const int64_t nblk = (g.K + kBlockCodes - 1) / kBlockCodes;
+    const int64_t items_w = p.tiles_n * nblk * p.BN, items_a = mode == 2 ? p.tiles_m * nblk * p.TM * 128 : 0;
     void* scratch = nullptr;
-    cudaError_t e = cudaMallocAsync(&scratch, wbytes, s);
+    cudaError_t e = cudaMallocAsync(&scratch, (size_t)(items_w + items_a) * 128, s);
     if (e != cudaSuccess) return e;
-    const int64_t items = p.tiles_n * nblk * p.BN;
-    gemm_expand_weights_kernel<<<(unsigned)((items + 255) / 256), 256, 0, s>>>(g, p, reinterpret_cast<uint4*>(scratch));
+    uint4* wexp = reinterpret_cast<uint4*>(scratch);
+    uint4* aexp = mode == 2 ? wexp + items_w * 8 : nullptr;
+    gemm_expand_operands_kernel<<<(unsigned)((items_w + items_a + 255) / 256), 256, 0, s>>>(g, p, wexp, aexp);
     e = cudaGetLastError();
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
-    if (e == cudaSuccess)
-        e = launch_pdl(gemm_i8_kernel<true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, g, p,
-                       (const uint4*)scratch);
+    if (e == cudaSuccess && mode == 1) {
+        e = cudaFuncSetAttribute(gemm_i8_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+        if (e == cudaSuccess)
+            e = launch_pdl(gemm_i8_kernel<true, false>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, g, p,
+                           (const uint4*)wexp, (const uint4*)aexp);
+    } else if (e == cudaSuccess) {
+        e = cudaFuncSetAttribute(gemm_i8_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+        if (e == cudaSuccess)
+            e = launch_pdl(gemm_i8_kernel<true, true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, g, p,
+                           (const uint4*)wexp, (const uint4*)aexp);
+    }
     const cudaError_t e2 = cudaFreeAsync(scratch, s);
     return e != cudaSuccess ? e : e2;
 }

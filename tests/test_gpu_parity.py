@@ -244,7 +244,7 @@ def test_conv_thresholds_out_of_order(variant):
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
-@pytest.mark.parametrize("shape", [(256, 512, 4096), (384, 272, 1152), (130, 520, 260)], ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("shape", [(256, 512, 4096), (384, 272, 1152), (130, 520, 260), (515, 300, 1001), (300, 302, 200)], ids=lambda s: "x".join(map(str, s)))
 def test_gemm_multi_tile_shapes(shape, variant):
     M, N, K = shape
     case = inputs.gemm_case(f"gemm_{M}x{N}x{K}", M, N, K, seed=M + K, p_zero=0.3, act="uniform3",
