@@ -127,6 +127,57 @@ def roofline_of(workload, kernel_bytes, kernel_ops, kernel_ms):
             "traffic": traffic, "peak_source": src, "ops_per_launch": kernel_ops, "kernel_ms": kernel_ms}
 
 
+def time_e2e(torch, step, xs, host_in, host_out, n_sets, n_steps, barrier):
+    """Milliseconds per step of: pinned host input -> device, step(j) (the C-ABI calls), result -> pinned host.
+
+    Consecutive steps overlap as a caller with a queue of batches would run them: the upload of step i + 1, the
+    kernels of step i and the download of step i - 1 on three streams (the two copy directions use different
+    engines), each buffer set guarded by events.  With one buffer set the steps run back to back.  Returns
+    (ms per step, whether steps overlapped)."""
+    pipelined = n_sets >= 2
+    host_outs = [host_out, torch.empty_like(host_out).pin_memory()] if pipelined else [host_out]
+    main = torch.cuda.current_stream()
+    s_in, s_c, s_out = (torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()) if pipelined else (main, main, main)
+    ev_in = [torch.cuda.Event() for _ in range(n_sets)]
+    ev_c = [torch.cuda.Event() for _ in range(n_sets)]
+    ev_out = [torch.cuda.Event() for _ in range(n_sets)]
+
+    def run(n):
+        for st in (s_in, s_c, s_out):
+            if st is not main:
+                st.wait_stream(main)
+        for i in range(n):
+            j = i % n_sets
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_c[j])                 # the step that last read xs[j] is done
+                xs[j].copy_(host_in, non_blocking=True)
+                ev_in[j].record(s_in)
+            with torch.cuda.stream(s_c):
+                s_c.wait_event(ev_in[j])
+                s_c.wait_event(ev_out[j])                # the download that last read this set's output is done
+                res = step(j)
+                ev_c[j].record(s_c)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_c[j])
+                host_outs[i % len(host_outs)].copy_(res, non_blocking=True)
+                ev_out[j].record(s_out)
+        for st in (s_in, s_c, s_out):
+            if st is not main:
+                main.wait_stream(st)
+
+    run(2)
+    barrier()
+    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_begin.record()
+    run(n_steps)
+    e_end.record()
+    barrier()
+    return e_begin.elapsed_time(e_end) / n_steps, pipelined
+
+
+E2E_OVERLAP = "upload, kernels and download of consecutive steps on three streams"
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -417,20 +468,7 @@ def run_body(args, case, name):
     barrier()
     if rtn.rtn_last_device_status() != 0:
         raise RuntimeError("device status after the timed region")
-    e2e_steps = max(3, min(steps, 10))
-    for i in range(2):
-        xs[0].copy_(host_in, non_blocking=True)
-        host_out.copy_(step(0), non_blocking=True)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(e2e_steps):
-        j = i % n_sets
-        xs[j].copy_(host_in, non_blocking=True)
-        host_out.copy_(step(j), non_blocking=True)
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    e2e_ms, pipelined = time_e2e(torch, step, xs, host_in, host_out, n_sets, max(3, min(steps, 20)), barrier)
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, "cuda")
     ms_per_step = total_ms / steps
     ops = bodies[0].ops()
@@ -451,7 +489,8 @@ def run_body(args, case, name):
                        "parallelism": "replicas only" if world > 1 else "1 GPU"},
             "clocks": clocks,
             "e2e": {"value": whole_job_tops(ops, world, e2e_ms), "unit": "TOPS", "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": int(host_in.numel() * 4), "d2h_bytes_per_step": int(host_out.numel() * 4)},
+                    "h2d_bytes_per_step": int(host_in.numel() * 4), "d2h_bytes_per_step": int(host_out.numel() * 4),
+                    "overlap": E2E_OVERLAP if pipelined else "none: one buffer set"},
             "gpu_launches": launches * steps,
             "roofline": roofline_of(name, bodies[0].algorithmic_bytes(), ops, ms_per_step),
         }
@@ -757,50 +796,8 @@ def run_ours(args, case, name):
         gemm_kernel_ms = k0.elapsed_time(k1) / reps
         gemm_kernel_bytes = (M + N) * ((K + 127) // 128) * 32 + 4 * M * N
 
-    # ---- end to end: pinned host input -> device, the C-ABI call(s), result -> pinned host, every step.
-    # Consecutive steps overlap as a caller with a queue of batches would run them: the upload of step i + 1,
-    # the kernels of step i and the download of step i - 1 on three streams (the two copy directions use
-    # different engines), each buffer guarded by events.  With one buffer set the steps run back to back.
-    e2e_steps = max(3, min(args.steps, 40))
-    pipelined = n_sets >= 2
-    host_outs = [host_out, torch.empty_like(host_out).pin_memory()] if pipelined else [host_out]
-    main = torch.cuda.current_stream()
-    s_in, s_c, s_out = (torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()) if pipelined else (main, main, main)
-    ev_in = [torch.cuda.Event() for _ in range(n_sets)]
-    ev_c = [torch.cuda.Event() for _ in range(n_sets)]
-    ev_out = [torch.cuda.Event() for _ in range(n_sets)]
-
-    def e2e_run(n):
-        for st in (s_in, s_c, s_out):
-            if st is not main:
-                st.wait_stream(main)
-        for i in range(n):
-            j = i % n_sets
-            with torch.cuda.stream(s_in):
-                s_in.wait_event(ev_c[j])                 # the step that last read xs[j] is done
-                xs[j].copy_(host_in, non_blocking=True)
-                ev_in[j].record(s_in)
-            with torch.cuda.stream(s_c):
-                s_c.wait_event(ev_in[j])
-                s_c.wait_event(ev_out[j])                # the download that last read outs[j] is done
-                res = step(j)
-                ev_c[j].record(s_c)
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(ev_c[j])
-                host_outs[i % len(host_outs)].copy_(res, non_blocking=True)
-                ev_out[j].record(s_out)
-        for st in (s_in, s_c, s_out):
-            if st is not main:
-                main.wait_stream(st)
-
-    e2e_run(2)
-    barrier()
-    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e_begin.record()
-    e2e_run(e2e_steps)
-    e_end.record()
-    barrier()
-    e2e_ms = e_begin.elapsed_time(e_end) / e2e_steps
+    # ---- end to end: pinned host input -> device, the C-ABI call(s), result -> pinned host, every step
+    e2e_ms, pipelined = time_e2e(torch, step, xs, host_in, host_out, n_sets, max(3, min(args.steps, 40)), barrier)
 
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, "cuda")
     ms_per_step = total_ms / args.steps
@@ -831,8 +828,7 @@ def run_ours(args, case, name):
             "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": int(host_in.numel() * host_in.element_size()),
                     "d2h_bytes_per_step": int(host_out.numel() * host_out.element_size()),
-                    "overlap": ("upload, kernels and download of consecutive steps on three streams" if pipelined
-                                else "none: one buffer set")},
+                    "overlap": E2E_OVERLAP if pipelined else "none: one buffer set"},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline_of(name if not packed_io else name + "/packed", kernel_bytes, ops, kernel_ms),
         }
