@@ -77,3 +77,12 @@ def test_k_slices_only_for_small_outputs_with_a_long_k():
     assert rtn.rtn_gemm_k_slices(16, 256, 9216) > 1
     assert rtn.rtn_gemm_k_slices(64, 4096, 9216) == 1         # enough output tiles without slicing
     assert rtn.rtn_gemm_k_slices(0, 4, 4) == 0
+
+
+def test_gemm_kernel_launches_follow_the_operand_expansion():
+    assert rtn.rtn_gemm_kernel_launches(0, 4, 4) == 0
+    assert rtn.rtn_gemm_kernel_launches(64, 64, 576) == 1         # bit-plane kernel, one launch
+    assert rtn.rtn_gemm_kernel_launches(16, 256, 9216) == 2       # K in slices: contraction + epilogue in place
+    if rtn.rtn_choose_gemm_variant(4096, 4096, 4096) == rtn.VARIANT_I8:
+        assert rtn.rtn_gemm_kernel_launches(4096, 4096, 4096) == 2    # operands expanded ahead, then the contraction
+        assert rtn.rtn_gemm_kernel_launches(128, 4096, 4096) == 1     # one row tile: everything inside the kernel
