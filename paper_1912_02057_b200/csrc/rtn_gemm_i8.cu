@@ -10,7 +10,11 @@
 //                 expansion, 16-byte shared stores) into a ring of stages, then fences and arrives
 //   warp  0       one thread waits for a stage, issues its 4*TM MMAs (K = 32 each) and commits them
 //                 to the stage's "empty" barrier; after the last block it commits the accumulators
-//   warps 4..11   epilogue: tcgen05.ld, out = a_s (w_s S_xw + w_o S_x) + a_o (w_s S_w + K w_o)
+//   warps 4..11   epilogue: tcgen05.ld, out = a_s (w_s S_xw + w_o S_x) + a_o (w_s S_w + K w_o), transposed
+//                 through a small staging block so that a warp store covers whole sectors of 16 rows
+//   warp  1       (operands expanded ahead of the kernel, see gemm_pre_mode) one thread fills the weight part of
+//                 every stage, or both parts, with bulk asynchronous copies from the scratch buffer
+//                 gemm_expand_operands_kernel wrote; with both parts copied the expander warps join the epilogue
 // Operand stages are K-major without swizzle: [16-byte k chunk][row][16 B]; an 8-row core matrix is
 // 128 contiguous bytes and consecutive threads (rows) store consecutive 16-byte slots.
 #include "rtn_internal.cuh"
