@@ -227,6 +227,82 @@ ternarize_pack_vec_kernel(const float* __restrict__ a, int64_t M, int64_t K,
     }
 }
 
+// Short rows of 32, 64, 128 or 256 values (the channel counts of pixel rows): a row would leave most of a warp's
+// lanes of the kernel above without work, so here the matrix is walked as one flat array, 256 values per warp and
+// unit; 256 / K rows share a unit, lane l holds eight values of row (8 l) / K, a quad still holds one plane word,
+// and the row's code sum is added up over its K / 8 lanes.  The quad's first lane stores the two words (and, for
+// K < 128, the first quad of a row the block's unused words as zeros).  Two units per trip.
+template <bool kPerK>
+__global__ void __launch_bounds__(256, 4)
+ternarize_pack_rows_kernel(const float* __restrict__ a, int64_t M, int K,
+                           const float* __restrict__ t_lo, const float* __restrict__ t_hi,
+                           uint8_t* __restrict__ packed, int32_t* __restrict__ a_sum)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t total = M * K, nunits = (total + 255) / 256;
+    const int lanes_per_row = K / 8, words = K / 32, nblk = (K + kBlockCodes - 1) / kBlockCodes;
+    const float lo0 = t_lo[0], hi0 = t_hi[0];
+
+    for (int64_t u0 = warp * 2; u0 < nunits; u0 += nwarps * 2) {
+        float4 x[2][2];
+        #pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int64_t flat = (u0 + u) * 256 + 8 * lane;
+            const bool in = flat < total;                        // total is a multiple of 32
+            x[u][0] = in ? __ldg(reinterpret_cast<const float4*>(a + flat)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x[u][1] = in ? __ldg(reinterpret_cast<const float4*>(a + flat) + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        #pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int64_t flat = (u0 + u) * 256 + 8 * lane;
+            const bool in = flat < total;
+            const int64_t m = flat / K;
+            const int col = (int)(flat - m * K);
+            const float v[8] = {x[u][0].x, x[u][0].y, x[u][0].z, x[u][0].w, x[u][1].x, x[u][1].y, x[u][1].z, x[u][1].w};
+            float lo[8], hi[8];
+            if (kPerK && in) {
+                const float4 l0 = __ldg(reinterpret_cast<const float4*>(t_lo + col)), l1 = __ldg(reinterpret_cast<const float4*>(t_lo + col) + 1);
+                const float4 h0 = __ldg(reinterpret_cast<const float4*>(t_hi + col)), h1 = __ldg(reinterpret_cast<const float4*>(t_hi + col) + 1);
+                lo[0] = l0.x; lo[1] = l0.y; lo[2] = l0.z; lo[3] = l0.w; lo[4] = l1.x; lo[5] = l1.y; lo[6] = l1.z; lo[7] = l1.w;
+                hi[0] = h0.x; hi[1] = h0.y; hi[2] = h0.z; hi[3] = h0.w; hi[4] = h1.x; hi[5] = h1.y; hi[6] = h1.z; hi[7] = h1.w;
+            } else {
+                #pragma unroll
+                for (int t = 0; t < 8; ++t) { lo[t] = lo0; hi[t] = hi0; }
+            }
+            uint32_t nzb = 0, posb = 0;
+            if (in) {
+                #pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    bool nz, pos;
+                    ternarize(v[t], lo[t], hi[t], nz, pos);
+                    nzb |= nz ? (1u << t) : 0u;
+                    posb |= pos ? (1u << t) : 0u;
+                }
+            }
+            int sum = __popc(posb) - __popc(nzb & ~posb);
+            uint32_t xn = nzb << (8 * (lane & 3)), xp = posb << (8 * (lane & 3));
+            xn |= __shfl_xor_sync(0xffffffffu, xn, 1);
+            xp |= __shfl_xor_sync(0xffffffffu, xp, 1);
+            xn |= __shfl_xor_sync(0xffffffffu, xn, 2);
+            xp |= __shfl_xor_sync(0xffffffffu, xp, 2);
+            for (int d = 1; d < lanes_per_row; d <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+            if (in) {
+                uint32_t* dst = reinterpret_cast<uint32_t*>(packed + m * nblk * kBlockBytes);
+                const int wj = col >> 5;                            // the word of the row this quad holds
+                if ((lane & 3) == 0) {
+                    dst[(wj >> 2) * 8 + (wj & 3)] = xn;
+                    dst[(wj >> 2) * 8 + 4 + (wj & 3)] = xp;
+                    if (wj == 0)
+                        for (int z = words; z < 4; ++z) { dst[z] = 0u; dst[4 + z] = 0u; }
+                }
+                if (a_sum != nullptr && col == 0) a_sum[m] = sum;
+            }
+        }
+    }
+}
+
 cudaError_t launch_ternarize_pack(const float* a, int64_t M, int64_t K, const float* t_lo,
                                   const float* t_hi, int64_t n_thr, uint8_t* packed, int32_t* a_sum,
                                   cudaStream_t s)
@@ -240,6 +316,16 @@ cudaError_t launch_ternarize_pack(const float* a, int64_t M, int64_t K, const fl
     const bool per_k = n_thr != 1;
     const bool vec = (K % 8) == 0 && (reinterpret_cast<uintptr_t>(a) & 15) == 0 &&
                      (!per_k || ((reinterpret_cast<uintptr_t>(t_lo) | reinterpret_cast<uintptr_t>(t_hi)) & 15) == 0);
+    if (vec && (K == 32 || K == 64 || K == 128 || K == 256)) {
+        const int64_t units = (M * K + 255) / 256, warps = (units + 1) / 2;
+        int64_t blk = (warps + 7) / 8;
+        if (blk > 148 * 16) blk = 148 * 16;
+        if (!per_k)
+            ternarize_pack_rows_kernel<false><<<(unsigned)blk, threads, 0, s>>>(a, M, (int)K, t_lo, t_hi, packed, a_sum);
+        else
+            ternarize_pack_rows_kernel<true><<<(unsigned)blk, threads, 0, s>>>(a, M, (int)K, t_lo, t_hi, packed, a_sum);
+        return cudaGetLastError();
+    }
     if (vec && !per_k)
         ternarize_pack_vec_kernel<false><<<(unsigned)blocks, threads, 0, s>>>(a, M, K, t_lo, t_hi, packed, a_sum, wpr);
     else if (vec)

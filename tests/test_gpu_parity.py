@@ -30,7 +30,10 @@ def run_or_skip_unsupported(fn, variant):
                                        (64, 576, False), (33, 1000, True), (300, 4097, False),
                                        # rows of a multiple of 8 values take the vector kernel; teams of 1..8 warps
                                        (5, 8, False), (5, 136, True), (21, 1000, False), (19, 2056, True),
-                                       (11, 4096, False), (3, 9216, True), (2, 9224, False)])
+                                       (11, 4096, False), (3, 9216, True), (2, 9224, False),
+                                       # pixel rows of 32..256 channels: several rows share a warp
+                                       (5, 32, False), (7, 64, True), (1001, 64, False), (3, 128, True), (9, 256, False),
+                                       (33, 256, True), (1, 32, True)])
 def test_ternarize_pack_act(M, K, per_k):
     case = inputs.gemm_case("pack", M, 2, K, seed=M * 1000 + K, p_zero=0.4, thresholds=(0.3, 1.0),
                             per_k_thresholds=per_k)
