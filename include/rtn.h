@@ -55,8 +55,8 @@ typedef enum {
     RTN_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait gave up (see last_device_status) */
 } rtn_status;
 
-/* Treatment of filter taps that fall outside the image.  The paper never mentions padding; it
- * calls the Eq. 10 constant C "a constant which can be pre-stored", which holds only for
+/* Treatment of filter taps that fall outside the image.  The paper never mentions padding; the
+ * constant term C of Eq. 10 can be stored ahead of time, as the paper has it, only under
  * RTN_PAD_CODE_ZERO: an outside tap has CODE 0, i.e. real value a_offset, and S_w and K cover
  * all C*kh*kw taps.  RTN_PAD_VALUE_ZERO makes an outside tap contribute nothing (what a
  * floating-point conv2d on the de-quantised tensor does): S_w and K then cover inside taps only. */
@@ -142,8 +142,8 @@ rtn_status rtn_ternary_conv2d(const float* x, int64_t B, int64_t C, int64_t H, i
 /* Variant of rtn_ternary_conv2d that allocates nothing (the paper has no counterpart; it is for
  * callers that must not touch an allocator on the hot path).  It always takes the two-kernel
  * tensor-core path (int8 codes of the input in a scratch buffer, filter bank split over CTAs),
- * the path rtn_ternary_conv2d chooses for layers with more than 256 filters and for strided 3x3
- * layers, and gives the same bits.  The scratch is one array of 16 MiB per device, part of the library's image; the
+ * the path rtn_ternary_conv2d chooses for strided 3x3 layers and, by its cost estimate, for some 1x1
+ * stride-2 layers and wide layers at large batch, and gives the same bits.  The scratch is one array of 16 MiB per device, part of the library's image; the
  * call performs no cudaMalloc, cudaMallocAsync, cudaFree or other allocating routine.
  *   - RTN_ERR_UNSUPPORTED: a shape the path does not take (e.g. 3x3 with stride 3), or a layer whose codes
  *     (about B*(H+2pad)*(W+2pad)*(C rounded up to 32) bytes) exceed the array.
@@ -180,10 +180,12 @@ rtn_status rtn_ternary_conv2d_noalloc(const float* x, int64_t B, int64_t C, int6
  *               the row; canonical zeros, zero fill past N.  This is the x_packed of
  *               rtn_ternary_conv2d_packed.
  *   dbg_acc     NULL, or int32 [B][N][Ho][Wo] raw S_xw
- * At least one of out, out_packed must be given.  Takes the two-kernel tensor-core path (int8 codes in
- * a scratch buffer from the stream-ordered allocator); RTN_ERR_UNSUPPORTED for shapes that path does
- * not take (see rtn_ternary_conv2d_noalloc).  Stream-order rule as for rtn_ternary_conv2d; the
- * next-layer thresholds count as parameters of the layer. */
+ * At least one of out, out_packed must be given.  Runs on the tensor cores only: the one-kernel variant with
+ * the filters resident in shared memory where they fit (stride 1), else the streamed-filter variant or the
+ * two-kernel variant with int8 codes in a scratch buffer from the stream-ordered allocator
+ * (rtn_conv_next_kernel_launches says how many launches a shape takes); RTN_ERR_UNSUPPORTED for shapes none of
+ * the three takes (e.g. 3x3 with stride 3).  Stream-order rule as for rtn_ternary_conv2d; the next-layer
+ * thresholds count as parameters of the layer. */
 rtn_status rtn_ternary_conv2d_fused(const float* x, int64_t B, int64_t C, int64_t H, int64_t W,
                                     const float* t_lo, const float* t_hi, int64_t n_thr,
                                     const void* w_packed, const int32_t* w_sum,
@@ -224,8 +226,8 @@ rtn_status rtn_quaternary_gemm(const void* a_packed, const void* w_packed, int64
 /* The variant RTN_VARIANT_AUTO resolves to for a shape (never AUTO). */
 rtn_variant rtn_choose_gemm_variant(int64_t M, int64_t N, int64_t K);
 /* Slices of K that RTN_VARIANT_AUTO cuts a GEMM shape into (1 = none).  A linear layer with few rows and
- * columns and a long K (the paper's "both convolution and linear layers", section "Efficient Computation
- * Pattern") has too few output tiles to fill the GPU: the bit-plane kernel then works on slices of K in
+ * columns and a long K (linear layers are covered by the pattern of section "Efficient Computation
+ * Pattern" as much as convolutions) has too few output tiles to fill the GPU: the bit-plane kernel then works on slices of K in
  * parallel, adds their exact integer parts into the output buffer and applies the affine form in place
  * (3 launches instead of 1; the integers do not depend on the order of the additions). */
 int64_t rtn_gemm_k_slices(int64_t M, int64_t N, int64_t K);
@@ -251,6 +253,13 @@ int64_t rtn_conv_next_kernel_launches(int64_t B, int64_t C, int64_t H, int64_t W
  * RTN_OK, or RTN_ERR_DEVICE_TIMEOUT if a kernel's bounded wait (on an mbarrier of the
  * tensor-core pipeline) ran out since the last call; that kernel's output is then invalid. */
 rtn_status rtn_last_device_status(void* stream);
+
+/* Self-test of the bounded waits (the safety net behind RTN_ERR_DEVICE_TIMEOUT): launches one small kernel
+ * whose single waiting thread polls, `polls` times (1..4096, each poll parks the thread for up to about 2 us),
+ * an mbarrier that nothing arrives on, with the same wait routine the tensor-core kernels use.  The wait must
+ * give up: *gave_up (device int32) receives 1, and the next rtn_last_device_status returns
+ * RTN_ERR_DEVICE_TIMEOUT once.  Nothing traps or spins without limit; the context stays usable.  Only enqueues. */
+rtn_status rtn_selftest_wait_timeout(int64_t polls, int32_t* gave_up, void* stream);
 
 /* Static text for a status code. */
 const char* rtn_status_string(rtn_status s);

@@ -341,3 +341,12 @@ def within_tolerance(got, ref, mag):
     """Elementwise: |err| <= 1e-5 |ref|  or  |err| <= 1e-6 max(1, sum |term_i|)."""
     err = np.abs(np.asarray(got, np.float64) - ref)
     return (err <= REL_TOL * np.abs(ref)) | (err <= ABS_TOL * np.maximum(1.0, mag))
+
+
+def strict_miss(got, ref):
+    """How far the outputs are from the rule without the sum-of-terms relaxation: (count, largest |err|) over the
+    outputs with |err| > 1e-5 |ref| and |err| > 1e-6.  Reported next to the tolerance verdict, never a verdict."""
+    ref = np.asarray(ref, np.float64)
+    err = np.abs(np.asarray(got, np.float64) - ref)
+    miss = (err > REL_TOL * np.abs(ref)) & (err > ABS_TOL)
+    return int(miss.sum()), float(err[miss].max()) if miss.any() else 0.0

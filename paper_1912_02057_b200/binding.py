@@ -95,6 +95,8 @@ def lib():
         L.rtn_conv_next_kernel_launches.argtypes = [_i64] * 9
         L.rtn_last_device_status.restype = _int
         L.rtn_last_device_status.argtypes = [_vp]
+        L.rtn_selftest_wait_timeout.restype = _int
+        L.rtn_selftest_wait_timeout.argtypes = [_i64, _vp, _vp]
         L.rtn_status_string.restype = C.c_char_p
         L.rtn_status_string.argtypes = [_int]
         _lib = L
@@ -301,3 +303,12 @@ def rtn_conv_next_kernel_launches(B, Cin, H, W, N, kh, kw, stride, pad):
 
 def rtn_last_device_status(stream=None):
     return int(lib().rtn_last_device_status(_stream(stream)))
+
+
+def rtn_selftest_wait_timeout(polls=1024, stream=None):
+    """Runs the library's bounded wait on an mbarrier nothing arrives on.  Returns the device int32 tensor that
+    receives 1 when the wait gave up; the next rtn_last_device_status then reports RTN_ERR_DEVICE_TIMEOUT once."""
+    gave_up = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    _check(lib().rtn_selftest_wait_timeout(int(polls), _ptr(gave_up, torch.int32), _stream(stream)),
+           "rtn_selftest_wait_timeout")
+    return gave_up

@@ -52,10 +52,12 @@ class Body:
         return (d["wp"], d["ws"], l.cout, l.k, l.k, l.stride, l.pad, self.pad_mode, l.a_scale, l.a_offset,
                 d["w_s"], d["w_o"])
 
-    def forward(self, s):
+    def forward(self, s, dbg=None):
         """s: fp32 [B, 64, H, H] (the stem's output).  Returns (final residual stream fp32, per-block
         packed rows p_next) -- the last block's p_next uses its own conv1 thresholds as a stand-in for
-        the classifier's (full-precision) input and is not consumed."""
+        the classifier's (full-precision) input and is not consumed.  dbg: optional dict, layer name ->
+        int32 tensor of the layer's output shape that receives the raw S_xw (the entry points' dbg_acc)."""
+        acc = (lambda l: None) if dbg is None else (lambda l: dbg.get(l.name))
         p = None
         for i, blk in enumerate(self.blocks):
             c1, c2, down, e = blk["conv1"], blk["conv2"], blk["down"], self.bufs[i]
@@ -63,20 +65,23 @@ class Body:
             if p is None:       # the body's first layer ternarizes the fp32 stream itself
                 d1 = self.d[c1.name]
                 rtn.rtn_ternary_conv2d_fused(s, d1["t_lo"], d1["t_hi"], *self._args(c1), relu=True,
-                                             next_t_lo=n2["t_lo"], next_t_hi=n2["t_hi"], out_packed=e["q"])
+                                             next_t_lo=n2["t_lo"], next_t_hi=n2["t_hi"], out_packed=e["q"],
+                                             dbg_acc=acc(c1))
             else:
                 rtn.rtn_ternary_conv2d_packed(p, self.B, c1.cin, c1.hin, c1.hin, *self._args(c1), relu=True,
-                                              next_t_lo=n2["t_lo"], next_t_hi=n2["t_hi"], out_packed=e["q"])
+                                              next_t_lo=n2["t_lo"], next_t_hi=n2["t_hi"], out_packed=e["q"],
+                                              dbg_acc=acc(c1))
             skip = s
             if down is not None:
                 dd = self.d[down.name]
-                rtn.rtn_ternary_conv2d_fused(s, dd["t_lo"], dd["t_hi"], *self._args(down), relu=True, out=e["skip"])
+                rtn.rtn_ternary_conv2d_fused(s, dd["t_lo"], dd["t_hi"], *self._args(down), relu=True, out=e["skip"],
+                                             dbg_acc=acc(down))
                 skip = e["skip"]
             nxt = self.blocks[i + 1]["conv1"] if i + 1 < len(self.blocks) else c1
             nn = self.d[nxt.name]
             rtn.rtn_ternary_conv2d_packed(e["q"], self.B, c2.cin, c2.hin, c2.hin, *self._args(c2), relu=True,
                                           skip=skip, out=e["s_next"], next_t_lo=nn["t_lo"], next_t_hi=nn["t_hi"],
-                                          out_packed=e["p_next"])
+                                          out_packed=e["p_next"], dbg_acc=acc(c2))
             s, p = e["s_next"], e["p_next"]
         return s, [e["p_next"] for e in self.bufs]
 

@@ -1,5 +1,6 @@
 // C ABI of librtn_b200 (declared in rtn.h): argument checks, variant choice, launches.
 #include "rtn_internal.cuh"
+#include "rtn_tcgen05.cuh"
 
 #include <limits.h>
 
@@ -23,6 +24,20 @@ unsigned* status_word()
         g_status_ptr[dev] = static_cast<unsigned*>(p);
     }
     return g_status_ptr[dev];
+}
+
+// Self-test of the give-up path of the bounded waits: one thread waits, with the library's wait routine and a
+// caller-chosen number of polls, on an mbarrier that nothing ever arrives on.  The wait must come back false
+// and leave the time-out bit in the status word; `result` receives 1 if it did, 0 if the wait claimed success.
+__global__ void selftest_wait_kernel(unsigned* status, uint32_t polls, int* result)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        rtn::tc::mbar_init(&bar, 1);
+        rtn::tc::mbar_init_fence();
+        const bool completed = rtn::tc::mbar_wait(&bar, 0, status, polls);
+        *result = completed ? 0 : 1;
+    }
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -406,6 +421,17 @@ rtn_status rtn_quaternary_gemm(const void* a_packed, const void* w_packed, int64
                                                       static_cast<const uint8_t*>(w_packed), M, N, K, out,
                                                       static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
+rtn_status rtn_selftest_wait_timeout(int64_t polls, int32_t* gave_up, void* stream)
+{
+    if (gave_up == nullptr) return RTN_ERR_NULL;
+    if (polls < 1 || polls > 4096) return RTN_ERR_SHAPE;
+    if (!aligned4(gave_up)) return RTN_ERR_ALIGN;
+    unsigned* st = status_word();
+    if (st == nullptr) return RTN_ERR_CUDA;
+    selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(st, (uint32_t)polls, gave_up);
+    return cudaGetLastError() == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
 }
 
 rtn_status rtn_last_device_status(void* stream)

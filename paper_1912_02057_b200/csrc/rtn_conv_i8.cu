@@ -109,7 +109,7 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms, bool next = false)
     if ((int64_t)c.B * p.PH > (1 << 20)) return false;                // fast division ranges
     p.total_rows = c.B * p.PH;
     // two sub-tiles when the accumulators fit twice (double buffered) and there is enough work
-    p.TM = (4 * p.Np <= 512 && (int64_t)p.total_rows * p.PW >= (int64_t)4 * 148 * kTileM) ? 2 : 1;
+    p.TM = (4 * p.Np <= 512 && (int64_t)p.total_rows * p.PW >= (int64_t)4 * sms * kTileM) ? 2 : 1;
     if (2 * p.TM * p.Np > 512) return false;
     p.RT = p.TM * kTileM / p.PW;
     if (p.RT > kMaxSlots - p.halo) p.RT = kMaxSlots - p.halo;
@@ -905,14 +905,6 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
 }
 
-int sm_count()
-{
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
-    return sms;
-}
-
 // cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -937,19 +929,19 @@ EncodeTiledFn encode_tiled_fn()
 bool conv_i8_supported(const ConvArgs& c)
 {
     ConvI8Plan p;
-    return make_plan(c, p, 148);
+    return make_plan(c, p, device_sm_count());
 }
 
 bool conv_i8_next_supported(const ConvArgs& c)
 {
     ConvI8Plan p;
-    return make_plan(c, p, 148, true);
+    return make_plan(c, p, device_sm_count(), true);
 }
 
 static cudaError_t launch_conv_i8_any_mode(const ConvArgs& c, const NextLayerArgs* f, cudaStream_t s)
 {
     ConvI8Plan p;
-    if (!make_plan(c, p, sm_count(), f != nullptr)) return cudaErrorInvalidConfiguration;
+    if (!make_plan(c, p, device_sm_count(), f != nullptr)) return cudaErrorInvalidConfiguration;
     CUtensorMap tmap;
     memset(&tmap, 0, sizeof(tmap));
     if (f != nullptr && f->x_packed != nullptr) {

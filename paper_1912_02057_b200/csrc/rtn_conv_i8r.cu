@@ -628,14 +628,6 @@ void* static_scratch()
     return addr[dev];
 }
 
-int sm_count_r()
-{
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
-    return sms;
-}
-
 cudaError_t launch_with_scratch(const ConvArgs& c, const ConvI8RPlan& p, void* scratch, cudaStream_t s,
                                 const NextLayerArgs* f = nullptr)
 {
@@ -667,13 +659,13 @@ cudaError_t launch_with_scratch(const ConvArgs& c, const ConvI8RPlan& p, void* s
 bool conv_i8r_supported(const ConvArgs& c)
 {
     ConvI8RPlan p;
-    return make_plan_r(c, p, 148);
+    return make_plan_r(c, p, device_sm_count());
 }
 
 bool conv_i8r_next_supported(const ConvArgs& c)
 {
     ConvI8RPlan p;
-    return make_plan_r(c, p, 148, true);
+    return make_plan_r(c, p, device_sm_count(), true);
 }
 
 // Rough time of this variant for a shape, in microseconds (negative: not taken).  Measured on B200: about
@@ -682,7 +674,7 @@ bool conv_i8r_next_supported(const ConvArgs& c)
 double conv_i8r_estimate_us(const ConvArgs& c)
 {
     ConvI8RPlan p;
-    if (!make_plan_r(c, p, 148)) return -1.0;
+    if (!make_plan_r(c, p, device_sm_count())) return -1.0;
     const double macs = (double)p.Ptot * p.Cp * p.T * (double)(p.S * p.Nq);     // padded output pixels x K x filters
     return 12.0 + macs / ((p.Nq >= 64 ? 600.0 : 370.0) * 1e6);
 }
@@ -690,7 +682,7 @@ double conv_i8r_estimate_us(const ConvArgs& c)
 size_t conv_i8r_scratch_bytes(const ConvArgs& c)
 {
     ConvI8RPlan p;
-    return make_plan_r(c, p, 148) ? p.scratch_bytes : 0;
+    return make_plan_r(c, p, device_sm_count()) ? p.scratch_bytes : 0;
 }
 
 // The scratch buffer comes from the stream-ordered allocator and goes back to it right after the two
@@ -699,7 +691,7 @@ size_t conv_i8r_scratch_bytes(const ConvArgs& c)
 cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s)
 {
     ConvI8RPlan p;
-    if (!make_plan_r(c, p, sm_count_r())) return cudaErrorInvalidConfiguration;
+    if (!make_plan_r(c, p, device_sm_count())) return cudaErrorInvalidConfiguration;
     void* scratch = nullptr;
     cudaError_t e = cudaMallocAsync(&scratch, p.scratch_bytes, s);
     if (e != cudaSuccess) return e;
@@ -713,7 +705,7 @@ cudaError_t launch_conv_i8r(const ConvArgs& c, cudaStream_t s)
 cudaError_t launch_conv_i8r_static(const ConvArgs& c, cudaStream_t s)
 {
     ConvI8RPlan p;
-    if (!make_plan_r(c, p, sm_count_r())) return cudaErrorInvalidConfiguration;
+    if (!make_plan_r(c, p, device_sm_count())) return cudaErrorInvalidConfiguration;
     if (p.scratch_bytes > kStaticScratchBytes) return cudaErrorInvalidValue;
     void* scratch = static_scratch();
     if (scratch == nullptr) return cudaErrorInvalidDevicePointer;
@@ -727,7 +719,7 @@ size_t conv_i8r_static_scratch_bytes() { return kStaticScratchBytes; }
 cudaError_t launch_conv_i8r_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s)
 {
     ConvI8RPlan p;
-    if (!make_plan_r(c, p, sm_count_r(), true)) return cudaErrorInvalidConfiguration;
+    if (!make_plan_r(c, p, device_sm_count(), true)) return cudaErrorInvalidConfiguration;
     void* scratch = nullptr;
     cudaError_t e = cudaMallocAsync(&scratch, p.scratch_bytes, s);
     if (e != cudaSuccess) return e;

@@ -648,20 +648,12 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
 }
 
-int sm_count_s()
-{
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
-    return sms;
-}
-
 }  // namespace
 
 bool conv_i8s_supported(const ConvArgs& c)
 {
     ConvI8SPlan p;
-    return make_plan_s(c, p, 148);
+    return make_plan_s(c, p, device_sm_count());
 }
 
 // A filter stream of four stages or more is expanded once into scratch (an extra small kernel).
@@ -670,7 +662,7 @@ static bool pre_expand(const ConvI8SPlan& p) { return p.pre != 0; }
 int conv_i8s_launches(const ConvArgs& c)
 {
     ConvI8SPlan p;
-    if (!make_plan_s(c, p, 148)) return 0;
+    if (!make_plan_s(c, p, device_sm_count())) return 0;
     return pre_expand(p) ? 2 : 1;
 }
 
@@ -678,7 +670,7 @@ template <bool kNext>
 static cudaError_t launch_i8s_mode(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s)
 {
     ConvI8SPlan p;
-    if (!make_plan_s(c, p, sm_count_s(), kNext)) return cudaErrorInvalidConfiguration;
+    if (!make_plan_s(c, p, device_sm_count(), kNext)) return cudaErrorInvalidConfiguration;
     if (!pre_expand(p)) {
         cudaError_t e = cudaFuncSetAttribute(conv_i8s_kernel<false, kNext>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)p.smem_bytes);
@@ -714,7 +706,7 @@ cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s) { return launch_i
 double conv_i8s_estimate_us(const ConvArgs& c)
 {
     ConvI8SPlan p;
-    if (!make_plan_s(c, p, 148)) return -1.0;
+    if (!make_plan_s(c, p, device_sm_count())) return -1.0;
     const int strip_rows = (p.total_rows + p.grid - 1) / p.grid;
     const int tiles = (strip_rows + p.RT - 1) / p.RT;
     const double stage_us = (p.pre ? 0.75 : 1.0) * (double)p.NpP / 256.0;
@@ -725,12 +717,12 @@ double conv_i8s_estimate_us(const ConvArgs& c)
 bool conv_i8s_next_supported(const ConvArgs& c)
 {
     ConvI8SPlan p;
-    return make_plan_s(c, p, 148, true);
+    return make_plan_s(c, p, device_sm_count(), true);
 }
 int conv_i8s_next_launches(const ConvArgs& c)
 {
     ConvI8SPlan p;
-    if (!make_plan_s(c, p, 148, true)) return 0;
+    if (!make_plan_s(c, p, device_sm_count(), true)) return 0;
     return pre_expand(p) ? 2 : 1;
 }
 cudaError_t launch_conv_i8s_next(const ConvArgs& c, const NextLayerArgs& f, cudaStream_t s)

@@ -413,14 +413,6 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
 }
 
-int sm_count_g()
-{
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
-    return sms;
-}
-
 // Pre-expansion mode of a plan: 0 = both operands expanded inside the kernel (one row tile: every weight row
 // is expanded once anyway), 1 = weights expanded ahead (several row tiles, one column tile), 2 = both ahead
 // (several tiles each way: every row of either operand would be expanded once per tile it takes part in).
@@ -438,20 +430,20 @@ int gemm_pre_mode(const GemmI8Plan& p, int64_t K)
 bool gemm_i8_supported(int64_t M, int64_t N, int64_t K)
 {
     GemmI8Plan p;
-    return make_gemm_plan(M, N, K, p, 148);
+    return make_gemm_plan(M, N, K, p, device_sm_count());
 }
 
 int gemm_i8_launches(int64_t M, int64_t N, int64_t K)
 {
     GemmI8Plan p;
-    if (!make_gemm_plan(M, N, K, p, 148)) return 0;
+    if (!make_gemm_plan(M, N, K, p, device_sm_count())) return 0;
     return gemm_pre_mode(p, K) == 0 ? 1 : 2;
 }
 
 cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s)
 {
     GemmI8Plan p;
-    if (!make_gemm_plan(g.M, g.N, g.K, p, sm_count_g())) return cudaErrorInvalidConfiguration;
+    if (!make_gemm_plan(g.M, g.N, g.K, p, device_sm_count())) return cudaErrorInvalidConfiguration;
     const int mode = gemm_pre_mode(p, g.K);
     if (mode == 0) {
         cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);

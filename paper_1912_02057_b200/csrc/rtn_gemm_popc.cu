@@ -151,8 +151,9 @@ int gemm_popc_slices(int64_t M, int64_t N, int64_t K)
 {
     const int64_t tiles = ((M + 15) / 16) * ((N + 15) / 16);
     const int64_t nblk = (K + kBlockCodes - 1) / kBlockCodes;
-    if (tiles >= 74 || nblk < 8) return 1;
-    int64_t slices = (296 + tiles - 1) / tiles;
+    const int sms = device_sm_count();
+    if (tiles >= sms / 2 || nblk < 8) return 1;
+    int64_t slices = (2 * sms + tiles - 1) / tiles;
     if (slices > nblk / 2) slices = nblk / 2;
     return slices < 2 ? 1 : (int)slices;
 }
@@ -173,10 +174,10 @@ cudaError_t launch_gemm_popc(const GemmArgs& g, cudaStream_t s)
         return cudaGetLastError();
     }
     auto ctas = [&](int64_t t) { return ((g.M + t - 1) / t) * ((g.N + t - 1) / t); };
-    if (ctas(64) >= 148) {
+    if (ctas(64) >= device_sm_count()) {
         dim3 grid((unsigned)((g.M + 63) / 64), (unsigned)((g.N + 63) / 64));
         gemm_popc_kernel<4, 4><<<grid, 256, 0, s>>>(g);
-    } else if (ctas(32) >= 148) {
+    } else if (ctas(32) >= device_sm_count()) {
         dim3 grid((unsigned)((g.M + 31) / 32), (unsigned)((g.N + 31) / 32));
         gemm_popc_kernel<2, 2><<<grid, 256, 0, s>>>(g);
     } else {

@@ -72,6 +72,25 @@ struct NextLayerArgs {
     uint8_t* out_packed;    // [B*Ho*Wo] packed rows of N codes
 };
 
+// Multiprocessors of the current device, asked once per device.  Plans, *_supported answers, launch counts,
+// scratch sizes and the launchers all size their grids with this number, so they agree on any part.  Without a
+// usable device (a host-only query) the answer is a B200's 148.
+inline int device_sm_count()
+{
+    constexpr int kSlots = 64;
+    static int cached[kSlots];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+    if (dev >= 0 && dev < kSlots && cached[dev] > 0) return cached[dev];
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+        cudaGetLastError();
+        return 148;
+    }
+    if (dev >= 0 && dev < kSlots) cached[dev] = sms;
+    return sms;
+}
+
 // Launchers (each returns the cudaError_t of its launch).
 cudaError_t launch_pack_weights(const int8_t* w, int64_t N, int64_t C, int kh, int kw,
                                 uint8_t* packed, int32_t* w_sum, unsigned* status, cudaStream_t s);

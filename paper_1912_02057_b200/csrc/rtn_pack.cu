@@ -62,7 +62,7 @@ cudaError_t launch_pack_weights(const int8_t* w, int64_t N, int64_t C, int kh, i
     const int64_t total = N * (((words + 3) / 4) * 4);
     const int threads = 256;
     int64_t blocks = (total + threads - 1) / threads;
-    if (blocks > 148 * 64) blocks = 148 * 64;
+    if (blocks > device_sm_count() * 64) blocks = device_sm_count() * 64;
     pack_weights_kernel<<<(unsigned)blocks, threads, 0, s>>>(w, N, C, kh, kw, packed, w_sum, status);
     return cudaGetLastError();
 }
@@ -312,14 +312,14 @@ cudaError_t launch_ternarize_pack(const float* a, int64_t M, int64_t K, const fl
     const int wpr = ntrip >= 8 ? 8 : ntrip >= 4 ? 4 : ntrip >= 2 ? 2 : 1;
     const int rpb = 8 / wpr;
     int64_t blocks = (M + rpb - 1) / rpb;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > device_sm_count() * 16) blocks = device_sm_count() * 16;
     const bool per_k = n_thr != 1;
     const bool vec = (K % 8) == 0 && (reinterpret_cast<uintptr_t>(a) & 15) == 0 &&
                      (!per_k || ((reinterpret_cast<uintptr_t>(t_lo) | reinterpret_cast<uintptr_t>(t_hi)) & 15) == 0);
     if (vec && (K == 32 || K == 64 || K == 128 || K == 256)) {
         const int64_t units = (M * K + 255) / 256, warps = (units + 1) / 2;
         int64_t blk = (warps + 7) / 8;
-        if (blk > 148 * 16) blk = 148 * 16;
+        if (blk > device_sm_count() * 16) blk = device_sm_count() * 16;
         if (!per_k)
             ternarize_pack_rows_kernel<false><<<(unsigned)blk, threads, 0, s>>>(a, M, (int)K, t_lo, t_hi, packed, a_sum);
         else

@@ -123,10 +123,10 @@ cudaError_t launch_gemm_quaternary(const uint8_t* a, const uint8_t* w, int64_t M
                                    cudaStream_t s)
 {
     auto ctas = [&](int64_t t) { return ((M + t - 1) / t) * ((N + t - 1) / t); };
-    if (ctas(64) >= 148) {
+    if (ctas(64) >= device_sm_count()) {
         dim3 grid((unsigned)((M + 63) / 64), (unsigned)((N + 63) / 64));
         gemm_quaternary_kernel<4, 4><<<grid, 256, 0, s>>>(a, w, M, N, K, out);
-    } else if (ctas(32) >= 148) {
+    } else if (ctas(32) >= device_sm_count()) {
         dim3 grid((unsigned)((M + 31) / 32), (unsigned)((N + 31) / 32));
         gemm_quaternary_kernel<2, 2><<<grid, 256, 0, s>>>(a, w, M, N, K, out);
     } else {

@@ -58,10 +58,11 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity)
 // returns false, so a lost arrival can never hang the GPU.
 constexpr uint32_t kWaitPolls = 1u << 19;
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned* status)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned* status,
+                                          uint32_t polls = kWaitPolls)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < kWaitPolls; ++i) {
+    for (uint32_t i = 0; i < polls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
     }
     atomicOr(status, 2u);       // kStatusWaitTimeout

@@ -37,3 +37,21 @@ def read_golden(name):
             if line and not line.startswith("#"):
                 rows.append(line.split())
     return rows
+
+
+def pytest_terminal_summary(terminalreporter):
+    """How far the fp32 outputs are from the rule without the sum-of-terms relaxation, per case."""
+    try:
+        from helpers import STRICT_REPORT
+    except Exception:
+        return
+    if not STRICT_REPORT:
+        return
+    tr = terminalreporter
+    tr.write_sep("-", "fp32 outputs outside 1e-5 |ref| and 1e-6 (all inside the tolerance the tests assert)")
+    total = missed = 0
+    for what, (n, m, worst) in sorted(STRICT_REPORT.items()):
+        total, missed = total + n, missed + m
+        if m:
+            tr.write_line(f"{what}: {m} of {n} outputs, largest |err| {worst:.3e}")
+    tr.write_line(f"all cases: {missed} of {total} outputs")

@@ -69,6 +69,9 @@ def test_argument_errors_come_back_as_codes_without_a_gpu():
     assert conv(4, 3, 1, 1, 0, nthr=3) == 2
     assert conv(4, 3, 1, 1, 7) == 4
     assert rtn.lib().rtn_status_string(2).startswith(b"RTN_ERR_SHAPE")
+    assert L.rtn_selftest_wait_timeout(16, None, None) == 1
+    assert L.rtn_selftest_wait_timeout(0, fake, None) == 2
+    assert L.rtn_selftest_wait_timeout(1 << 20, fake, None) == 2
 
 
 def test_k_slices_only_for_small_outputs_with_a_long_k():

@@ -9,7 +9,7 @@ import oracle
 import paper_1912_02057_b200 as rtn
 from paper_1912_02057_b200 import inputs
 from helpers import (conv_parity, conv_parity_sampled, conv_through_abi, dev, gemm_parity,
-                     gemm_through_abi)
+                     gemm_parity_sampled, gemm_through_abi)
 
 pytestmark = pytest.mark.gpu
 
@@ -149,6 +149,15 @@ def test_gemm_config5_2048(variant):
     run_or_skip_unsupported(lambda: gemm_parity(inputs.config5(2048), variant), variant)
 
 
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("n,n_rows", [(4096, 384), (8192, 256), (16384, 160)])
+def test_gemm_config5_large_sampled(n, n_rows, variant):
+    """The sweep's larger sizes (Eq. 9 at M = N = K = n): sampled rows x all columns against the plain oracle."""
+    case = inputs.config5(n)
+    rows = run_or_skip_unsupported(lambda: gemm_parity_sampled(case, variant, n_rows, seed=n), variant)
+    assert rows[0] == 0 and rows[-1] == n - 1 and {127, 128, 255, 256, n - 128, n - 129}.issubset(set(rows.tolist()))
+
+
 def test_gemm_is_deterministic():
     case = inputs.gemm_case("det", 257, 129, 640, seed=9, p_zero=0.3, act="uniform3", thresholds=(-0.5, 0.5))
     for variant in (rtn.VARIANT_POPC, rtn.VARIANT_I8):
@@ -267,3 +276,23 @@ def test_conv_variants_agree_bit_for_bit():
         assert e.code == 5
         pytest.skip("tensor-core variant does not take this shape")
     assert np.array_equal(a1, a2)
+
+
+# ------------------------------------------------------------------------------------ bounded waits
+def test_a_wait_that_nothing_ends_gives_up_and_is_reported_once():
+    """Every device-side wait of the tensor-core kernels is bounded.  A wait on an mbarrier nothing arrives on
+    must return (the self-test kernel uses the kernels' own wait routine with a short limit), the status word
+    must say RTN_ERR_DEVICE_TIMEOUT exactly once, and the context must stay usable."""
+    assert rtn.rtn_last_device_status() == 0
+    gave_up = rtn.rtn_selftest_wait_timeout(1024)
+    torch.cuda.synchronize()
+    assert int(gave_up.item()) == 1
+    assert rtn.rtn_last_device_status() == 7          # RTN_ERR_DEVICE_TIMEOUT, read and cleared
+    assert rtn.rtn_last_device_status() == 0
+    # the device still works: a tensor-core conv right after, checked against the oracle
+    case = inputs.config2(batch=2, thresholds=(0.3, 1.0))
+    conv_parity(case, rtn.VARIANT_I8)
+    assert rtn.rtn_last_device_status() == 0
+    with pytest.raises(rtn.RtnError) as e:
+        rtn.rtn_selftest_wait_timeout(1 << 20)          # the limit itself is bounded
+    assert e.value.code == 2

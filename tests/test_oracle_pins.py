@@ -209,6 +209,91 @@ def test_epilogue_each_term_has_its_own_factor():
     assert oracle.gemm(x, w, 0.0, 7.0, 0.0, 5.0)[1][0, 0] == K * 7 * 5
 
 
+def test_epilogue_mag_is_the_sum_of_absolute_terms():
+    # mag scales every fp32 tolerance: pin it to a hand-written sum of |term_i| (dyadic values, exact)
+    x = np.array([[1, 1, 0]], np.int8)      # S_x = 2
+    w = np.array([[-1, 0, 0]], np.int8)     # S_w = -1, S_xw = -1
+    K = 3
+    a_s, a_o, w_s, w_o = 2.0, -0.5, 3.0, 0.25
+    _, out, mag = oracle.gemm(x, w, a_s, a_o, w_s, w_o)
+    terms = [a_s * w_s * -1, a_s * w_o * 2, a_o * w_s * -1, K * a_o * w_o]      # -6, 1, 1.5, -0.375
+    assert out[0, 0] == sum(terms) == -3.875
+    assert mag[0, 0] == sum(abs(t) for t in terms) == 8.875
+    # one term at a time: each |term| arrives in mag with its own factor
+    assert oracle.gemm(x, w, 2.0, 0.0, 3.0, 0.0)[2][0, 0] == 6.0
+    assert oracle.gemm(x, w, 2.0, 0.0, 0.0, 5.0)[2][0, 0] == 20.0
+    assert oracle.gemm(x, w, 0.0, 7.0, 3.0, 0.0)[2][0, 0] == 21.0
+    assert oracle.gemm(x, w, 0.0, 7.0, 0.0, 5.0)[2][0, 0] == 105.0
+    # random small cases against a pure-Python sum, per-row and per-column parameters
+    g = np.random.default_rng(12)
+    x = inputs.weight_codes(g, (4, 23), 0.3)
+    w = inputs.weight_codes(g, (3, 23), 0.3)
+    a_s, a_o = inputs.uniform(g, 0.5, 1.5, (4,)), inputs.uniform(g, -0.5, 0.5, (4,))
+    w_s, w_o = inputs.uniform(g, 0.5, 1.5, (3,)), inputs.uniform(g, -0.5, 0.5, (3,))
+    _, _, mag = oracle.gemm(x, w, a_s, a_o, w_s, w_o)
+    for m in range(4):
+        for n in range(3):
+            sxw = sum(int(p) * int(q) for p, q in zip(x[m], w[n]))
+            sx, sw = int(x[m].sum()), int(w[n].sum())
+            As, Ao, Ws, Wo = float(a_s[m]), float(a_o[m]), float(w_s[n]), float(w_o[n])
+            want = abs(As * Ws * sxw) + abs(As * Wo * sx) + abs(Ao * Ws * sw) + abs(23 * Ao * Wo)
+            assert abs(mag[m, n] - want) <= 1e-13 * want
+            assert mag[m, n] >= abs(oracle.gemm(x, w, a_s, a_o, w_s, w_o)[1][m, n])
+
+
+def test_conv_mag_both_pad_modes_hand_case():
+    # 1 channel, 2x2 image of all +1, one 3x3 filter of all -1, pad 1: the output at (0, 0) sees 4 inside taps
+    x = np.ones((1, 1, 2, 2), np.int8)
+    w = -np.ones((1, 1, 3, 3), np.int8)
+    a_s, a_o, w_s, w_o = 2.0, 0.5, 4.0, 0.25
+    # code-zero padding: S_xw = -4, S_x = 4, S_w = -9, K = 9
+    terms0 = [a_s * w_s * -4, a_s * w_o * 4, a_o * w_s * -9, 9 * a_o * w_o]     # -32, 2, -18, 1.125
+    S, out, mag = oracle.conv2d(x, w, 1, 1, oracle.PAD_CODE_ZERO, a_s, a_o, np.float32(w_s), np.float32(w_o))
+    assert S[0, 0, 0, 0] == -4 and out[0, 0, 0, 0] == sum(terms0) and mag[0, 0, 0, 0] == 53.125
+    # value-zero padding: S_w and K over the 4 inside taps only
+    terms1 = [a_s * w_s * -4, a_s * w_o * 4, a_o * w_s * -4, 4 * a_o * w_o]     # -32, 2, -8, 0.5
+    S, out, mag = oracle.conv2d(x, w, 1, 1, oracle.PAD_VALUE_ZERO, a_s, a_o, np.float32(w_s), np.float32(w_o))
+    assert S[0, 0, 0, 0] == -4 and out[0, 0, 0, 0] == sum(terms1) and mag[0, 0, 0, 0] == 42.5
+    pts = np.array([[0, 0, 0, 0], [0, 0, 1, 1]], np.int64)
+    _, op, mp = oracle.conv2d_points(x, w, 1, 1, oracle.PAD_VALUE_ZERO, a_s, a_o, np.float32(w_s), np.float32(w_o), pts)
+    assert list(op) == [sum(terms1)] * 2 and list(mp) == [42.5, 42.5]
+
+
+def test_within_tolerance_branches_on_hand_made_triples():
+    T = oracle.within_tolerance
+    one = lambda got, ref, mag: bool(T(np.array([got]), np.array([ref]), np.array([mag]))[0])
+    # relative branch alone decides (mag tiny): 1e-5 |ref| with |ref| = 1000 -> 0.01
+    assert one(1000.0 + 0.0099, 1000.0, 0.0)
+    assert not one(1000.0 + 0.0101, 1000.0, 0.0)
+    assert one(-1000.0 - 0.0099, -1000.0, 0.0)
+    assert not one(-1000.0 + 0.0101, -1000.0, 0.0)
+    # absolute branch with mag < 1: the floor max(1, mag) = 1 -> 1e-6
+    assert one(0.9e-6, 0.0, 0.25)
+    assert not one(1.1e-6, 0.0, 0.25)
+    assert one(-0.9e-6, 0.0, 0.0)
+    # absolute branch scaled by mag > 1 (terms cancel: ref near 0, mag = 400 -> 4e-4)
+    assert one(0.01 + 3.9e-4, 0.01, 400.0)
+    assert not one(0.01 + 4.1e-4, 0.01, 400.0)
+    # the two branches are alternatives (or), not both required (and)
+    assert one(1000.0 + 0.009, 1000.0, 1.0)         # relative holds, absolute (1e-6) does not
+    assert one(1e-3 + 3e-4, 1e-3, 400.0)            # absolute holds, relative (1e-8) does not
+    # a mag a thousand times too large would accept this one
+    assert not one(0.5, 0.0, 400.0)
+    # shapes broadcast elementwise
+    got = np.array([[0.0, 2e-6], [1.0, 1.0 + 2e-5]])
+    ref = np.array([[0.0, 0.0], [1.0, 1.0]])
+    assert T(got, ref, np.ones((2, 2))).tolist() == [[True, False], [True, False]]
+    assert (oracle.REL_TOL, oracle.ABS_TOL) == (1e-5, 1e-6)
+
+
+def test_strict_miss_counts_the_outputs_outside_the_unrelaxed_rule():
+    # the unrelaxed rule: |err| <= 1e-5 |ref| or |err| <= 1e-6
+    got = np.array([0.0, 2e-6, 1.0 + 2e-5, 1000.0 + 0.009])
+    ref = np.array([0.0, 0.0, 1.0, 1000.0])
+    n, worst = oracle.strict_miss(got, ref)
+    assert n == 2 and abs(worst - 2e-5) < 1e-9
+
+
 # ------------------------------------------------------------------ convolution
 def _deq(codes, s, o):
     return s * torch.from_numpy(codes.astype(np.float64)) + o

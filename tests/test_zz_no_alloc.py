@@ -1,13 +1,43 @@
 """The conv entry point that allocates nothing (collected last: its first call does the per-device
 set-up of the static scratch array)."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_1912_02057_b200 as rtn
 from paper_1912_02057_b200 import inputs
+from helpers import check_fp32
 
 pytestmark = pytest.mark.gpu
+
+# cudaMemPoolAttr values of the CUDA runtime API
+_RESERVED_HIGH, _USED_HIGH = 6, 8
+
+
+class DefaultPool:
+    """High-water marks of the device's default stream-ordered memory pool: the pool cudaMallocAsync draws
+    from.  (Free-memory readings miss an allocation that is given back before the next synchronize.)"""
+
+    def __init__(self):
+        self.rt = ctypes.CDLL("libcudart.so.12")
+        self.pool = ctypes.c_void_p()
+        assert self.rt.cudaDeviceGetDefaultMemPool(ctypes.byref(self.pool), torch.cuda.current_device()) == 0
+
+    def reset(self):
+        zero = ctypes.c_uint64(0)
+        for attr in (_RESERVED_HIGH, _USED_HIGH):
+            assert self.rt.cudaMemPoolSetAttribute(self.pool, attr, ctypes.byref(zero)) == 0
+
+    def high(self):
+        v = ctypes.c_uint64(0)
+        out = []
+        for attr in (_RESERVED_HIGH, _USED_HIGH):
+            assert self.rt.cudaMemPoolGetAttribute(self.pool, attr, ctypes.byref(v)) == 0
+            out.append(int(v.value))
+        return tuple(out)
 
 
 def _dev(a):
@@ -41,15 +71,40 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row(shape, pad_mo
     out1.fill_(float("nan"))
     torch.cuda.synchronize()
     free_before = torch.cuda.mem_get_info()[0]
+    pool = DefaultPool()
+    pool.reset()
     rtn.rtn_ternary_conv2d_noalloc(pad_mode=pad_mode, out=out1, **a)
     rtn.rtn_ternary_conv2d_noalloc(pad_mode=pad_mode, out=out2, dbg_acc=acc2, **a)      # reuses the same scratch
     torch.cuda.synchronize()
     assert torch.cuda.mem_get_info()[0] == free_before, "device memory in use changed across the calls"
+    assert pool.high() == (0, 0), "the stream-ordered pool was used during the calls"
     assert rtn.rtn_last_device_status() == 0
+    # against the oracle directly: integers bit for bit, fp32 within the library's tolerance
+    codes = oracle.ternarize(case.x, case.t_lo, case.t_hi, channel_axis=1)
+    S, want, mag = oracle.conv2d(codes, case.w_codes, case.stride, case.pad, pad_mode, case.a_scale,
+                                 case.a_offset, case.w_scale, case.w_offset)
+    assert np.array_equal(acc2.cpu().numpy().astype(np.int64), S), "integer accumulators differ from the oracle"
+    check_fp32(out1.cpu().numpy(), want, mag, case.name)
+    check_fp32(out2.cpu().numpy(), want, mag, case.name)
     # same arithmetic as the allocating entry point: integers equal, fp32 equal bit for bit
     assert torch.equal(acc2, acc_ref)
     assert torch.equal(out1.view(torch.int32), ref.view(torch.int32))
     assert torch.equal(out2.view(torch.int32), ref.view(torch.int32))
+
+
+def test_pool_high_water_marks_see_an_allocating_call():
+    """The instrument of the test above works: the allocating entry point on the same two-kernel path does
+    raise the pool's high-water marks."""
+    case = inputs.conv_case("alloc_3x3s2", 2, 128, 14, 14, 256, 3, 2, 1, seed=3, p_zero=0.4, thresholds=(0.3, 1.0))
+    assert rtn.rtn_conv_kernel_launches(2, 128, 14, 14, 256, 3, 3, 2, 1) == 2
+    a = _args(case)
+    rtn.rtn_ternary_conv2d(pad_mode=rtn.PAD_CODE_ZERO, **a)
+    torch.cuda.synchronize()
+    pool = DefaultPool()
+    pool.reset()
+    rtn.rtn_ternary_conv2d(pad_mode=rtn.PAD_CODE_ZERO, **a)
+    torch.cuda.synchronize()
+    assert pool.high()[1] > 0
 
 
 def test_noalloc_rejects_what_does_not_fit_or_is_not_taken():
