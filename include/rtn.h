@@ -261,6 +261,24 @@ rtn_status rtn_last_device_status(void* stream);
  * RTN_ERR_DEVICE_TIMEOUT once.  Nothing traps or spins without limit; the context stays usable.  Only enqueues. */
 rtn_status rtn_selftest_wait_timeout(int64_t polls, int32_t* gave_up, void* stream);
 
+/* Peak probes (measurement aids; the paper has no counterpart).  The contraction kernels are judged against two
+ * ceilings that no memory copy measures: the int8 tensor-pipe rate and the issue rate of the AND / XOR /
+ * popcount pattern of Eq. 9.  Each probe launches rtn_probe_ctas() CTAs (one per multiprocessor) that run
+ * nothing but that work on on-chip operands, and writes the SM-clock cycles of each CTA's loop to `cycles`
+ * (device int64 [rtn_probe_ctas()], 8-byte aligned); time the launch with events for the rate in seconds.
+ *   rtn_probe_peak_i8   n_mma (1..2^22) tcgen05.mma kind::i8 of M = 128, N = 256, K = 32 per CTA, operands in
+ *                       shared memory, one accumulator; rtn_probe_i8_ops_per_mma() = 2*128*256*32 operations each.
+ *                       The final wait is bounded like every other (rtn_last_device_status reports a time-out).
+ *   rtn_probe_peak_popc rounds (1..2^24) rounds per thread of 64 word pairs, 1024 threads per CTA, registers
+ *                       only; rtn_probe_popc_ops_per_round() operations (2 per code pair) per CTA and round.
+ *                       `sink`: device int32 the kernel never writes in practice (keeps the loop alive).
+ * Both only enqueue. */
+int64_t rtn_probe_ctas(void);
+int64_t rtn_probe_i8_ops_per_mma(void);
+int64_t rtn_probe_popc_ops_per_round(void);
+rtn_status rtn_probe_peak_i8(int64_t n_mma, int64_t* cycles, void* stream);
+rtn_status rtn_probe_peak_popc(int64_t rounds, int64_t* cycles, int32_t* sink, void* stream);
+
 /* Static text for a status code. */
 const char* rtn_status_string(rtn_status s);
 

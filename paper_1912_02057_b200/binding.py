@@ -95,6 +95,16 @@ def lib():
         L.rtn_conv_next_kernel_launches.argtypes = [_i64] * 9
         L.rtn_last_device_status.restype = _int
         L.rtn_last_device_status.argtypes = [_vp]
+        L.rtn_probe_ctas.restype = _i64
+        L.rtn_probe_ctas.argtypes = []
+        L.rtn_probe_i8_ops_per_mma.restype = _i64
+        L.rtn_probe_i8_ops_per_mma.argtypes = []
+        L.rtn_probe_popc_ops_per_round.restype = _i64
+        L.rtn_probe_popc_ops_per_round.argtypes = []
+        L.rtn_probe_peak_i8.restype = _int
+        L.rtn_probe_peak_i8.argtypes = [_i64, _vp, _vp]
+        L.rtn_probe_peak_popc.restype = _int
+        L.rtn_probe_peak_popc.argtypes = [_i64, _vp, _vp, _vp]
         L.rtn_selftest_wait_timeout.restype = _int
         L.rtn_selftest_wait_timeout.argtypes = [_i64, _vp, _vp]
         L.rtn_status_string.restype = C.c_char_p
@@ -312,3 +322,21 @@ def rtn_selftest_wait_timeout(polls=1024, stream=None):
     _check(lib().rtn_selftest_wait_timeout(int(polls), _ptr(gave_up, torch.int32), _stream(stream)),
            "rtn_selftest_wait_timeout")
     return gave_up
+
+
+def rtn_probe_peak_i8(n_mma, stream=None):
+    """Launches the int8 tensor-pipe probe; returns (cycles int64 [CTAs] on the device, operations per CTA)."""
+    ctas = int(lib().rtn_probe_ctas())
+    cycles = torch.zeros((ctas,), dtype=torch.int64, device="cuda")
+    _check(lib().rtn_probe_peak_i8(int(n_mma), _ptr(cycles, torch.int64), _stream(stream)), "rtn_probe_peak_i8")
+    return cycles, int(n_mma) * int(lib().rtn_probe_i8_ops_per_mma())
+
+
+def rtn_probe_peak_popc(rounds, stream=None):
+    """Launches the AND / XOR / popcount probe; returns (cycles int64 [CTAs] on the device, operations per CTA)."""
+    ctas = int(lib().rtn_probe_ctas())
+    cycles = torch.zeros((ctas,), dtype=torch.int64, device="cuda")
+    sink = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    _check(lib().rtn_probe_peak_popc(int(rounds), _ptr(cycles, torch.int64), _ptr(sink, torch.int32), _stream(stream)),
+           "rtn_probe_peak_popc")
+    return cycles, int(rounds) * int(lib().rtn_probe_popc_ops_per_round())

@@ -56,6 +56,10 @@ rtn_status check_params(const float* s, const float* o, int64_t n, int64_t full)
 
 }  // namespace
 
+namespace rtn {
+unsigned* device_status_word() { return status_word(); }
+}
+
 extern "C" {
 
 size_t rtn_packed_row_bytes(int64_t K)

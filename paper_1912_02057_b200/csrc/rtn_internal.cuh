@@ -91,6 +91,9 @@ inline int device_sm_count()
     return sms;
 }
 
+// Device address of the current device's status word (NULL on failure); defined with the C ABI.
+unsigned* device_status_word();
+
 // Launchers (each returns the cudaError_t of its launch).
 cudaError_t launch_pack_weights(const int8_t* w, int64_t N, int64_t C, int kh, int kw,
                                 uint8_t* packed, int32_t* w_sum, unsigned* status, cudaStream_t s);

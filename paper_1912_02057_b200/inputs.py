@@ -201,6 +201,16 @@ def resnet18_layer(name, batch=128, p_zero=0.5):
     raise KeyError(name)
 
 
+def resnet18_fp32_ends(seed=46):
+    """Random-init weights of the two full-precision ends of ResNet-18 (section "Implementation Details":
+    first and last layer stay full precision): stem conv [64,3,7,7] ~ N(0, 2/(64*49)), classifier
+    [1000,512] ~ U(-1/sqrt(512), 1/sqrt(512)) with a bias of the same range."""
+    g = rng(seed)
+    stem = (g.standard_normal((64, 3, 7, 7), dtype=np.float32) * np.float32(np.sqrt(2.0 / (64 * 49)))).astype(np.float32)
+    bound = 1.0 / np.sqrt(512.0)
+    return stem, uniform(g, -bound, bound, (1000, 512)), uniform(g, -bound, bound, (1000,))
+
+
 # ------------------------------------------------------------------ the ternary body of ResNet-18 as a chain
 @dataclass
 class BodyLayer:
