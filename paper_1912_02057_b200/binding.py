@@ -27,7 +27,9 @@ class RtnError(RuntimeError):
 
 
 def lib_path():
-    return os.path.join(_HERE, _LIB_NAME)
+    """The product library; RTN_B200_LIBRARY names another build of it (the instrumented one of
+    paper_1912_02057_b200.timeline)."""
+    return os.environ.get("RTN_B200_LIBRARY") or os.path.join(_HERE, _LIB_NAME)
 
 
 _lib = None

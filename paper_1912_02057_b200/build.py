@@ -1,6 +1,9 @@
 """Builds librtn_b200.so in-tree with nvcc for sm_100a.
 
-Usage: python -m paper_1912_02057_b200.build [--force] [--verbose]
+Usage: python -m paper_1912_02057_b200.build [--force] [--verbose] [--timeline]
+
+--timeline builds a second library, librtn_b200_timeline.so, with the in-kernel clock stamps of
+csrc/rtn_timeline.cuh compiled in (for paper_1912_02057_b200.timeline; the product library never has them).
 """
 import glob
 import os
@@ -25,7 +28,16 @@ def _newer(target, deps):
     return all(os.path.getmtime(d) <= t for d in deps)
 
 
-def build(force=False, verbose=False):
+LIB_TIMELINE = os.path.join(HERE, "librtn_b200_timeline.so")
+
+
+def build(force=False, verbose=False, timeline=False):
+    if timeline:
+        return _build(os.path.join(HERE, "_build_timeline"), LIB_TIMELINE, ["-DRTN_TIMELINE"], force, verbose)
+    return _build(OBJ, LIB, [], force, verbose)
+
+
+def _build(OBJ, LIB, extra, force, verbose):
     os.makedirs(OBJ, exist_ok=True)
     headers = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
     sources = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
@@ -34,7 +46,7 @@ def build(force=False, verbose=False):
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or not _newer(obj, [src] + headers):
-            cmd = ["nvcc", *NVCC_FLAGS, "-c", src, "-o", obj]
+            cmd = ["nvcc", *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)
@@ -60,4 +72,4 @@ def build(force=False, verbose=False):
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, timeline="--timeline" in sys.argv))

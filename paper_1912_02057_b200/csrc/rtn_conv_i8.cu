@@ -33,9 +33,16 @@
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
 #include "rtn_conv_i8_common.cuh"
+#include "rtn_timeline.cuh"
 
 #include <cuda.h>
 #include <string.h>
+
+// Timeline slots (instrumented build only): 0 kernel entry, 1 set-up done, 2 filters expanded, 3 epilogue constants
+// ready, 4 kernel end; per tile i < 8: 8+2i / 9+2i producer issues first / last batch, 24+2i / 25+2i converters begin /
+// end, 40+2i / 41+2i first MMA can issue / commit, 56+2i / 57+2i epilogue begins / ends; per tile i < 6 and channel group
+// j < 2: 72+4i+2j the group's staged rows have landed, 73+4i+2j converter thread 0 has converted its share.
+RTN_TL_DEFINE(conv_i8)
 
 namespace rtn {
 
@@ -58,6 +65,7 @@ constexpr int kMaxStages = 8;                         // input batches (one tile
 constexpr int kMaxGroups = 16;                          // groups of 32 input channels (C <= 512)
 constexpr int kMaxMma = 160;                           // MMAs per sub-tile the descriptor table holds
 constexpr int kMaxSlots = 32;                          // row slots of a tile (rows + halo rows)
+constexpr int kRowwiseMinPW = 24;                      // padded width from which a warp per staged image row pays
 constexpr int kTileM = 128;                            // pixels per MMA (TMEM lanes)
 constexpr size_t kSmemLimit = 220 * 1024;
 constexpr int kConvBarrier = 1;                        // named barrier of the converter warps
@@ -73,6 +81,7 @@ struct ConvI8Plan {
     int R0;                // padded rows of a strip's first tile (<= RT)
     int halo;              // kh - 1 rows shared with the next tile
     int ppix;              // pixels allocated per code buffer
+    int strip;             // one code buffer holds the CTA's whole strip (no double buffering, no halo copies)
     int total_rows;        // B*PH
     int grid;              // CTAs = strips
     uint32_t tmem_cols;
@@ -118,9 +127,24 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms, bool next = false)
     // epilogue then start after half the input, and (the strip length permitting) the last tile,
     // whose epilogue nothing overlaps, is short as well.
     p.R0 = (p.RT >= 2 && (int64_t)p.total_rows >= (int64_t)2 * p.RT * sms) ? p.RT / 2 : p.RT;
+#ifdef RTN_KNOB_R0
+    if (p.R0 > RTN_KNOB_R0) p.R0 = RTN_KNOB_R0;
+#endif
     p.ppix = (p.TM * kTileM + p.halo * p.PW + (c.kw - 1) + 7) / 8 * 8;
     const int tiles = (p.total_rows + p.RT - 1) / p.RT;
     p.grid = tiles < sms ? tiles : sms;
+    // Short strips (small batches): the codes of a CTA's whole strip fit in shared memory at one byte per value.
+    // The converters then run ahead of the tensor core as fast as the input arrives (nothing waits for a code
+    // buffer to be free, no halo rows are copied), which takes the input stream off the critical path.
+    const int strip_rows = (p.total_rows + p.grid - 1) / p.grid;
+    const int strip_tiles = strip_rows <= p.R0 ? 1 : 1 + (strip_rows - p.R0 + p.RT - 1) / p.RT;
+    const int strip_ppix = ((strip_rows - 1 + p.halo) * p.PW + p.TM * kTileM + (c.kw - 1) + 7) / 8 * 8;
+    // (room must remain for the filters and for a staging ring of two tiles' rows)
+    const int64_t strip_need = (int64_t)strip_ppix * p.Cp + (int64_t)p.T * p.Cp * p.Np +
+                               (int64_t)2 * (p.RT + p.halo) * 32 * c.W * 4 + 8192;
+    p.strip = (strip_tiles >= 2 && strip_tiles * (p.Cp / 32) <= 2 * kMaxGroups &&
+               strip_need <= (int64_t)kSmemLimit) ? 1 : 0;
+    if (p.strip) p.ppix = strip_ppix;
     p.Nc = (uint32_t)((c.N + 15) / 16 * 16);
     p.cbase = (uint32_t)(2 * p.TM * p.Np);
     p.const_tmem = (p.cbase + 3 * p.Nc <= 512) ? 1 : 0;
@@ -141,7 +165,7 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms, bool next = false)
     uint32_t o = 0;
     const uint32_t a_bytes = (uint32_t)(p.Cp / 16) * p.ppix * 16;
     p.off_a[0] = o; o += a_bytes;
-    p.off_a[1] = o; o += a_bytes;
+    p.off_a[1] = p.strip ? p.off_a[0] : o; o += p.strip ? 0 : a_bytes;
     p.off_w = o;    o += (uint32_t)p.T * (p.Cp / 16) * p.Np * 16;
     p.off_lo = o;   o += (uint32_t)p.Cp * 4;
     p.off_hi = o;   o += (uint32_t)p.Cp * 4;
@@ -162,7 +186,9 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms, bool next = false)
         // steady-state batches in flight measured fastest (a deeper ring lost 3 %), so the ring is
         // capped at two tiles' worth of new rows.
         int ns = base < kSmemLimit ? (int)((kSmemLimit - base) / p.box_bytes) : 0;
-        const int cap = 2 * p.RT > p.RT + p.halo ? 2 * p.RT : p.RT + p.halo;
+        // (with the whole strip's codes resident the converters free a slot as soon as it lands: the ring is
+        // then as deep as shared memory allows, which is what keeps enough bytes in flight from the start)
+        const int cap = p.strip ? kMaxSlots * 2 : 2 * p.RT > p.RT + p.halo ? 2 * p.RT : p.RT + p.halo;
         if (ns > cap) ns = cap;
         if (ns >= p.RT + p.halo) {
             p.use_tma = 1; p.stages = kMaxStages; p.nslots = ns; p.off_stage = base;
@@ -320,6 +346,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
 
     // ---------------------------------------------------------------- set-up (all threads)
+    RTN_TL_INIT(conv_i8)
+    if (threadIdx.x == 0) RTN_TL(conv_i8, 0);
     tc::pdl_trigger();
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
@@ -342,6 +370,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
+    if (threadIdx.x == 0) RTN_TL(conv_i8, 1);
 
     if (is_conv_warp(warp)) {
         // ------------------------------------------------------------ converters
@@ -370,13 +399,15 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         int it = 0;
         for (int g = s0; g < s1; g += it == 0 ? p.R0 : p.RT, ++it) {
             const int buf = it & 1;
-            uint4* sA = reinterpret_cast<uint4*>(smem + (buf ? p.off_a[1] : p.off_a[0]));      // [Cp/16][ppix]
+            // [Cp/16][ppix]; with the whole strip resident the tile's window starts at its first row
+            uint4* sA = reinterpret_cast<uint4*>(smem + (buf ? p.off_a[1] : p.off_a[0])) + (p.strip ? (g - s0) * p.PW : 0);
             const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
             const int slot0 = it == 0 ? 0 : p.halo;            // first row slot that is new
             const int pp0 = slot0 * p.PW, pp1 = (nrows + p.halo) * p.PW;
             // (the barrier inside also orders this tile after every converter's writes to the previous buffer)
-            role_wait(tid < 32, &a_empty[buf], ((it >> 1) & 1) ^ 1, a.status, dead, kConvBarrier, kConvThreads);
-            if (it > 0) {
+            if (!p.strip) role_wait(tid < 32, &a_empty[buf], ((it >> 1) & 1) ^ 1, a.status, dead, kConvBarrier, kConvThreads);
+            if (tid == 0 && it < 8) RTN_TL(conv_i8, 24 + 2 * it);
+            if (it > 0 && !p.strip) {
                 // the kh-1 rows shared with the previous tile: copy their codes
                 const uint4* prev = reinterpret_cast<const uint4*>(smem + (buf ? p.off_a[0] : p.off_a[1]));
                 const int ncopy = p.halo * p.PW;
@@ -420,6 +451,51 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     role_wait(tid < 32, &st_full[s], (st_count / (uint32_t)kMaxStages) & 1, a.status, dead,
                               kConvBarrier, kConvThreads);
                     const float* ring = reinterpret_cast<const float*>(smem + p.off_stage);
+                    if (tid == 0 && it < 6 && grp < 2) RTN_TL(conv_i8, 72 + 4 * it + 2 * grp);
+                    if (p.PW >= kRowwiseMinPW) {
+                        // Wide rows: a warp takes a whole (row slot, 16-channel half) and its lanes walk the
+                        // row's padded columns, so the row's image, ring slot and validity are worked out once
+                        // per warp and row instead of once per value group (index arithmetic was the larger
+                        // part of this loop's instructions).
+                        const int nnew = nrows + p.halo - slot0;
+                        const int W = a.W, PW = p.PW, pad = a.pad;
+                        for (int u = tid >> 5; u < 2 * nnew; u += kConvWarps) {
+                            const int rowi = u >> 1, hf = u & 1;
+                            const int sl = slot0 + rowi;
+                            const uint32_t G = (uint32_t)(g + sl);
+                            const uint32_t b = fdiv(G, p.div_ph);
+                            const int r = (int)(G - b * (uint32_t)p.PH) - pad;
+                            const bool row_ok = b < (uint32_t)a.B && r >= 0 && r < a.H;
+                            int rs = row_base + rowi;
+                            if (rs >= p.nslots) rs -= p.nslots;
+                            const int ch = 2 * grp + hf;
+                            const float* src_row = ring + ((uint32_t)rs * 32u + 16u * hf) * (uint32_t)W;
+                            uint4* dst = sA + ch * p.ppix + sl * PW;
+                            // two columns per lane at a time: 32 shared-memory loads in flight per thread
+                            for (int cp0 = lane; cp0 < PW; cp0 += 64) {
+                                const int cp1 = cp0 + 32;
+                                uint4 w0 = make_uint4(0, 0, 0, 0), w1 = w0;
+                                if (row_ok) {
+                                    const bool ok0 = cp0 >= pad && cp0 < pad + W, ok1 = cp1 >= pad && cp1 < pad + W;
+                                    const float* q0 = src_row + (ok0 ? cp0 - pad : 0);      // always inside the slot
+                                    const float* q1 = src_row + (ok1 ? cp1 - pad : 0);
+                                    float v0[16], v1[16];
+                                    #pragma unroll
+                                    for (int e = 0; e < 16; ++e) v0[e] = q0[perm16(e) * W];
+                                    #pragma unroll
+                                    for (int e = 0; e < 16; ++e) v1[e] = q1[perm16(e) * W];
+                                    const uint4 t0 = per_layer ? codes16<true>(v0, sLo, sHi, ch * 16, lo0, hi0)
+                                                               : codes16<false>(v0, sLo, sHi, ch * 16, lo0, hi0);
+                                    const uint4 t1 = per_layer ? codes16<true>(v1, sLo, sHi, ch * 16, lo0, hi0)
+                                                               : codes16<false>(v1, sLo, sHi, ch * 16, lo0, hi0);
+                                    w0 = make_uint4(ok0 ? t0.x : 0u, ok0 ? t0.y : 0u, ok0 ? t0.z : 0u, ok0 ? t0.w : 0u);
+                                    w1 = make_uint4(ok1 ? t1.x : 0u, ok1 ? t1.y : 0u, ok1 ? t1.z : 0u, ok1 ? t1.w : 0u);
+                                }
+                                dst[cp0] = w0;
+                                if (cp1 < PW) dst[cp1] = w1;
+                            }
+                        }
+                    } else
                     // item = (padded pixel, half of the group's 32 channels)
                     for (int i = tid; i < 2 * npix; i += kConvThreads) {
                         const int hf = i >= npix ? 1 : 0;
@@ -444,9 +520,10 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                         }
                         sA[ch * p.ppix + pp] = w;
                     }
+                    if (tid == 0 && it < 6 && grp < 2) RTN_TL(conv_i8, 73 + 4 * it + 2 * grp);
                     tc::mbar_arrive(&st_empty[s]);
                     tc::fence_smem_to_async_proxy();
-                    tc::mbar_arrive(&a_full[buf * kMaxGroups + grp]);
+                    tc::mbar_arrive(&a_full[p.strip ? it * ngroup + grp : buf * kMaxGroups + grp]);
                     row_base += nrows + p.halo - slot0;
                     if (row_base >= p.nslots) row_base -= p.nslots;
                 }
@@ -474,14 +551,18 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             }
             if (!p.use_tma) {
                 tc::fence_smem_to_async_proxy();
-                for (int grp = 0; grp < ngroup; ++grp) tc::mbar_arrive(&a_full[buf * kMaxGroups + grp]);
+                for (int grp = 0; grp < ngroup; ++grp)
+                    tc::mbar_arrive(&a_full[p.strip ? it * ngroup + grp : buf * kMaxGroups + grp]);
             }
+            if (tid == 0 && it < 8) RTN_TL(conv_i8, 25 + 2 * it);
         }
     } else if (warp == kProdWarp) {
         // ------------------------------------------------------------ producer
         if (p.use_tma) {
-            tc::pdl_wait();                         // x may be the previous kernel's output
             const int ngroup = p.Cp / 32;
+            // the tensor map sits in the kernel's parameters: fetch it while the previous kernel drains
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
+            tc::pdl_wait();                         // x may be the previous kernel's output
             uint32_t st_count = 0;              // batches issued
             uint32_t rel = 0;                   // batches known to be released by the converters
             int rel_it = 0, rel_grp = 0;        // (tile, channel group) of batch `rel`
@@ -504,6 +585,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 __syncwarp();
                 sRows[lane] = info;
                 __syncwarp();
+                if (lane == 0 && it < 8) RTN_TL(conv_i8, 8 + 2 * it);
                 for (int grp = 0; grp < ngroup && alive; ++grp, ++st_count) {
                     // room in the ring and a free pair of barriers: retire the oldest batches
                     while (used + nnew > p.nslots || st_count - rel >= (uint32_t)kMaxStages) {
@@ -542,6 +624,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     used += nnew;
                     __syncwarp();
                 }
+                if (lane == 0 && it < 8) RTN_TL(conv_i8, 9 + 2 * it);
             }
         }
     } else if (warp == kMmaWarp) {
@@ -570,13 +653,16 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
                 const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;          // sub-tiles with any row
                 if (!wait_or_die(&acc_empty[buf], ph ^ 1, a.status, dead)) break;
-                const uint32_t a16 = tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4;
+                const uint32_t a16 = (tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4) +
+                                     (p.strip ? (uint32_t)((g - s0) * p.PW) : 0u);
                 bool alive = true;
                 // channel group by channel group, as the converters finish them
                 for (int grp = 0; grp < p.Cp / 32 && alive; ++grp) {
-                    alive = wait_or_die(&a_full[buf * kMaxGroups + grp], ph, a.status, dead);
+                    alive = wait_or_die(&a_full[p.strip ? it * (p.Cp / 32) + grp : buf * kMaxGroups + grp], p.strip ? 0u : ph,
+                                        a.status, dead);
                     if (!alive) break;
                     tc::tc_fence_after_sync();
+                    if (grp == 0 && it < 8) RTN_TL(conv_i8, 40 + 2 * it);
                     for (int tm = 0; tm < ntm; ++tm) {
                         const uint32_t d = tmem + (uint32_t)((buf * p.TM + tm) * p.Np);
                         const uint32_t a_tm = a16 + (uint32_t)(tm * kTileM) + a_lbo_field;
@@ -609,6 +695,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 if (!alive) break;
                 tc::mma_commit(&a_empty[buf]);
                 tc::mma_commit(&acc_full[buf]);
+                if (it < 8) RTN_TL(conv_i8, 41 + 2 * it);
             }
         }
     } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
@@ -660,6 +747,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         }
         tc::fence_smem_to_async_proxy();
         tc::mbar_arrive(w_ready);
+        if (etid == 0) RTN_TL(conv_i8, 2);
         {   // per-output-channel constants in double, rounded once (first needed by the first epilogue):
             //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
             const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
@@ -687,6 +775,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         }
         asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible
         tc::pdl_wait();                             // out may still be read by the previous kernel
+        if (etid == 0) RTN_TL(conv_i8, 3);
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;      // kEpiWarp0 is a multiple of 4
         const int64_t ostride = (int64_t)a.Ho * a.Wo;
         const int nblk16 = (a.N + 15) / 16;
@@ -718,6 +807,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             role_wait(warp == kEpiWarp0, &acc_full[buf], (it >> 1) & 1, a.status, dead, kEpiBarrier, kEpiThreads);
             const bool alive = !*dead;
             tc::tc_fence_after_sync();
+            if (etid == 0 && it < 8) RTN_TL(conv_i8, 56 + 2 * it);
             if constexpr (kNext) {
                 next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, buf, g, nrows,
                                    alive, q, lane, half);
@@ -749,6 +839,9 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 for (int blk = blk_begin; blk < blk_end; ++blk) {
                     const int n0 = blk * 16;
                     if (n0 + 16 <= a.N) {
+                        // running pointers: one 64-bit add per store instead of a 64-bit product and a shift
+                        float* q0 = optr2[0] + (int64_t)n0 * ostride;
+                        float* q1 = optr2[1] + (int64_t)n0 * ostride;
                         #pragma unroll
                         for (int h8 = 0; h8 < 16; h8 += 8) {
                             uint32_t u0[8], u1[8], k1[8], k2[8], k3[8];
@@ -760,17 +853,15 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                             tc::tmem_ld_wait();
                             if (ok2[0]) {
                                 #pragma unroll
-                                for (int j = 0; j < 8; ++j)
-                                    optr2[0][(int64_t)(n0 + h8 + j) * ostride] =
-                                        fmaf(__uint_as_float(k1[j]), (float)(int)u0[j],
-                                             fmaf(__uint_as_float(k2[j]), fsx0, __uint_as_float(k3[j])));
+                                for (int j = 0; j < 8; ++j, q0 += ostride)
+                                    *q0 = fmaf(__uint_as_float(k1[j]), (float)(int)u0[j],
+                                               fmaf(__uint_as_float(k2[j]), fsx0, __uint_as_float(k3[j])));
                             }
                             if (ok2[1]) {
                                 #pragma unroll
-                                for (int j = 0; j < 8; ++j)
-                                    optr2[1][(int64_t)(n0 + h8 + j) * ostride] =
-                                        fmaf(__uint_as_float(k1[j]), (float)(int)u1[j],
-                                             fmaf(__uint_as_float(k2[j]), fsx1, __uint_as_float(k3[j])));
+                                for (int j = 0; j < 8; ++j, q1 += ostride)
+                                    *q1 = fmaf(__uint_as_float(k1[j]), (float)(int)u1[j],
+                                               fmaf(__uint_as_float(k2[j]), fsx1, __uint_as_float(k3[j])));
                             }
                         }
                     } else {
@@ -898,11 +989,13 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[buf]);
+            if (etid == 0 && it < 8) RTN_TL(conv_i8, 57 + 2 * it);
         }
     }
     tc::tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
+    if (threadIdx.x == 0) RTN_TL(conv_i8, 4);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)

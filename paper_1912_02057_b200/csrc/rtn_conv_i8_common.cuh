@@ -33,7 +33,7 @@ __device__ __forceinline__ bool wait_or_die(uint64_t* bar, uint32_t parity, unsi
     if (tc::mbar_try_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < tc::kWaitPolls; ++i) {
         if (tc::mbar_try_wait(bar, parity)) return true;
-        if (*dead) return false;
+        if ((i & 15u) == 15u && *dead) return false;        // a look at the flag now and then keeps the poll short
     }
     *dead = 1;
     atomicOr(status, kStatusWaitTimeout);
