@@ -272,12 +272,16 @@ rtn_status rtn_selftest_wait_timeout(int64_t polls, int32_t* gave_up, void* stre
  *   rtn_probe_peak_popc rounds (1..2^24) rounds per thread of 64 word pairs, 1024 threads per CTA, registers
  *                       only; rtn_probe_popc_ops_per_round() operations (2 per code pair) per CTA and round.
  *                       `sink`: device int32 the kernel never writes in practice (keeps the loop alive).
- * Both only enqueue. */
+ *   rtn_probe_copy      copies `bytes` (a multiple of 16; both pointers 16-byte aligned) from src to dst with two
+ *                       CTAs of 1024 threads per multiprocessor, 16 bytes per thread and trip: the time a kernel
+ *                       that only moves a layer's input and output takes at that size.
+ * All only enqueue. */
 int64_t rtn_probe_ctas(void);
 int64_t rtn_probe_i8_ops_per_mma(void);
 int64_t rtn_probe_popc_ops_per_round(void);
 rtn_status rtn_probe_peak_i8(int64_t n_mma, int64_t* cycles, void* stream);
 rtn_status rtn_probe_peak_popc(int64_t rounds, int64_t* cycles, int32_t* sink, void* stream);
+rtn_status rtn_probe_copy(const void* src, void* dst, int64_t bytes, void* stream);
 
 /* Static text for a status code. */
 const char* rtn_status_string(rtn_status s);

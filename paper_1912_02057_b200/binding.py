@@ -107,6 +107,8 @@ def lib():
         L.rtn_probe_peak_i8.argtypes = [_i64, _vp, _vp]
         L.rtn_probe_peak_popc.restype = _int
         L.rtn_probe_peak_popc.argtypes = [_i64, _vp, _vp, _vp]
+        L.rtn_probe_copy.restype = _int
+        L.rtn_probe_copy.argtypes = [_vp, _vp, _i64, _vp]
         L.rtn_selftest_wait_timeout.restype = _int
         L.rtn_selftest_wait_timeout.argtypes = [_i64, _vp, _vp]
         L.rtn_status_string.restype = C.c_char_p
@@ -342,3 +344,10 @@ def rtn_probe_peak_popc(rounds, stream=None):
     _check(lib().rtn_probe_peak_popc(int(rounds), _ptr(cycles, torch.int64), _ptr(sink, torch.int32), _stream(stream)),
            "rtn_probe_peak_popc")
     return cycles, int(rounds) * int(lib().rtn_probe_popc_ops_per_round())
+
+
+def rtn_probe_copy(src, dst, stream=None):
+    """Plain device copy of src into dst (same size, a multiple of 16 bytes) by the library's copy probe."""
+    nbytes = src.numel() * src.element_size()
+    _check(lib().rtn_probe_copy(_ptr(src), _ptr(dst), nbytes, _stream(stream)), "rtn_probe_copy")
+    return dst

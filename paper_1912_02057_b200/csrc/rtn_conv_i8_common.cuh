@@ -146,7 +146,7 @@ __device__ __forceinline__ void next_layer_block16(const ConvArgs& a, const Next
     }
     if (f.relu) {
         #pragma unroll
-        for (int j = 0; j < 16; ++j) y[j] = y[j] > 0.f ? y[j] : 0.f;
+        for (int j = 0; j < 16; ++j) y[j] = fmaxf(y[j], 0.f);          // (a NaN becomes 0 either way)
     }
     if (f.skip != nullptr) {
         float sk[16];
@@ -168,13 +168,21 @@ __device__ __forceinline__ void next_layer_block16(const ConvArgs& a, const Next
     }
     nzb = 0; sgb = 0;                          // one bit per column and plane
     if (want_codes) {
+        // The bits of a plane are summed as powers of two in fp32 (exact below 2^24): a comparison that yields
+        // 1.0f / 0.0f and one FMA per value and plane, against a predicate, a select and an OR each.  +1 is tested
+        // first: the sign plane is "y > t_hi" alone, and a value that is both above t_hi and below t_lo (possible
+        // only when t_lo > t_hi) has its non-zero bit set by either comparison.
+        float above0 = 0.f, above1 = 0.f, below0 = 0.f, below1 = 0.f;
         #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const float2 t = sT[j];
-            const bool pos = y[j] > t.y, neg = !pos && y[j] < t.x;
-            nzb |= (uint32_t)(pos || neg) << j;
-            sgb |= (uint32_t)pos << j;
+        for (int j = 0; j < 16; j += 2) {
+            const float2 t0 = sT[j], t1 = sT[j + 1];
+            above0 = fmaf(y[j] > t0.y ? 1.f : 0.f, (float)(1u << j), above0);
+            below0 = fmaf(y[j] < t0.x ? 1.f : 0.f, (float)(1u << j), below0);
+            above1 = fmaf(y[j + 1] > t1.y ? 1.f : 0.f, (float)(2u << j), above1);
+            below1 = fmaf(y[j + 1] < t1.x ? 1.f : 0.f, (float)(2u << j), below1);
         }
+        sgb = (uint32_t)(above0 + above1);
+        nzb = sgb | (uint32_t)(below0 + below1);
     }
 }
 

@@ -32,6 +32,12 @@
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
 #include "rtn_conv_i8_common.cuh"
+#include "rtn_timeline.cuh"
+
+// Timeline slots (instrumented build only; same plan as conv_i8_kernel): 0 kernel entry, 1 set-up done, 4 kernel end;
+// per tile i < 8: 24+2i / 25+2i ternarizer thread 0 begins / ends, 40+2i / 41+2i first MMA issued / accumulators
+// committed, 56+2i / 57+2i epilogue begins / ends.
+RTN_TL_DEFINE(conv_i8s)
 
 namespace rtn {
 
@@ -258,6 +264,8 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
     const int ntile = (s1 - s0 + p.RT - 1) / p.RT;
     const int rt = ntile > 0 ? (s1 - s0 + ntile - 1) / ntile : 1;
 
+    RTN_TL_INIT(conv_i8s)
+    if (threadIdx.x == 0) RTN_TL(conv_i8s, 0);
     tc::pdl_trigger();
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
@@ -310,6 +318,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
     tc::pdl_wait();         // from here on: x, out (the set-up above read only the layer's parameters)
+    if (threadIdx.x == 0) RTN_TL(conv_i8s, 1);
 
     if (warp >= 1 && warp < 1 + kTernWarps) {
         // ------------------------------------------------------------ ternarizers / epilogue
@@ -335,6 +344,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             const int npix = (nrows + p.halo) * p.PW;
             int* psum = sPsum + (it & (kPsumRing - 1)) * p.ppix;
             role_wait(tid < 32, &a_empty[buf], use_ph ^ 1, a.status, dead, kTernBarrier, kTernThreads);
+            if (tid == 0 && it < 8) RTN_TL(conv_i8s, 24 + 2 * it);
             for (int i = tid; i < p.ppix; i += kTernThreads) psum[i] = 0;
             asm volatile("bar.sync %0, %1;" ::"r"(kTernBarrier), "r"(kTernThreads) : "memory");
             uint64_t* full = &a_full[buf * kMaxGroups];
@@ -394,6 +404,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                     for (; arrived < h && arrived < ngroup; ++arrived) tc::mbar_arrive(&full[arrived]);
                 }
             }
+            if (tid == 0 && it < 8) RTN_TL(conv_i8s, 25 + 2 * it);
             }
             if (step >= 1 && epi_warp) {
                 const int it = step - 1, g = s0 + it * rt;
@@ -408,6 +419,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             role_wait(warp == kEpiWarp0, &acc_full[slot_acc], acc_ph, a.status, dead, kEpiBarrier, kEpiThreads);
             const bool alive = !*dead;
             tc::tc_fence_after_sync();
+            if (warp == kEpiWarp0 && lane == 0 && pass == 0 && it < 8) RTN_TL(conv_i8s, 56 + 2 * it);
             const int pass_blocks = p.npass == 2 ? min(p.NpP / 16, nblk16 - pass * (p.NpP / 16)) : nblk16;
             const int pb_begin = half == 0 ? 0 : (pass_blocks + 1) / 2;
             const int pb_end = half == 0 ? (pass_blocks + 1) / 2 : pass_blocks;
@@ -499,6 +511,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[acc]);
+            if (warp == kEpiWarp0 && lane == 0 && pass == p.npass - 1 && it < 8) RTN_TL(conv_i8s, 57 + 2 * it);
           }
             }
         }
@@ -626,6 +639,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                             if (alive) {
                                 const uint64_t bd = desc_hi | (uint64_t)(w16 + st * wstage16 + (uint32_t)j * wslice16);
                                 const uint32_t aw = a16 + (ta[j] & 0xFFFFFFu);
+                                if (!accum && pass == 0 && it < 8) RTN_TL(conv_i8s, 40 + 2 * it);
                                 tc::mma_i8_ss(tmem + (uint32_t)((slot_acc * p.TM) * p.NpP), desc_hi | (uint64_t)aw, bd, idesc, accum);
                                 if (ntm == 2)
                                     tc::mma_i8_ss(tmem + (uint32_t)((slot_acc * p.TM + 1) * p.NpP),
@@ -637,6 +651,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                     if (alive) tc::mma_commit(&w_empty[st]);
                 }
                 if (alive) tc::mma_commit(&acc_full[slot_acc]);      // this pass's accumulators are complete
+                if (pass == p.npass - 1 && it < 8) RTN_TL(conv_i8s, 41 + 2 * it);
               }
                 if (!alive) break;
                 tc::mma_commit(&a_empty[buf]);
@@ -646,6 +661,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
     tc::tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
+    if (threadIdx.x == 0) RTN_TL(conv_i8s, 4);
 }
 
 }  // namespace

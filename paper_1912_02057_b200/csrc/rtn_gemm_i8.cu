@@ -19,6 +19,12 @@
 // 128 contiguous bytes and consecutive threads (rows) store consecutive 16-byte slots.
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
+#include "rtn_timeline.cuh"
+
+// Timeline slots (instrumented build only): 0 kernel entry, 1 set-up done (expanded operands visible), 4 kernel end;
+// per tile i < 8 of the CTA: 40+2i first stage of the tile ready for the tensor core, 41+2i accumulators committed,
+// 56+2i / 57+2i epilogue (thread 0 of its first warp) begins / ends.
+RTN_TL_DEFINE(gemm_i8)
 #include "rtn_conv_i8_common.cuh"
 
 namespace rtn {
@@ -165,6 +171,8 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
     const int64_t nblk = (g.K + kBlockCodes - 1) / kBlockCodes;
     const int rowsA = p.TM * 128;
 
+    RTN_TL_INIT(gemm_i8)
+    if (threadIdx.x == 0) RTN_TL(gemm_i8, 0);
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
         for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], kPreA ? kMaxEpiWarps * 32 : kEpiThreads); }
@@ -177,6 +185,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
     if constexpr (kPreW) tc::pdl_wait();           // the expanded weights come from the kernel before
+    if (threadIdx.x == 0) RTN_TL(gemm_i8, 1);
 
     if (!kPreA && warp >= kExpWarp0) {
         // ------------------------------------------------------------ expanders
@@ -290,6 +299,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
                     const uint32_t s = count % (uint32_t)p.stages;
                     if (!wait_or_die(&full[s], (count / (uint32_t)p.stages) & 1, g.status, dead)) { alive = false; break; }
                     tc::tc_fence_after_sync();
+                    if (kb == 0 && tc_ < 8) RTN_TL(gemm_i8, 40 + 2 * (int)tc_);
                     const uint32_t a16 = stage16 + s * (p.stage_bytes >> 4) + a_lbo;
                     const uint32_t b16 = stage16 + s * (p.stage_bytes >> 4) + (uint32_t)(rowsA * 8) + b_lbo;
                     uint32_t la[8], lb[4];
@@ -310,6 +320,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
                     tc::mma_commit(&empty[s]);
                 }
                 if (alive) tc::mma_commit(&acc_full[acc]);
+                if (tc_ < 8) RTN_TL(gemm_i8, 41 + 2 * (int)tc_);
             }
         }
     } else if (warp >= kEpiWarp0) {
@@ -345,6 +356,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
             asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(nEpiThreads) : "memory");
             const bool alive = wait_or_die(&acc_full[acc], acc_ph, g.status, dead);
             tc::tc_fence_after_sync();
+            if (etid == 0 && tc_ < 8) RTN_TL(gemm_i8, 56 + 2 * (int)tc_);
             const int per = ((p.BN + nParts - 1) / nParts + 15) / 16 * 16;     // columns per range, whole blocks of 16
             const int c_begin = part * per < p.BN ? part * per : p.BN;
             const int c_end = c_begin + per < p.BN ? c_begin + per : p.BN;
@@ -406,11 +418,13 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[acc]);
+            if (etid == 0 && tc_ < 8) RTN_TL(gemm_i8, 57 + 2 * (int)tc_);
         }
     }
     tc::tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
+    if (threadIdx.x == 0) RTN_TL(gemm_i8, 4);
 }
 
 // Pre-expansion mode of a plan: 0 = both operands expanded inside the kernel (one row tile: every weight row

@@ -99,6 +99,15 @@ probe_popc_kernel(uint32_t rounds, long long* cycles, int* sink)
     if (both - 2 * differ == 0x7FFFFFFF) *sink = 1;            // keeps the loop alive; never true
 }
 
+// Plain copy, 16 bytes per thread and trip: what a kernel that only moves a layer's input and output can reach at
+// that size (launch ramp and tail included), the yardstick for the HBM-bound conv shapes.
+__global__ void __launch_bounds__(1024, 2)
+probe_copy_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16)
+{
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride) dst[i] = src[i];
+}
+
 }  // namespace
 
 }  // namespace rtn
@@ -123,6 +132,16 @@ rtn_status rtn_probe_peak_i8(int64_t n_mma, int64_t* cycles, void* stream)
     if (word == nullptr) return RTN_ERR_CUDA;
     rtn::probe_i8_kernel<<<(unsigned)rtn::device_sm_count(), rtn::kProbeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         (uint32_t)n_mma, reinterpret_cast<long long*>(cycles), word);
+    return cudaGetLastError() == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
+}
+
+rtn_status rtn_probe_copy(const void* src, void* dst, int64_t bytes, void* stream)
+{
+    if (src == nullptr || dst == nullptr) return RTN_ERR_NULL;
+    if (bytes <= 0 || bytes % 16 != 0) return RTN_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(src) % 16 != 0 || reinterpret_cast<uintptr_t>(dst) % 16 != 0) return RTN_ERR_ALIGN;
+    rtn::probe_copy_kernel<<<(unsigned)(2 * rtn::device_sm_count()), 1024, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(src), static_cast<uint4*>(dst), (size_t)bytes / 16);
     return cudaGetLastError() == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
 }
 

@@ -6,13 +6,15 @@
 
 The CSV is the log of
 
-    ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none -k regex:REGEX -c <several> \\
-        --csv --log-file launches.csv python bench.py --workload WORKLOAD --eager --steps <several> ...
+    ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none --cache-control none \\
+        -k regex:REGEX -s <warm-up launches> -c <several> --csv --log-file launches.csv \\
+        python bench.py --workload WORKLOAD --eager --steps 4 --warmup 3 --no-cpu-baseline
 
-over several CONSECUTIVE launches of the kernel on the benchmark's rotating buffers: a kernel's fp32 output is
-still in L2 when it ends, so one launch alone shows almost no writes; summed over consecutive launches the
-write-back of one launch falls into the window of the next, and the total divided by the launches is the
-traffic of a launch.  The record keeps a SHA-256 of every source file the kernel is built from; ``bench.py``
+over several CONSECUTIVE launches of the kernel on the benchmark's rotating buffers, WITHOUT the profiler's cache
+flush between launches (--cache-control none): a kernel's fp32 output is still in L2 when it ends, so one launch
+alone (or every launch, when the caches are flushed outside the counted window) shows almost no writes; with
+the caches left alone the write-back of one launch falls into the window of the next ones, and the total
+divided by the launches is the traffic of a launch (both counters come from one pass).  The record keeps a SHA-256 of every source file the kernel is built from; ``bench.py``
 prints ``traffic: null`` once one of them has changed since the capture.
 """
 import argparse
