@@ -34,6 +34,7 @@
 #include "rtn_tcgen05.cuh"
 #include "rtn_conv_i8_common.cuh"
 #include "rtn_timeline.cuh"
+#include "rtn_tensormap.cuh"
 
 #include <cuda.h>
 #include <string.h>
@@ -996,25 +997,6 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
     __syncthreads();
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
     if (threadIdx.x == 0) RTN_TL(conv_i8, 4);
-}
-
-// cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
 }
 
 }  // namespace

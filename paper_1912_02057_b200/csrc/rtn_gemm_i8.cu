@@ -20,6 +20,7 @@
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
 #include "rtn_timeline.cuh"
+#include "rtn_tensormap.cuh"
 
 // Timeline slots (instrumented build only): 0 kernel entry, 1 set-up done (expanded operands visible), 4 kernel end;
 // per tile i < 8 of the CTA: 40+2i first stage of the tile ready for the tensor core, 41+2i accumulators committed,
@@ -48,6 +49,13 @@ constexpr int kEpiBarrier = 3;
 constexpr int kStageRow = 48;
 constexpr int kStageWarp = 32 * kStageRow;
 constexpr int kMaxEpiWarps = kEpiWarps + kExpWarps;     // with both operands expanded ahead the expander warps join
+// Output through TMA stores: a warp stages 32 rows x 16 columns of fp32 (64-byte rows, the 64-byte swizzle of the
+// tensor map: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3), which also makes a quarter warp's row-wise
+// writes fall on distinct banks) and one thread hands the block to the copy engine, which writes whole row segments
+// while the warp works on the next block.  No global store instruction and no address arithmetic in the warp.
+constexpr int kTmaStageWarp = 32 * 64;
+constexpr int kTmaCols = 16;
+constexpr int kTmaWarpsPre = 12;                        // warps that write out when the expander warps are free to help
 
 struct GemmI8Plan {
     int TM;                 // 128-row sub-tiles per tile
@@ -60,6 +68,7 @@ struct GemmI8Plan {
     uint32_t tmem_cols;
     uint32_t stage_bytes, off_stage, off_c, off_bar, off_misc, off_t;
     size_t smem_bytes;
+    int tma_out;            // the epilogue writes the output with TMA stores (set by the launcher)
 };
 
 bool make_gemm_plan(int64_t M, int64_t N, int64_t K, GemmI8Plan& p, int sms)
@@ -97,7 +106,11 @@ bool make_gemm_plan(int64_t M, int64_t N, int64_t K, GemmI8Plan& p, int sms)
     p.off_c = o;    o += (uint32_t)p.BN * 16;                  // float4 {p1, p2, p3, 0} per column
     p.off_bar = o;  o += (4 + 2 * kMaxStages) * 8;             // acc_full[2] acc_empty[2] full[] empty[]
     p.off_misc = o; o += 16;
-    p.off_t = o;    o += kMaxEpiWarps * kStageWarp;             // 16-byte aligned: every term above is
+    o = (o + 1023) / 1024 * 1024;                              // the swizzled staging blocks want 1 KB alignment
+    p.off_t = o;                                               // staging of either way of writing out
+    o += kMaxEpiWarps * kStageWarp > 1024 + kTmaWarpsPre * kTmaStageWarp ? kMaxEpiWarps * kStageWarp
+                                                                           : 1024 + kTmaWarpsPre * kTmaStageWarp;
+    p.tma_out = 0;
     o = (o + 127) / 128 * 128;
     p.off_stage = o;
     int ns = (int)((kSmemLimit - o) / p.stage_bytes);
@@ -155,7 +168,7 @@ gemm_expand_operands_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan
 template <bool kPreW, bool kPreA>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uint4* __restrict__ wexp,
-               const uint4* __restrict__ aexp)
+               const uint4* __restrict__ aexp, const __grid_constant__ CUtensorMap omap)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     float4* sC = reinterpret_cast<float4*>(smem + p.off_c);
@@ -334,6 +347,10 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
         uint8_t* sT = smem + p.off_t + (warp - kEpiWarp0) * kStageWarp;
         // whole-row float4 stores need every row start on a 16-byte boundary (the same for all lanes)
         const bool vec_ok = g.dbg_acc == nullptr && (g.N & 3) == 0 && (((uintptr_t)g.out) & 15) == 0;
+        // TMA-store staging block of this warp (the first 8 or, with the expander warps free, 12 warps write out;
+        // 1 KB aligned shared address)
+        const uint32_t tma_stage = ((tc::smem_addr(smem + p.off_t) + 1023u) & ~1023u) + (uint32_t)(warp - kEpiWarp0) * kTmaStageWarp;
+        const int parts_used = p.tma_out ? (kPreA ? kTmaWarpsPre : kEpiWarps) / 4 : nParts;
         uint32_t tc_ = 0;
         for (int64_t tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++tc_) {
             const int acc = p.nAcc == 2 ? (tc_ & 1) : 0;
@@ -357,7 +374,7 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
             const bool alive = wait_or_die(&acc_full[acc], acc_ph, g.status, dead);
             tc::tc_fence_after_sync();
             if (etid == 0 && tc_ < 8) RTN_TL(gemm_i8, 56 + 2 * (int)tc_);
-            const int per = ((p.BN + nParts - 1) / nParts + 15) / 16 * 16;     // columns per range, whole blocks of 16
+            const int per = ((p.BN + parts_used - 1) / parts_used + 15) / 16 * 16;     // columns per range, whole blocks of 16
             const int c_begin = part * per < p.BN ? part * per : p.BN;
             const int c_end = c_begin + per < p.BN ? c_begin + per : p.BN;
             for (int tm = 0; tm < p.TM; ++tm) {
@@ -377,6 +394,32 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
                     uint32_t v[16];
                     tc::tmem_ld16(trow + (uint32_t)c0, v);
                     tc::tmem_ld_wait();
+                    if (p.tma_out) {
+                        // (uniform over the kernel) columns past N and rows past M are clipped by the copy engine
+                        float r[kTmaCols];
+                        #pragma unroll
+                        for (int j = 0; j < kTmaCols; ++j) {
+                            const float4 c = sC[c0 + j];
+                            r[j] = fmaf(a_s, fmaf(c.x, (float)(int)v[j], c.y * s_x), a_o * c.z);
+                        }
+                        // the copy of the block before has read the staging block
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+                        #pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            const uint32_t dst = tma_stage + (uint32_t)lane * 64u + (uint32_t)((ch ^ ((lane >> 1) & 3)) << 4);
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};"
+                                         ::"r"(dst), "f"(r[4 * ch]), "f"(r[4 * ch + 1]), "f"(r[4 * ch + 2]), "f"(r[4 * ch + 3]) : "memory");
+                        }
+                        tc::fence_smem_to_async_proxy();
+                        __syncwarp();
+                        if (lane == 0 && alive && mbase < g.M && n0 + c0 < g.N) {
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(reinterpret_cast<uint64_t>(&omap)), "r"((int)(n0 + c0)), "r"((int)mbase), "r"(tma_stage)
+                                         : "memory");
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        }
+                    } else
                     if (vec_ok && n0 + c0 + 16 <= g.N) {
                         // A lane holds 16 columns of ONE row; stored as is, a warp store would touch 32 rows
                         // with 16 bytes each.  Through the staging block (8 columns at a time) a store covers
@@ -420,6 +463,8 @@ gemm_i8_kernel(const GemmArgs g, const __grid_constant__ GemmI8Plan p, const uin
             tc::mbar_arrive(&acc_empty[acc]);
             if (etid == 0 && tc_ < 8) RTN_TL(gemm_i8, 57 + 2 * (int)tc_);
         }
+        // the copies this thread handed over have written their rows before the CTA ends
+        if (p.tma_out && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
     tc::tc_fence_before_sync();
     __syncthreads();
@@ -459,10 +504,25 @@ cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s)
     GemmI8Plan p;
     if (!make_gemm_plan(g.M, g.N, g.K, p, device_sm_count())) return cudaErrorInvalidConfiguration;
     const int mode = gemm_pre_mode(p, g.K);
+    // Output as a 2-D tensor for the epilogue's TMA stores: rows of N floats, boxes of 32 rows x 16 columns,
+    // 64-byte swizzle.  Needs 16-byte aligned rows; the debug output keeps the store-instruction epilogue.
+    CUtensorMap omap;
+    memset(&omap, 0, sizeof(omap));
+    if (g.dbg_acc == nullptr && (g.N & 3) == 0 && g.N >= kTmaCols && (reinterpret_cast<uintptr_t>(g.out) & 15) == 0) {
+        EncodeTiledFn enc = encode_tiled_fn();
+        const cuuint64_t dims[2] = {(cuuint64_t)g.N, (cuuint64_t)g.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)g.N * 4};
+        const cuuint32_t box[2] = {(cuuint32_t)kTmaCols, 32};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc != nullptr &&
+            enc(&omap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, g.out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+            p.tma_out = 1;
+    }
     if (mode == 0) {
         cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
         if (e != cudaSuccess) return e;
-        gemm_i8_kernel<false, false><<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(g, p, nullptr, nullptr);
+        gemm_i8_kernel<false, false><<<(unsigned)p.grid, kThreads, p.smem_bytes, s>>>(g, p, nullptr, nullptr, omap);
         return cudaGetLastError();
     }
     // scratch from the stream-ordered allocator: N (and M) rounded up to tiles, times K rounded up to blocks, bytes
@@ -479,12 +539,12 @@ cudaError_t launch_gemm_i8(const GemmArgs& g, cudaStream_t s)
         e = cudaFuncSetAttribute(gemm_i8_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
         if (e == cudaSuccess)
             e = launch_pdl(gemm_i8_kernel<true, false>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, g, p,
-                           (const uint4*)wexp, (const uint4*)aexp);
+                           (const uint4*)wexp, (const uint4*)aexp, omap);
     } else if (e == cudaSuccess) {
         e = cudaFuncSetAttribute(gemm_i8_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
         if (e == cudaSuccess)
             e = launch_pdl(gemm_i8_kernel<true, true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, g, p,
-                           (const uint4*)wexp, (const uint4*)aexp);
+                           (const uint4*)wexp, (const uint4*)aexp, omap);
     }
     const cudaError_t e2 = cudaFreeAsync(scratch, s);
     return e != cudaSuccess ? e : e2;
