@@ -254,6 +254,73 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
     const int64_t ostride = (int64_t)a.Ho * a.Wo;
     const int nblk16 = (a.N + 15) / 16;
     const int ncb = (a.N + kBlockCodes - 1) / kBlockCodes;
+    const int nwords = a.N / 32;
+    if (ntm == 2 && a.pad_mode == RTN_PAD_CODE_ZERO && (a.N == 64 || a.N == 128)) {
+        // Full tile of a 64- or 128-filter layer without border classes: the two warps of a lane quarter split
+        // the output channels, and a thread takes its pixel of BOTH sub-tiles through its channels, 16 at a time
+        // (next_layer_block16_pair).  A warp writes its 32-bit words of each pixel's packed row; the words past N
+        // of a 64-filter row (its zero fill) are shared out between the two warps.
+        bool ok2[2];
+        uint32_t trow2[2];
+        int64_t obase2[2];
+        uint8_t* row2[2];
+        uint32_t sx2[2];
+        #pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const uint32_t pl = (uint32_t)(t * kTileM + q * 32 + lane);
+            const uint32_t row = fdiv(pl, p.div_pw);
+            const int wo = (int)(pl - row * (uint32_t)p.PW);
+            const uint32_t G = (uint32_t)g + row;
+            const uint32_t b = fdiv(G, p.div_ph);
+            const int ho = (int)(G - b * (uint32_t)p.PH);
+            ok2[t] = alive && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
+            trow2[t] = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + t) * p.Np);
+            obase2[t] = (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
+            row2[t] = (ok2[t] && f.out_packed != nullptr)
+                          ? f.out_packed + (((int64_t)b * a.Ho + ho) * a.Wo + wo) * (int64_t)(ncb * kBlockBytes) : nullptr;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
+                         : "=r"(sx2[t]) : "r"(trow2[t] + (uint32_t)a.N) : "memory");
+        }
+        tc::tmem_ld_wait();
+        const float fsx0 = (float)(int)sx2[0], fsx1 = (float)(int)sx2[1];
+        const bool want = f.out_packed != nullptr;
+        for (int w = half * (nwords / 2); w < (half + 1) * (nwords / 2); ++w) {
+            uint32_t nz0 = 0, sg0 = 0, nz1 = 0, sg1 = 0;
+            #pragma unroll 1
+            for (int hb = 0; hb < 2; ++hb) {
+                const int n0 = w * 32 + hb * 16;
+                uint32_t u0[16], u1[16];
+                tc::tmem_ld16(trow2[0] + (uint32_t)n0, u0);
+                tc::tmem_ld16(trow2[1] + (uint32_t)n0, u1);
+                tc::tmem_ld_wait();
+                uint32_t a0, b0, a1, b1;
+                next_layer_block16_pair(a, f, u0, u1, sC + n0, sT + n0, fsx0, fsx1, ok2[0], ok2[1],
+                                        obase2[0] + (int64_t)n0 * ostride, obase2[1] + (int64_t)n0 * ostride, ostride, want,
+                                        a0, b0, a1, b1);
+                nz0 |= a0 << (16 * hb); sg0 |= b0 << (16 * hb);
+                nz1 |= a1 << (16 * hb); sg1 |= b1 << (16 * hb);
+            }
+            const int off = (w >> 2) * kBlockBytes + (w & 3) * 4;
+            if (row2[0] != nullptr) {
+                *reinterpret_cast<uint32_t*>(row2[0] + off) = nz0;
+                *reinterpret_cast<uint32_t*>(row2[0] + off + 16) = sg0;
+            }
+            if (row2[1] != nullptr) {
+                *reinterpret_cast<uint32_t*>(row2[1] + off) = nz1;
+                *reinterpret_cast<uint32_t*>(row2[1] + off + 16) = sg1;
+            }
+        }
+        for (int w = nwords + half; w < ncb * 4; w += 2) {          // zero fill past N
+            const int off = (w >> 2) * kBlockBytes + (w & 3) * 4;
+            #pragma unroll
+            for (int t = 0; t < 2; ++t)
+                if (row2[t] != nullptr) {
+                    *reinterpret_cast<uint32_t*>(row2[t] + off) = 0u;
+                    *reinterpret_cast<uint32_t*>(row2[t] + off + 16) = 0u;
+                }
+        }
+        return;
+    }
     for (int tm = 0; tm < ntm; ++tm) {
         const uint32_t pl = (uint32_t)(tm * kTileM + q * 32 + lane);     // pixel within the tile
         const uint32_t row = fdiv(pl, p.div_pw);

@@ -186,6 +186,74 @@ __device__ __forceinline__ void next_layer_block16(const ConvArgs& a, const Next
     }
 }
 
+// The hand-over step for TWO pixels of a thread and one block of 16 output channels, all of which exist (layers
+// without border classes): every constant and threshold pair is fetched once and serves both pixels, and the two
+// pixels' arithmetic interleaves, which is what an epilogue bound by the round trips of its loads needs.
+// v0, v1: the block's accumulators of the two pixels; o0_0, o0_1: offsets of (b, n0, ho, wo) of each pixel;
+// ok0, ok1: the pixel exists (nothing is read or written for one that does not).
+__device__ __forceinline__ void next_layer_block16_pair(const ConvArgs& a, const NextLayerArgs& f,
+                                                        const uint32_t (&v0)[16], const uint32_t (&v1)[16],
+                                                        const float4* sC, const float2* sT, float fsx0, float fsx1,
+                                                        bool ok0, bool ok1, int64_t o0_0, int64_t o0_1, int64_t ostride,
+                                                        bool want_codes, uint32_t& nzb0, uint32_t& sgb0,
+                                                        uint32_t& nzb1, uint32_t& sgb1)
+{
+    nzb0 = sgb0 = nzb1 = sgb1 = 0;
+    #pragma unroll
+    for (int h = 0; h < 16; h += 8) {
+        float y0[8], y1[8];
+        #pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float4 c = sC[h + j];
+            y0[j] = fmaf(c.x, (float)(int)v0[h + j], fmaf(c.y, fsx0, c.z));
+            y1[j] = fmaf(c.x, (float)(int)v1[h + j], fmaf(c.y, fsx1, c.z));
+        }
+        if (f.relu) {
+            #pragma unroll
+            for (int j = 0; j < 8; ++j) { y0[j] = fmaxf(y0[j], 0.f); y1[j] = fmaxf(y1[j], 0.f); }
+        }
+        if (f.skip != nullptr) {
+            float s0[8], s1[8];
+            #pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                s0[j] = ok0 ? __ldg(f.skip + o0_0 + (int64_t)(h + j) * ostride) : 0.f;
+                s1[j] = ok1 ? __ldg(f.skip + o0_1 + (int64_t)(h + j) * ostride) : 0.f;
+            }
+            #pragma unroll
+            for (int j = 0; j < 8; ++j) { y0[j] += s0[j]; y1[j] += s1[j]; }
+        }
+        if (a.out != nullptr) {
+            #pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (ok0) a.out[o0_0 + (int64_t)(h + j) * ostride] = y0[j];
+                if (ok1) a.out[o0_1 + (int64_t)(h + j) * ostride] = y1[j];
+            }
+        }
+        if (a.dbg_acc != nullptr) {
+            #pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (ok0) a.dbg_acc[o0_0 + (int64_t)(h + j) * ostride] = (int)v0[h + j];
+                if (ok1) a.dbg_acc[o0_1 + (int64_t)(h + j) * ostride] = (int)v1[h + j];
+            }
+        }
+        if (want_codes) {
+            float ab0 = 0.f, be0 = 0.f, ab1 = 0.f, be1 = 0.f;          // bits summed as powers of two (exact)
+            #pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float2 t = sT[h + j];
+                const float bit = (float)(1u << (h + j));
+                ab0 = fmaf(y0[j] > t.y ? 1.f : 0.f, bit, ab0);
+                be0 = fmaf(y0[j] < t.x ? 1.f : 0.f, bit, be0);
+                ab1 = fmaf(y1[j] > t.y ? 1.f : 0.f, bit, ab1);
+                be1 = fmaf(y1[j] < t.x ? 1.f : 0.f, bit, be1);
+            }
+            const uint32_t s0 = (uint32_t)ab0, s1 = (uint32_t)ab1;
+            sgb0 |= s0; nzb0 |= s0 | (uint32_t)be0;
+            sgb1 |= s1; nzb1 |= s1 | (uint32_t)be1;
+        }
+    }
+}
+
 // Zero codes for the columns from n_begin (a multiple of 16) to the end of a packed pixel row.
 __device__ __forceinline__ void zero_fill_packed_row(uint8_t* out_row, int n_begin, int packed_cols)
 {

@@ -32,7 +32,9 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="cfg2", choices=sorted(WORKLOADS))
     ap.add_argument("--batch", type=int, default=None, help="conv workloads: batch size (default: the workload's own)")
-    ap.add_argument("--io", default="fp32", choices=["fp32", "packed"])
+    ap.add_argument("--io", default="fp32", choices=["fp32", "packed", "packed_skip"],
+                    help="conv workloads: fp32 in and out; packed rows in and out (a block's first layer); or packed rows in, "
+                         "fp32 skip connection in, fp32 and packed rows out (a block's second layer)")
     ap.add_argument("--runs", type=int, default=4)
     a = ap.parse_args()
     from . import build
@@ -66,22 +68,28 @@ def main():
             case = inputs.resnet18_layer("layer2.0.conv2", batch=a.batch or 64)
         w_packed, w_sum = rtn.rtn_pack_weights(dev(case.w_codes))
         t_lo, t_hi, w_s, w_o = dev(case.t_lo), dev(case.t_hi), dev(case.w_scale), dev(case.w_offset)
-        if a.io == "packed":
+        if a.io != "fp32":
             nhwc = dev(np.ascontiguousarray(case.x.transpose(0, 2, 3, 1)).reshape(-1, case.C))
             xp, _ = rtn.rtn_ternarize_pack_act(nhwc, t_lo, t_hi, want_sum=False)
             rows = [torch.empty((case.B * case.Ho * case.Wo, rtn.rtn_packed_row_bytes(case.N)), dtype=torch.uint8, device="cuda")
                     for _ in range(a.runs)]
             n_lo, n_hi = dev(np.array([0.5], np.float32)), dev(np.array([2.0], np.float32))
+            extra = {}
+            if a.io == "packed_skip":
+                skip = torch.randn((case.B, case.N, case.Ho, case.Wo), dtype=torch.float32, device="cuda")
+                ys = [torch.empty_like(skip) for _ in range(a.runs)]
         else:
             xs = [dev(case.x) for _ in range(a.runs)]
             outs = [torch.empty((case.B, case.N, case.Ho, case.Wo), dtype=torch.float32, device="cuda") for _ in range(a.runs)]
         torch.cuda.synchronize()
         assert reader(None, 1) == 0
         for j in range(a.runs):
-            if a.io == "packed":
+            if a.io != "fp32":
+                if a.io == "packed_skip":
+                    extra = dict(skip=skip, out=ys[j])
                 rtn.rtn_ternary_conv2d_packed(xp, case.B, case.C, case.H, case.W, w_packed, w_sum, case.N, case.kh, case.kw,
                                               case.stride, case.pad, rtn.PAD_CODE_ZERO, case.a_scale, case.a_offset, w_s, w_o,
-                                              relu=True, next_t_lo=n_lo, next_t_hi=n_hi, out_packed=rows[j])
+                                              relu=True, next_t_lo=n_lo, next_t_hi=n_hi, out_packed=rows[j], **extra)
             else:
                 rtn.rtn_ternary_conv2d(xs[j], t_lo, t_hi, w_packed, w_sum, case.N, case.kh, case.kw, case.stride, case.pad,
                                        rtn.PAD_CODE_ZERO, case.a_scale, case.a_offset, w_s, w_o, out=outs[j])
