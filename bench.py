@@ -172,6 +172,8 @@ def file_sha256(path):
 def traffic_of(key):
     """DRAM bytes per launch of the workload's dominant kernel from the tracked ncu record, or None when there
     is no record or a source file of the kernel has changed since the counters were taken."""
+    import re
+    key = re.sub(r"_z0\.\d+", "", key)          # the weight-zero fraction does not change what a kernel moves
     try:
         with open(TRAFFIC_FILE) as f:
             rec = json.load(f).get(key)
