@@ -1,9 +1,9 @@
 """Role timelines of the tensor-core kernels from in-kernel clock stamps.
 
-    python -m paper_1912_02057_b200.timeline [--workload cfg2|layer2|cfg3a|gemm2048|gemm4096|gemm8192] [--batch B] [--io fp32|packed]
+    python -m paper_1912_02057_b200.timeline [--workload cfg2|layer2|cfg3a|cfg3b|gemm2048|gemm4096|gemm8192] [--batch B] [--io fp32|packed]
 
 Builds librtn_b200_timeline.so (the library with -DRTN_TIMELINE, see csrc/rtn_timeline.cuh), runs the workload's
-layer (conv_i8_kernel for cfg2 / layer2, conv_i8s_kernel for cfg3a, gemm_i8_kernel for the square GEMMs) on it a few
+layer (conv_i8_kernel for cfg2 / layer2, conv_i8s_kernel for cfg3a and cfg3b, gemm_i8_kernel for the square GEMMs) on it a few
 times (the last run is reported; earlier ones warm the caches and overlap each launch's
 set-up with the previous kernel's tail as in a stream of layers) and prints, for four CTAs spread over the grid,
 the microseconds after the CTA's entry at which each role began and ended each tile.  The stamps are SM cycle
@@ -24,7 +24,7 @@ SLOTS = {"conv_i8": {"entry": 0, "set-up done": 1, "filters expanded": 2, "epilo
                       "roles": {"ternarizers": 24, "mma": 40, "epilogue": 56}, "tiles": 8},
          "gemm_i8": {"entry": 0, "set-up done": 1, "end": 4, "roles": {"mma": 40, "epilogue": 56}, "tiles": 8}}
 # workload -> (instrumented kernel, how to build the case)
-WORKLOADS = {"cfg2": "conv_i8", "layer2": "conv_i8", "cfg3a": "conv_i8s", "cfg3b_streamed": "conv_i8s",
+WORKLOADS = {"cfg2": "conv_i8", "layer2": "conv_i8", "cfg3a": "conv_i8s", "cfg3b": "conv_i8s",
              "gemm4096": "gemm_i8", "gemm2048": "gemm_i8", "gemm8192": "gemm_i8"}
 
 
@@ -64,6 +64,8 @@ def main():
             case = inputs.config2(batch=a.batch or 32)
         elif a.workload == "cfg3a":
             case = inputs.config3a(0.5, batch=a.batch or 128)
+        elif a.workload == "cfg3b":
+            case = inputs.config3b(0.5, batch=a.batch or 128)
         else:
             case = inputs.resnet18_layer("layer2.0.conv2", batch=a.batch or 64)
         w_packed, w_sum = rtn.rtn_pack_weights(dev(case.w_codes))
