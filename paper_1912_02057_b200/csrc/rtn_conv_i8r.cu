@@ -32,6 +32,12 @@
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
 #include "rtn_conv_i8_common.cuh"
+#include "rtn_timeline.cuh"
+
+// Timeline slots of conv_i8r_kernel (instrumented build only): 0 kernel entry, 1 set-up done (filters expanded, the code
+// kernel finished), 4 kernel end; per tile i < 8 of the CTA: 8+2i / 9+2i producer issues the first / last slot, 40+2i / 41+2i
+// first slot ready for the tensor core / accumulators committed, 56+2i / 57+2i epilogue begins / ends.
+RTN_TL_DEFINE(conv_i8r)
 
 namespace rtn {
 
@@ -330,6 +336,8 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
     const int n_base = fq * p.Nq;
 
     // ---------------------------------------------------------------- set-up (all threads)
+    RTN_TL_INIT(conv_i8r)
+    if (threadIdx.x == 0) RTN_TL(conv_i8r, 0);
     tc::pdl_trigger();
     if (warp == 0) tc::tmem_alloc(slot, p.tmem_cols);
     if (threadIdx.x == 32) {
@@ -408,7 +416,9 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem = *slot;
+    if (threadIdx.x == 0) RTN_TL(conv_i8r, 2);
     tc::pdl_wait();         // from here on: the codes and sums of the code kernel, and out
+    if (threadIdx.x == 0) RTN_TL(conv_i8r, 1);
 
     if (warp == 1) {
         // ------------------------------------------------------------ producer (one thread)
@@ -457,12 +467,14 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
             int acc = 0;
             uint32_t acc_ph = 0;
             bool alive = true, have = false;    // have: slot s is known to be full
-            for (int tile = first_tile; tile < p.ntiles && alive; tile += p.cpg) {
+            int tl_i = 0;
+            for (int tile = first_tile; tile < p.ntiles && alive; tile += p.cpg, ++tl_i) {
                 if (!wait_or_die(&acc_empty[acc], acc_ph ^ 1, a.status, dead)) break;
                 const uint32_t d = tmem + (uint32_t)(acc * p.Nq);
                 for (int h0 = 0; h0 < p.ngroup && alive; h0 += p.gps) {
                     if (!have && !wait_or_die(&slot_full[s], ph, a.status, dead)) { alive = false; break; }
                     tc::tc_fence_after_sync();
+                    if (h0 == 0 && tl_i < 8) RTN_TL(conv_i8r, 40 + 2 * tl_i);
                     const uint32_t s_cur = s;
                     if (++s == (uint32_t)p.nslots) { s = 0; ph ^= 1; }
                     have = tc::mbar_test(&slot_full[s], ph);
@@ -492,6 +504,7 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
                 }
                 if (!alive) break;
                 tc::mma_commit(&acc_full[acc]);
+                if (tl_i < 8) RTN_TL(conv_i8r, 41 + 2 * tl_i);
                 if (++acc == p.nAcc) { acc = 0; acc_ph ^= 1; }
             }
         }
@@ -502,14 +515,15 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
         const int nblk16 = p.Nq / 16;
         const int blk_begin = half == 0 ? 0 : (nblk16 + 1) / 2;
         const int blk_end = half == 0 ? (nblk16 + 1) / 2 : nblk16;
-        int acc = 0;
+        int acc = 0, tl_i = 0;
         uint32_t acc_ph = 0;
-        for (int tile = first_tile; tile < p.ntiles; tile += p.cpg) {
+        for (int tile = first_tile; tile < p.ntiles; tile += p.cpg, ++tl_i) {
             const int g = tile * p.RT;
             const int nrows = min(p.RT, p.total_rows - g);
             role_wait_r(warp == kEpiWarp0, &acc_full[acc], acc_ph, a.status, dead, kEpiBarrier, kEpiThreads);
             const bool alive = !*dead;
             tc::tc_fence_after_sync();
+            if (warp == kEpiWarp0 && lane == 0 && tl_i < 8) RTN_TL(conv_i8r, 56 + 2 * tl_i);
             const uint32_t pl = (uint32_t)(q * 32 + lane);         // pixel within the tile
             const uint32_t row = fdiv(pl, p.div_pw);
             const int wo = (int)(pl - row * (uint32_t)p.PW);
@@ -596,12 +610,14 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[acc]);
+            if (warp == kEpiWarp0 && lane == 0 && tl_i < 8) RTN_TL(conv_i8r, 57 + 2 * tl_i);
             if (++acc == p.nAcc) { acc = 0; acc_ph ^= 1; }
         }
     }
     tc::tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tc::tmem_dealloc(tmem, p.tmem_cols);
+    if (threadIdx.x == 0) RTN_TL(conv_i8r, 4);
 }
 
 // Scratch of the variant that allocates nothing: one array per device, part of the module's image.

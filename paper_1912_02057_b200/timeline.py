@@ -1,6 +1,6 @@
 """Role timelines of the tensor-core kernels from in-kernel clock stamps.
 
-    python -m paper_1912_02057_b200.timeline [--workload cfg2|layer2|cfg3a|cfg3b|gemm2048|gemm4096|gemm8192] [--batch B] [--io fp32|packed]
+    python -m paper_1912_02057_b200.timeline [--workload cfg2|layer2|layer3|layer4|cfg3a|cfg3b|gemm2048|gemm4096|gemm8192] [--batch B] [--io fp32|packed]
 
 Builds librtn_b200_timeline.so (the library with -DRTN_TIMELINE, see csrc/rtn_timeline.cuh), runs the workload's
 layer (conv_i8_kernel for cfg2 / layer2, conv_i8s_kernel for cfg3a and cfg3b, gemm_i8_kernel for the square GEMMs) on it a few
@@ -22,9 +22,11 @@ SLOTS = {"conv_i8": {"entry": 0, "set-up done": 1, "filters expanded": 2, "epilo
                      "roles": {"producer": 8, "converters": 24, "mma": 40, "epilogue": 56}, "tiles": 8},
          "conv_i8s": {"entry": 0, "set-up done": 1, "end": 4,
                       "roles": {"ternarizers": 24, "mma": 40, "epilogue": 56}, "tiles": 8},
+         "conv_i8r": {"entry": 0, "filters expanded": 2, "code kernel done": 1, "end": 4,
+                      "roles": {"mma": 40, "epilogue": 56}, "tiles": 8},
          "gemm_i8": {"entry": 0, "set-up done": 1, "end": 4, "roles": {"mma": 40, "epilogue": 56}, "tiles": 8}}
 # workload -> (instrumented kernel, how to build the case)
-WORKLOADS = {"cfg2": "conv_i8", "layer2": "conv_i8", "cfg3a": "conv_i8s", "cfg3b": "conv_i8s",
+WORKLOADS = {"layer3": "conv_i8r", "layer4": "conv_i8r", "cfg2": "conv_i8", "layer2": "conv_i8", "cfg3a": "conv_i8s", "cfg3b": "conv_i8s",
              "gemm4096": "gemm_i8", "gemm2048": "gemm_i8", "gemm8192": "gemm_i8"}
 
 
@@ -64,6 +66,8 @@ def main():
             case = inputs.config2(batch=a.batch or 32)
         elif a.workload == "cfg3a":
             case = inputs.config3a(0.5, batch=a.batch or 128)
+        elif a.workload in ("layer3", "layer4"):      # stride-1 3x3 layers of stages 3 and 4 (split-bank pair at batch 64)
+            case = inputs.resnet18_layer("layer3.1.conv1" if a.workload == "layer3" else "layer4.1.conv1", batch=a.batch or 64)
         elif a.workload == "cfg3b":
             case = inputs.config3b(0.5, batch=a.batch or 128)
         else:
