@@ -773,72 +773,42 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         // While the first input rows are in flight these warps, idle until the first accumulators are
         // complete, expand the filters and work out the epilogue constants.
         const int etid = threadIdx.x - kEpiWarp0 * 32;
-        {   // filters: bit planes -> int8, [tap][chunk][n]; row N is all +1, rows above it are 0.
-            // item = (32-channel word of a tap, filter row); a thread's loads of six items are in flight
-            // together (the expansion is on the path to the first MMA, and each load is a trip to HBM)
-            const int cwords = p.Cp / 32;
-            const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
-            const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
-            const int items = p.T * cwords * p.Np;
-            constexpr int kBatch = 6;
-            for (int base = etid; base < items; base += kBatch * kEpiThreads) {
-                uint32_t nz[kBatch], sg[kBatch];
-                #pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    const int i = base + u * kEpiThreads;
-                    nz[u] = 0; sg[u] = 0;
-                    if (i < items) {
-                        const int wd = (int)fdiv((uint32_t)i, p.div_np), n = i - wd * p.Np;
-                        if (n < a.N) {
-                            const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
-                            nz[u] = __ldg(blk + (wd & 3));
-                            sg[u] = __ldg(blk + 4 + (wd & 3));
-                        } else if (n == a.N) {
-                            nz[u] = 0xFFFFFFFFu; sg[u] = 0xFFFFFFFFu;
-                        }
-                    }
-                }
-                #pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    const int i = base + u * kEpiThreads;
-                    if (i < items) {
-                        const int wd = (int)fdiv((uint32_t)i, p.div_np), n = i - wd * p.Np;
-                        const int t = (int)fdiv((uint32_t)wd, p.div_cw), cw = wd - t * cwords;
-                        uint32_t o[8];
-                        tc::unpack32(nz[u], sg[u], o);
-                        uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Np + n);
-                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                        dst[p.Np] = make_uint4(o[4], o[5], o[6], o[7]);
-                    }
-                }
-            }
+        // The operands of the epilogue constants are fetched first, so that their trip to memory overlaps the filters'.
+        const bool has_col = etid < p.Np && etid < a.N;
+        float ws_f = 0.f, wo_f = 0.f;
+        int wsum_i = 0;
+        if (has_col) {
+            ws_f = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : etid];
+            wo_f = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : etid];
+            wsum_i = a.w_sum[etid];
         }
+        float2 next_t = make_float2(-INFINITY, INFINITY);
+        if constexpr (kNext) {
+            if (has_col && f.out_packed != nullptr)
+                next_t = make_float2(f.next_lo[f.n_next == 1 ? 0 : etid], f.next_hi[f.n_next == 1 ? 0 : etid]);
+        }
+        // filters: bit planes -> int8, [tap][chunk][n]; row N is all +1, rows above it are 0
+        expand_filter_rows<2>(a.w_packed, sW, p.T, p.Cp / 32, p.Np, p.div_np, p.div_cw, 0, a.N, a.N, etid, kEpiThreads);
         tc::fence_smem_to_async_proxy();
         tc::mbar_arrive(w_ready);
         if (etid == 0) RTN_TL(conv_i8, 2);
         {   // per-output-channel constants in double, rounded once (first needed by the first epilogue):
             //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
             const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
-            for (int n = etid; n < p.Np; n += kEpiThreads) {
+            if (etid < p.Np) {                          // Np <= 256 = the epilogue's threads: one column each
                 float c1 = 0.f, c2 = 0.f, c3 = 0.f;
-                if (n < a.N) {
-                    const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
-                    const double wo = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
+                if (has_col) {
+                    const double ws = ws_f, wo = wo_f;
                     c1 = (float)(a_s * ws);
                     c2 = (float)(a_s * wo);
-                    c3 = (float)(a_o * (ws * (double)a.w_sum[n] + (double)a.C * p.T * wo));
+                    c3 = (float)(a_o * (ws * (double)wsum_i + (double)a.C * p.T * wo));
                 }
-                sC[n] = make_float4(c1, c2, c3, 0.f);
+                sC[etid] = make_float4(c1, c2, c3, 0.f);
             }
             if constexpr (kNext) {
                 // the next layer's threshold pair per column; columns past N code to 0
                 float2* sT = reinterpret_cast<float2*>(smem + p.off_t);
-                for (int n = etid; n < p.Np; n += kEpiThreads) {
-                    float2 t = make_float2(-INFINITY, INFINITY);
-                    if (f.out_packed != nullptr && n < a.N)
-                        t = make_float2(f.next_lo[f.n_next == 1 ? 0 : n], f.next_hi[f.n_next == 1 ? 0 : n]);
-                    sT[n] = t;
-                }
+                if (etid < p.Np) sT[etid] = next_t;
             }
         }
         asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible

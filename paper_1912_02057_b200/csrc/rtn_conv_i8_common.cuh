@@ -40,6 +40,66 @@ __device__ __forceinline__ bool wait_or_die(uint64_t* bar, uint32_t parity, unsi
     return false;
 }
 
+// Filters of rows n_base .. n_base + ld - 1: bit planes (Table 1) in global memory -> int8 in shared memory,
+// sW[(tap * Cp/16 + 16-channel chunk) * ld + row][16 B] in tc::unpack32's byte order.  Row `ones_row` (relative to
+// n_base; -1 for none) becomes all +1 (it makes the tensor core produce the activation code sum), rows at or past
+// N become 0.  Item = (row, packed block of four 32-channel words of each plane): two 16-byte loads instead of
+// eight 4-byte ones.  Consecutive lanes take consecutive rows, so the shared-memory stores are conflict-free; the
+// loads of a warp then fall in 32 different lines, which the load unit takes one line at a time, and that, with
+// every CTA of the grid asking for the same few lines, is what this step's time is made of: a quarter of the load
+// instructions is a quarter of the time.  kBatch items' loads are in flight per thread.
+template <int kBatch>
+__device__ __forceinline__ void expand_filter_rows(const uint8_t* w_packed, uint4* sW, int T, int cwords, int ld,
+                                                   FastDiv div_ld, FastDiv div_cw, int n_base, int N, int ones_row,
+                                                   int tid, int nthreads)
+{
+    const int nwords = T * cwords;                     // 32-channel words per plane and row
+    const int nblocks = (nwords + 3) / 4;              // packed blocks per row
+    const int nchunk = 2 * cwords;
+    const uint4* Wp = reinterpret_cast<const uint4*>(w_packed);
+    const int items = nblocks * ld;
+    for (int base = tid; base < items; base += kBatch * nthreads) {
+        uint4 nz[kBatch], sg[kBatch];
+        #pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int i = base + u * nthreads;
+            nz[u] = make_uint4(0u, 0u, 0u, 0u); sg[u] = nz[u];
+            if (i < items) {
+                const int wb = (int)fdiv((uint32_t)i, div_ld), r = i - wb * ld;
+                const int n = n_base + r;
+                if (r == ones_row) {
+                    nz[u] = make_uint4(~0u, ~0u, ~0u, ~0u); sg[u] = nz[u];
+                } else if (n < N) {
+                    const uint4* blk = Wp + ((int64_t)n * nblocks + wb) * 2;
+                    nz[u] = __ldg(blk);
+                    sg[u] = __ldg(blk + 1);
+                }
+            }
+        }
+        #pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int i = base + u * nthreads;
+            if (i < items) {
+                const int wb = (int)fdiv((uint32_t)i, div_ld), r = i - wb * ld;
+                const uint32_t nzw[4] = {nz[u].x, nz[u].y, nz[u].z, nz[u].w};
+                const uint32_t sgw[4] = {sg[u].x, sg[u].y, sg[u].z, sg[u].w};
+                #pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int wd = 4 * wb + j;
+                    if (wd < nwords) {
+                        const int t = (int)fdiv((uint32_t)wd, div_cw), cw = wd - t * cwords;
+                        uint32_t o[8];
+                        tc::unpack32(nzw[j], sgw[j], o);
+                        uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * ld + r);
+                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                        dst[ld] = make_uint4(o[4], o[5], o[6], o[7]);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // Sixteen fp32 values -> sixteen int8 codes {-1,0,+1} in four words (byte e of the chunk = v[e]).
 // Branch-free: p = (v > hi), n = (v < lo) as 1.0f / 0.0f, then (1.5*2^23 + p) - n is a float whose
 // low mantissa byte is the two's-complement code; PRMT gathers the four low bytes of a word.  The

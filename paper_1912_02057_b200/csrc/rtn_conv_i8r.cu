@@ -346,70 +346,39 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
         tc::mbar_init_fence();
         *dead = 0;
     }
-    {   // this group's filters: bit planes -> int8, [tap][chunk][row]; rows beyond N are zero.
-        // item = (32-channel word of a tap, filter row); six items' loads in flight per thread
-        const int cwords = p.ngroup;
-        const int64_t row_words = ((int64_t)p.T * cwords + 3) / 4 * 4;          // words per plane per row
-        const uint32_t* Wp = reinterpret_cast<const uint32_t*>(a.w_packed);
-        const int items = p.T * cwords * p.Nq;
-        constexpr int kBatch = 6;
-        for (int base = threadIdx.x; base < items; base += kBatch * kThreads) {
-            uint32_t nz[kBatch], sg[kBatch];
-            #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                const int i = base + u * kThreads;
-                nz[u] = 0; sg[u] = 0;
-                if (i < items) {
-                    const int wd = (int)fdiv((uint32_t)i, p.div_nq), r = i - wd * p.Nq;
-                    const int n = n_base + r;
-                    if (n < a.N) {
-                        const uint32_t* blk = Wp + ((int64_t)n * (row_words / 4) + wd / 4) * 8;
-                        nz[u] = __ldg(blk + (wd & 3));
-                        sg[u] = __ldg(blk + 4 + (wd & 3));
-                    }
-                }
-            }
-            #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                const int i = base + u * kThreads;
-                if (i < items) {
-                    const int wd = (int)fdiv((uint32_t)i, p.div_nq), r = i - wd * p.Nq;
-                    const int t = (int)fdiv((uint32_t)wd, p.div_cw), cw = wd - t * cwords;
-                    uint32_t o[8];
-                    tc::unpack32(nz[u], sg[u], o);
-                    uint4* dst = sW + ((int64_t)(t * nchunk + 2 * cw) * p.Nq + r);
-                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[p.Nq] = make_uint4(o[4], o[5], o[6], o[7]);
-                }
-            }
+    // Nq <= 256 < the CTA's threads: one column per thread.  The operands of its epilogue constants (and the next
+    // layer's thresholds) are fetched first, so that their trip to memory overlaps the filters'.
+    const int col = n_base + (int)threadIdx.x;
+    const bool has_col = (int)threadIdx.x < p.Nq && col < a.N;
+    float ws_f = 0.f, wo_f = 0.f;
+    int wsum_i = 0;
+    float2 next_t = make_float2(-INFINITY, INFINITY);
+    if (has_col) {
+        ws_f = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : col];
+        wo_f = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : col];
+        wsum_i = a.w_sum[col];
+        if constexpr (kFused) {
+            // (as in the ternarizers: +1 is tested first)
+            if (f.out_packed != nullptr)
+                next_t = make_float2(f.next_lo[f.n_next == 1 ? 0 : col], f.next_hi[f.n_next == 1 ? 0 : col]);
         }
     }
-    {   // per-output-channel constants in double, rounded once:
+    // this group's filters: bit planes -> int8, [tap][chunk][row]; rows beyond N are zero
+    expand_filter_rows<2>(a.w_packed, sW, p.T, p.ngroup, p.Nq, p.div_nq, p.div_cw, n_base, a.N, -1, (int)threadIdx.x,
+                          kThreads);
+    if ((int)threadIdx.x < p.Nq) {
+        // per-output-channel constants in double, rounded once:
         //   c1 = a_s*w_s, c2 = a_s*w_o, c3 = a_o*(w_s*S_w + K*w_o)     (K = C*kh*kw)
         const double a_s = a.ep.a_scale_val, a_o = a.ep.a_offset_val;
-        for (int r = threadIdx.x; r < p.Nq; r += kThreads) {
-            const int n = n_base + r;
-            float c1 = 0.f, c2 = 0.f, c3 = 0.f;
-            if (n < a.N) {
-                const double ws = a.ep.w_scale[a.ep.n_wparam == 1 ? 0 : n];
-                const double wo = a.ep.w_offset[a.ep.n_wparam == 1 ? 0 : n];
-                c1 = (float)(a_s * ws);
-                c2 = (float)(a_s * wo);
-                c3 = (float)(a_o * (ws * (double)a.w_sum[n] + (double)a.C * p.T * wo));
-            }
-            sC[r] = make_float4(c1, c2, c3, 0.f);
+        float c1 = 0.f, c2 = 0.f, c3 = 0.f;
+        if (has_col) {
+            const double ws = ws_f, wo = wo_f;
+            c1 = (float)(a_s * ws);
+            c2 = (float)(a_s * wo);
+            c3 = (float)(a_o * (ws * (double)wsum_i + (double)a.C * p.T * wo));
         }
-    }
-    if constexpr (kFused) {
-        // the next layer's threshold pair per column (as in the ternarizers: +1 is tested first)
-        float2* sT = reinterpret_cast<float2*>(smem + p.off_t);
-        for (int r = threadIdx.x; r < p.Nq; r += kThreads) {
-            const int n = n_base + r;
-            float2 t = make_float2(-INFINITY, INFINITY);
-            if (f.out_packed != nullptr && n < a.N)
-                t = make_float2(f.next_lo[f.n_next == 1 ? 0 : n], f.next_hi[f.n_next == 1 ? 0 : n]);
-            sT[r] = t;
-        }
+        sC[threadIdx.x] = make_float4(c1, c2, c3, 0.f);
+        if constexpr (kFused) reinterpret_cast<float2*>(smem + p.off_t)[threadIdx.x] = next_t;
     }
     tc::fence_smem_to_async_proxy();
     tc::tc_fence_before_sync();
