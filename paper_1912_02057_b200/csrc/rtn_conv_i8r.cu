@@ -654,14 +654,14 @@ bool conv_i8r_next_supported(const ConvArgs& c)
 }
 
 // Rough time of this variant for a shape, in microseconds (negative: not taken).  Measured on B200: about
-// 12 us of fixed cost plus the multiply-accumulates over the padded pixels at 600 T/s (64 or more filters per
-// CTA) or 370 T/s (fewer: an MMA a quarter full).
+// 8 us of fixed cost (two launches, filter expansion, the last epilogue) plus the multiply-accumulates over the
+// padded pixels at 640 T/s (64 or more filters per CTA) or 370 T/s (fewer: an MMA a quarter full).
 double conv_i8r_estimate_us(const ConvArgs& c)
 {
     ConvI8RPlan p;
     if (!make_plan_r(c, p, device_sm_count())) return -1.0;
     const double macs = (double)p.Ptot * p.Cp * p.T * (double)(p.S * p.Nq);     // padded output pixels x K x filters
-    return 12.0 + macs / ((p.Nq >= 64 ? 600.0 : 370.0) * 1e6);
+    return 8.0 + macs / ((p.Nq >= 64 ? 640.0 : 370.0) * 1e6);
 }
 
 size_t conv_i8r_scratch_bytes(const ConvArgs& c)

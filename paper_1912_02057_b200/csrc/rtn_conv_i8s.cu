@@ -70,11 +70,13 @@ struct ConvI8SPlan {
     int nK;                // K = 32 slices per tile in stage order, padded to whole packed blocks
     int nW;                // filter ring depth
     int nAcc;              // accumulator sets (1 or 2)
-    int npass, NpP;        // passes over the output channels (2 when N > 256) and columns per pass
+    int npass, NpP;        // passes over the output channels (groups of NpP filters) and columns per pass
+    int split;             // the passes are dealt to CTAs (CTA = strip x filter group) instead of run one after the other
+    int nstrips;           // strips of rows; grid = nstrips * (split ? npass : 1)
     int nA;                // code buffers (1 or 2)
     uint32_t tmem_cols;
     FastDiv div_pw, div_ph, div_T;   // div_T: stage -> (128-channel block, tap)
-    uint32_t off_a[2], off_w, off_psum, off_lo, off_hi, off_c, off_t, off_bar, off_misc;
+    uint32_t off_a[2], off_w, off_psum, off_lo, off_hi, off_c, off_t, off_bar, off_misc, off_tab;
     size_t smem_bytes;
     int blocks_major;      // stage order: 128-channel block outer, tap inner (else the packed order)
     int pre;               // filters expanded beforehand into scratch, slices in (32-channel group, tap) order
@@ -83,7 +85,9 @@ struct ConvI8SPlan {
                            // 0xFFFFFFFF for the padding slices of the last packed block
 };
 
-bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
+// split: the filter bank is cut into groups of 128 filters and a CTA takes one group for its strip (it streams a
+// group's share of the bank only; its tensor-core instructions are 128 columns wide).
+bool make_plan_mode(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next, bool split)
 {
     if (c.Ho <= 0 || c.Wo <= 0) return false;
     p.T = c.kh * c.kw;
@@ -102,14 +106,32 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
     // accumulator sets and their barriers what a tile is, so with two sets the first pass's epilogue runs
     // under the second pass's MMAs.  Only with the filters expanded beforehand (checked below).
     if (p.Np > 512) return false;
-    p.npass = p.Np > 256 ? 2 : 1;
-    p.NpP = p.npass == 2 ? 256 : p.Np;
+    p.split = split ? 1 : 0;
+    if (split) {
+        if (p.Np <= 128) return false;
+        p.NpP = 128;
+        p.npass = (p.Np + 127) / 128;
+    } else {
+        p.npass = p.Np > 256 ? 2 : 1;
+        p.NpP = p.npass == 2 ? 256 : p.Np;
+    }
     if (p.Cp / 32 > kMaxGroups) return false;
     p.total_rows = c.B * p.PH;
-    p.grid = p.total_rows < sms ? p.total_rows : sms;
+    if (split) {
+        // one wave of CTAs: a strip per whole 256-pixel tile when that many CTAs fit, else as many strips as fit
+        const int rt2 = 2 * kTileM / p.PW;
+        if (rt2 < 1 || sms / p.npass < 1) return false;
+        const int tiles2 = (p.total_rows + rt2 - 1) / rt2;
+        p.nstrips = tiles2 * p.npass <= sms ? tiles2 : sms / p.npass;
+        if (p.nstrips > p.total_rows) p.nstrips = p.total_rows;
+        p.grid = p.nstrips * p.npass;
+    } else {
+        p.nstrips = p.total_rows < sms ? p.total_rows : sms;
+        p.grid = p.nstrips;
+    }
     // 256-pixel tiles whenever a CTA's strip has more than 128 pixels: a tile's filter stream costs
     // the same whatever its size
-    const int strip_rows = (p.total_rows + p.grid - 1) / p.grid;
+    const int strip_rows = (p.total_rows + p.nstrips - 1) / p.nstrips;
     p.TM = (2 * p.NpP <= 512 && strip_rows * p.PW > kTileM) ? 2 : 1;
     p.nAcc = (2 * p.TM * p.NpP <= 512) ? 2 : 1;
     p.RT = p.TM * kTileM / p.PW;
@@ -132,6 +154,7 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
     // first 32 channels are ternarized and follows the ternarizers group by group.
     p.pre = nblocks >= 4 ? 1 : 0;
     if (p.npass > 1 && !p.pre) return false;
+    if (split && !p.pre) return false;
     for (int i = 0; p.pre && i < p.nK; ++i) {
         uint32_t e = 0xFFFFFFFFu;
         if (i < nwords) {
@@ -156,8 +179,10 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
     const uint32_t a_bytes = (uint32_t)(p.Cp / 16) * p.ppix * 16;
     const uint32_t stage = (uint32_t)p.NpP * 32 * kSlices;
     const int nstages = p.nK / kSlices;
-    // two code buffers when they leave room for a filter ring of four stages (or all of them)
-    for (p.nA = 2; p.nA >= 1; --p.nA) {
+    // two code buffers when they leave room for a filter ring of four stages (or all of them); a CTA with a single
+    // tile has no use for the second one, and the ring, whose depth is what hides a stage's trip from L2, gets the room
+    const int strip_tiles = (strip_rows + p.RT - 1) / p.RT;
+    for (p.nA = strip_tiles == 1 ? 1 : 2; p.nA >= 1; --p.nA) {
         uint32_t o = 0;
         p.off_a[0] = o; o += a_bytes;
         p.off_a[1] = o; if (p.nA == 2) o += a_bytes;
@@ -169,6 +194,7 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
         p.off_t = o;    o += next ? (uint32_t)p.Np * 8 : 0;     // float2 {t_lo, t_hi} of the next layer per column
         p.off_bar = o;  o += (6 + 2 * kMaxWStages + 2 * kMaxGroups) * 8;   // a_empty[2] acc_full[2] acc_empty[2] w_full[] w_empty[] a_full[2][]
         p.off_misc = o; o += 16;
+        p.off_tab = o;  o += p.pre ? (uint32_t)(nstages + 1) * 16 : 0;     // per stage: the A windows of its four slices
         o = (o + 127) / 128 * 128;
         p.off_w = o;
         if (o > kSmemLimit) continue;
@@ -184,6 +210,40 @@ bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
         return true;
     }
     return false;
+}
+
+// Rough time of a plan, in microseconds, from measurements on B200 (packed input; fp32 input adds to every plan
+// alike).  With the filters streamed from scratch a tensor-core instruction of N columns costs about N/2 + 60
+// cycles in this kernel's issue loop and the stream keeps up; expanded in the kernel a 32 KB stage takes 1 us.  A
+// tile's codes take 2 ns per pixel and 32-channel group; the last tile's epilogue, which nothing overlaps, 1.5 us
+// plus a microsecond per 7500 outputs of a CTA; launch, set-up and the first stage's trip about 3 us.
+static double plan_estimate_us(const ConvI8SPlan& p)
+{
+    const int strip_rows = (p.total_rows + p.nstrips - 1) / p.nstrips;
+    const int tiles = (strip_rows + p.RT - 1) / p.RT;
+    const int nstages = p.nK / kSlices;
+    const int passes = p.split ? 1 : p.npass;
+    double stage_us = kSlices * p.TM * (p.NpP / 2.0 + 60.0) / 1900.0;
+    if (!p.pre && stage_us < (double)p.NpP / 256.0) stage_us = (double)p.NpP / 256.0;
+    const double px = (double)(strip_rows < p.RT ? strip_rows : p.RT) * p.PW;
+    const double tern_us = px * (p.Cp / 32) * 0.002;
+    const double mma_us = (double)passes * nstages * stage_us;
+    const double tile_us = mma_us > tern_us ? mma_us : tern_us;
+    return 3.0 + tile_us * tiles + tern_us / (p.Cp / 32) + 1.5 + px * p.NpP / 7500.0;
+}
+
+// The plan of the faster of the two ways to share out the filters.
+bool make_plan_s(const ConvArgs& c, ConvI8SPlan& p, int sms, bool next = false)
+{
+    ConvI8SPlan q;
+    const bool whole = make_plan_mode(c, p, sms, next, false);
+    const bool split = make_plan_mode(c, q, sms, next, true);
+#ifdef RTN_I8S_FORCE_SPLIT
+    if (RTN_I8S_FORCE_SPLIT == 0 && whole) return true;
+    if (RTN_I8S_FORCE_SPLIT == 1 && split) { p = q; return true; }
+#endif
+    if (split && (!whole || plan_estimate_us(q) < plan_estimate_us(p))) p = q;
+    return whole || split;
 }
 
 // One warp of a role waits on the mbarrier; the role's other warps sleep on a hardware named
@@ -258,9 +318,13 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ngroup = p.Cp / 32;
     const int nstages = p.nK / kSlices;
-    // this CTA's strip of rows, cut into equal tiles of at most RT rows
-    const int s0 = (int)((int64_t)blockIdx.x * p.total_rows / p.grid);
-    const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
+    // this CTA's strip of rows, cut into equal tiles of at most RT rows, and its passes over the filter groups (all
+    // of them, or the one group dealt to it)
+    const int strip = p.split ? (int)blockIdx.x / p.npass : (int)blockIdx.x;
+    const int pass0 = p.split ? (int)blockIdx.x % p.npass : 0;
+    const int npass_cta = p.split ? 1 : p.npass;
+    const int s0 = (int)((int64_t)strip * p.total_rows / p.nstrips);
+    const int s1 = (int)((int64_t)(strip + 1) * p.total_rows / p.nstrips);
     const int ntile = (s1 - s0 + p.RT - 1) / p.RT;
     const int rt = ntile > 0 ? (s1 - s0 + ntile - 1) / ntile : 1;
 
@@ -278,6 +342,22 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
         for (int i = 0; i < 2 * kMaxGroups; ++i) tc::mbar_init(&a_full[i], kTernThreads);
         tc::mbar_init_fence();
         *dead = 0;
+    }
+    if constexpr (kPre) {
+        // Per stage of the filter stream, the A windows of its four K = 32 slices (one 16-byte load for the issuing
+        // thread).  A padding slice of the last packed block gets window 0 of the last group: its filter slice is
+        // all zeros, so the instruction adds nothing and the issue loop needs no branch for it.
+        uint4* sTab = reinterpret_cast<uint4*>(smem + p.off_tab);
+        for (int i = threadIdx.x; i <= nstages; i += kThreads) {
+            const int st = i < nstages ? i : nstages - 1;
+            uint32_t e[kSlices];
+            #pragma unroll
+            for (int j = 0; j < kSlices; ++j) {
+                const uint32_t v = p.tab_a[st * kSlices + j];
+                e[j] = v == 0xFFFFFFFFu ? (uint32_t)(ngroup - 1) << 24 : v;
+            }
+            sTab[i] = make_uint4(e[0], e[1], e[2], e[3]);
+        }
     }
     bool packed_in = false;
     if constexpr (kNext) packed_in = f.x_packed != nullptr;
@@ -411,16 +491,16 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                 const int nrows = min(rt, s1 - g);
             const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
             const int* psum = sPsum + (it & (kPsumRing - 1)) * p.ppix;
-          for (int pass = 0; pass < p.npass; ++pass) {
-            const int vt = it * p.npass + pass;             // the accumulators go round per (tile, pass)
+          for (int pass = pass0; pass < pass0 + npass_cta; ++pass) {
+            const int vt = it * npass_cta + (pass - pass0);             // the accumulators go round per (tile, pass)
             const int acc = p.nAcc == 2 ? (vt & 1) : 0;
             const uint32_t acc_ph = p.nAcc == 2 ? ((vt >> 1) & 1) : (vt & 1);
             const int slot_acc = acc;
             role_wait(warp == kEpiWarp0, &acc_full[slot_acc], acc_ph, a.status, dead, kEpiBarrier, kEpiThreads);
             const bool alive = !*dead;
             tc::tc_fence_after_sync();
-            if (warp == kEpiWarp0 && lane == 0 && pass == 0 && it < 8) RTN_TL(conv_i8s, 56 + 2 * it);
-            const int pass_blocks = p.npass == 2 ? min(p.NpP / 16, nblk16 - pass * (p.NpP / 16)) : nblk16;
+            if (warp == kEpiWarp0 && lane == 0 && pass == pass0 && it < 8) RTN_TL(conv_i8s, 56 + 2 * it);
+            const int pass_blocks = p.npass > 1 ? min(p.NpP / 16, nblk16 - pass * (p.NpP / 16)) : nblk16;
             const int pb_begin = half == 0 ? 0 : (pass_blocks + 1) / 2;
             const int pb_end = half == 0 ? (pass_blocks + 1) / 2 : pass_blocks;
             for (int tm = 0; tm < ntm; ++tm) {
@@ -511,7 +591,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&acc_empty[acc]);
-            if (warp == kEpiWarp0 && lane == 0 && pass == p.npass - 1 && it < 8) RTN_TL(conv_i8s, 57 + 2 * it);
+            if (warp == kEpiWarp0 && lane == 0 && pass == pass0 + npass_cta - 1 && it < 8) RTN_TL(conv_i8s, 57 + 2 * it);
           }
             }
         }
@@ -527,7 +607,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                 uint32_t wcount = 0;
                 bool alive = true;
                 for (int it = 0; it < ntile && alive; ++it)
-                    for (int s = 0; s < p.npass * nstages; ++s, ++wcount) {      // pass after pass
+                    for (int s = pass0 * nstages; s < (pass0 + npass_cta) * nstages; ++s, ++wcount) {      // pass after pass
                         const uint32_t st = wcount % (uint32_t)p.nW;
                         if (!wait_or_die(&w_empty[st], ((wcount / (uint32_t)p.nW) & 1) ^ 1, a.status, dead)) { alive = false; break; }
                         tc::mbar_arrive_expect_tx(&w_full[st], stage_bytes);
@@ -600,6 +680,73 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
             uint32_t wcount = 0;
             int it = 0;
             bool alive = true;
+            if constexpr (kPre) {
+                // Filters streamed from scratch: slices come 32-channel group by group, so the groups a stage needs
+                // are a count; the stage's four A windows arrive with one shared-memory load, fetched a stage ahead;
+                // ring slot, phase and accumulator set advance by increments; the next stage's barrier is tested
+                // before this stage's MMAs go out.  What is left between two tensor-core instructions of a stage is
+                // one or two additions (a division, a chain of table look-ups and a branch per slice were 0.85 us
+                // per stage of eight instructions that the tensor core runs in 0.3 us).
+                const uint4* sTab = reinterpret_cast<const uint4*>(smem + p.off_tab);
+                uint32_t st = 0, wph = 0;           // filter ring slot and its phase
+                bool have = false;                  // slot st is known to be full
+                uint32_t acc = 0, acc_ph = 0;       // accumulator set and its phase
+                for (int g = s0; g < s1 && alive; g += rt, ++it) {
+                    const int buf = p.nA == 2 ? (it & 1) : 0;
+                    const uint32_t use_ph = p.nA == 2 ? ((it >> 1) & 1) : (it & 1);
+                    const bool two = min(rt, s1 - g) * p.PW > kTileM;      // the tile has a second 128-pixel sub-tile
+                    const uint32_t a16 = (tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4) + a_lbo_field;
+                    uint64_t* full = &a_full[buf * kMaxGroups];
+                    uint32_t nready = 0;            // 32-channel groups whose codes are known to be written
+                    for (int pass = 0; pass < npass_cta && alive; ++pass) {
+                        alive = wait_or_die(&acc_empty[acc], acc_ph ^ 1, a.status, dead);
+                        if (!alive) break;
+                        const uint32_t d0 = tmem + acc * (uint32_t)(p.TM * p.NpP), d1 = d0 + (uint32_t)p.NpP;
+                        uint4 cur = sTab[0];
+                        for (int sg = 0; sg < nstages; ++sg) {
+                            const uint4 nxt = sTab[sg + 1];
+                            if (!have && !wait_or_die(&w_full[st], wph, a.status, dead)) { alive = false; break; }
+                            const uint32_t hmax = cur.w >> 24;
+                            while (nready <= hmax && alive) {
+                                alive = wait_or_die(&full[nready], use_ph, a.status, dead);
+                                ++nready;
+                            }
+                            if (!alive) break;
+                            tc::tc_fence_after_sync();
+                            const uint32_t st_cur = st;
+                            if (++st == (uint32_t)p.nW) { st = 0; wph ^= 1u; }
+                            have = tc::mbar_test(&w_full[st], wph);
+                            const uint32_t b0 = w16 + st_cur * wstage16, b1 = b0 + wslice16, b2 = b1 + wslice16, b3 = b2 + wslice16;
+                            const uint32_t a0 = a16 + (cur.x & 0xFFFFFFu), a1 = a16 + (cur.y & 0xFFFFFFu);
+                            const uint32_t a2 = a16 + (cur.z & 0xFFFFFFu), a3 = a16 + (cur.w & 0xFFFFFFu);
+                            if (sg == 0 && pass == 0 && it < 8) RTN_TL(conv_i8s, 40 + 2 * it);
+                            if (two) {
+                                tc::mma_i8_ss(d0, desc_hi | a0, desc_hi | b0, idesc, sg > 0);
+                                tc::mma_i8_ss(d1, desc_hi | (a0 + (uint32_t)kTileM), desc_hi | b0, idesc, sg > 0);
+                                tc::mma_i8_ss_acc(d0, desc_hi | a1, desc_hi | b1, idesc);
+                                tc::mma_i8_ss_acc(d1, desc_hi | (a1 + (uint32_t)kTileM), desc_hi | b1, idesc);
+                                tc::mma_i8_ss_acc(d0, desc_hi | a2, desc_hi | b2, idesc);
+                                tc::mma_i8_ss_acc(d1, desc_hi | (a2 + (uint32_t)kTileM), desc_hi | b2, idesc);
+                                tc::mma_i8_ss_acc(d0, desc_hi | a3, desc_hi | b3, idesc);
+                                tc::mma_i8_ss_acc(d1, desc_hi | (a3 + (uint32_t)kTileM), desc_hi | b3, idesc);
+                            } else {
+                                tc::mma_i8_ss(d0, desc_hi | a0, desc_hi | b0, idesc, sg > 0);
+                                tc::mma_i8_ss_acc(d0, desc_hi | a1, desc_hi | b1, idesc);
+                                tc::mma_i8_ss_acc(d0, desc_hi | a2, desc_hi | b2, idesc);
+                                tc::mma_i8_ss_acc(d0, desc_hi | a3, desc_hi | b3, idesc);
+                            }
+                            tc::mma_commit(&w_empty[st_cur]);
+                            cur = nxt;
+                        }
+                        if (!alive) break;
+                        tc::mma_commit(&acc_full[acc]);      // this pass's accumulators are complete
+                        if (pass == npass_cta - 1 && it < 8) RTN_TL(conv_i8s, 41 + 2 * it);
+                        if (p.nAcc == 2) { acc ^= 1u; if (acc == 0) acc_ph ^= 1u; } else acc_ph ^= 1u;
+                    }
+                    if (!alive) break;
+                    tc::mma_commit(&a_empty[buf]);
+                }
+            } else
             for (int g = s0; g < s1 && alive; g += rt, ++it) {
                 const int buf = p.nA == 2 ? (it & 1) : 0;
                 const uint32_t use_ph = p.nA == 2 ? ((it >> 1) & 1) : (it & 1);
@@ -608,8 +755,8 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                 const uint32_t a16 = (tc::smem_addr(smem + (buf ? p.off_a[1] : p.off_a[0])) >> 4) + a_lbo_field;
                 uint64_t* full = &a_full[buf * kMaxGroups];
                 uint32_t ready = 0;             // 32-channel groups whose codes are known to be written
-              for (int pass = 0; pass < p.npass && alive; ++pass) {
-                const int vt = it * p.npass + pass;
+              for (int pass = 0; pass < npass_cta && alive; ++pass) {
+                const int vt = it * npass_cta + pass;
                 const int slot_acc = p.nAcc == 2 ? (vt & 1) : 0;
                 const uint32_t acc_ph = p.nAcc == 2 ? ((vt >> 1) & 1) : (vt & 1);
                 alive = wait_or_die(&acc_empty[slot_acc], acc_ph ^ 1, a.status, dead);
@@ -651,7 +798,7 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                     if (alive) tc::mma_commit(&w_empty[st]);
                 }
                 if (alive) tc::mma_commit(&acc_full[slot_acc]);      // this pass's accumulators are complete
-                if (pass == p.npass - 1 && it < 8) RTN_TL(conv_i8s, 41 + 2 * it);
+                if (pass == npass_cta - 1 && it < 8) RTN_TL(conv_i8s, 41 + 2 * it);
               }
                 if (!alive) break;
                 tc::mma_commit(&a_empty[buf]);
@@ -716,17 +863,12 @@ static cudaError_t launch_i8s_mode(const ConvArgs& c, const NextLayerArgs& f, cu
 cudaError_t launch_conv_i8s(const ConvArgs& c, cudaStream_t s) { return launch_i8s_mode<false>(c, NextLayerArgs{}, s); }
 
 // Rough time of this variant for a shape, in microseconds (negative: not taken), for the choice between it
-// and the variant that splits the filter bank over CTAs.  Measured on B200: a CTA's time is the filter stream of
-// its tiles, about 0.75 us per 32 KB stage from scratch (1 us when the stage is expanded in the kernel),
-// whatever the batch, plus about 13 us of ternarizing, epilogue and launch.
+// and the variant that keeps a share of the filter bank resident per CTA.
 double conv_i8s_estimate_us(const ConvArgs& c)
 {
     ConvI8SPlan p;
     if (!make_plan_s(c, p, device_sm_count())) return -1.0;
-    const int strip_rows = (p.total_rows + p.grid - 1) / p.grid;
-    const int tiles = (strip_rows + p.RT - 1) / p.RT;
-    const double stage_us = (p.pre ? 0.75 : 1.0) * (double)p.NpP / 256.0;
-    return 13.0 + (double)tiles * p.npass * (p.nK / kSlices) * stage_us;
+    return plan_estimate_us(p);
 }
 
 // The same kernels with the hand-over to the next layer (and, optionally, packed input).

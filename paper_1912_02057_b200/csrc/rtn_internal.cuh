@@ -148,7 +148,7 @@ inline bool conv_prefers_streamed(const ConvArgs& c)
     // a strided 1x1 layer: the streamed-filter kernel gathers only the pixels some tap lands on, in one launch; the
     // split-bank pair reads and codes the whole input first (measured 22.8 against 24.9 us on 128 -> 256 at 28 x 28, batch 128)
     if (ts >= 0.0 && c.kh == 1 && c.kw == 1 && c.stride > 1) return true;
-    return ts >= 0.0 && (tr < 0.0 || ts <= 0.9 * tr);      // the estimates are rough: a tie goes to the split bank
+    return ts >= 0.0 && (tr < 0.0 || ts <= 0.95 * tr);     // the estimates are rough: a tie goes to the split bank
 }
 inline cudaError_t launch_conv_i8_any(const ConvArgs& c, cudaStream_t s)
 {
