@@ -71,6 +71,7 @@ constexpr int kTileM = 128;                            // pixels per MMA (TMEM l
 constexpr size_t kSmemLimit = 220 * 1024;
 constexpr int kConvBarrier = 1;                        // named barrier of the converter warps
 constexpr int kEpiBarrier = 2;                         // named barrier of the epilogue warps
+constexpr int kConstBarrier = 3;                       // epilogue warps arrive (constants written), helper warps wait
 
 struct ConvI8Plan {
     int PW, PH;            // padded image extent
@@ -243,23 +244,25 @@ __device__ __forceinline__ void issue_mmas(const ConvI8Plan& p, int i0, uint32_t
 }
 
 // Hand-over epilogue (NextLayerArgs) of one tile for one warp.  The warp reads TMEM lanes 32 q .. 32 q + 31
-// (pixels).  Unit of work = (sub-tile, block of 128 output channels), dealt to the two warps of a lane quarter
-// in turn: a thread then holds all 128 codes of its pixel and writes each bit plane of the packed row with
-// one 16-byte store.  Constants and the next layer's thresholds come from shared memory.
+// (pixels) and is warp `part` of the `nparts` (2 or 4) that share this lane quarter.  Unit of work = (sub-tile,
+// block of 128 output channels), dealt to those warps in turn: a thread then holds all 128 codes of its pixel and
+// writes each bit plane of the packed row with one 16-byte store.  Constants and the next layer's thresholds come
+// from shared memory.
 __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const ConvI8Plan& p, const NextLayerArgs& f,
                                                    const float4* sC, const float2* sT, uint32_t tmem, int buf, int g,
-                                                   int nrows, bool alive, int q, int lane, int half)
+                                                   int nrows, bool alive, int q, int lane, int part, int nparts)
 {
     const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
     const int64_t ostride = (int64_t)a.Ho * a.Wo;
     const int nblk16 = (a.N + 15) / 16;
     const int ncb = (a.N + kBlockCodes - 1) / kBlockCodes;
     const int nwords = a.N / 32;
-    if (ntm == 2 && a.pad_mode == RTN_PAD_CODE_ZERO && (a.N == 64 || a.N == 128)) {
-        // Full tile of a 64- or 128-filter layer without border classes: the two warps of a lane quarter split
-        // the output channels, and a thread takes its pixel of BOTH sub-tiles through its channels, 16 at a time
-        // (next_layer_block16_pair).  A warp writes its 32-bit words of each pixel's packed row; the words past N
-        // of a 64-filter row (its zero fill) are shared out between the two warps.
+    if (a.pad_mode == RTN_PAD_CODE_ZERO && (a.N == 64 || a.N == 128)) {
+        // A 64- or 128-filter layer without border classes: the warps of a lane quarter split the output
+        // channels, and a thread takes its pixel of BOTH sub-tiles (of the one, where the tile has one: the second
+        // pixel then does not exist and nothing is read or written for it) through its channels, 16 at a time
+        // (next_layer_block16_pair).  A warp writes its 32- or 16-bit pieces of each pixel's packed row; the words
+        // past N of a 64-filter row (its zero fill) are shared out between the warps.
         bool ok2[2];
         uint32_t trow2[2];
         int64_t obase2[2];
@@ -273,8 +276,8 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
             const uint32_t G = (uint32_t)g + row;
             const uint32_t b = fdiv(G, p.div_ph);
             const int ho = (int)(G - b * (uint32_t)p.PH);
-            ok2[t] = alive && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
-            trow2[t] = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + t) * p.Np);
+            ok2[t] = alive && t < ntm && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
+            trow2[t] = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + (t < ntm ? t : 0)) * p.Np);
             obase2[t] = (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
             row2[t] = (ok2[t] && f.out_packed != nullptr)
                           ? f.out_packed + (((int64_t)b * a.Ho + ho) * a.Wo + wo) * (int64_t)(ncb * kBlockBytes) : nullptr;
@@ -284,33 +287,48 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
         tc::tmem_ld_wait();
         const float fsx0 = (float)(int)sx2[0], fsx1 = (float)(int)sx2[1];
         const bool want = f.out_packed != nullptr;
-        for (int w = half * (nwords / 2); w < (half + 1) * (nwords / 2); ++w) {
-            uint32_t nz0 = 0, sg0 = 0, nz1 = 0, sg1 = 0;
-            #pragma unroll 1
-            for (int hb = 0; hb < 2; ++hb) {
-                const int n0 = w * 32 + hb * 16;
-                uint32_t u0[16], u1[16];
-                tc::tmem_ld16(trow2[0] + (uint32_t)n0, u0);
-                tc::tmem_ld16(trow2[1] + (uint32_t)n0, u1);
-                tc::tmem_ld_wait();
-                uint32_t a0, b0, a1, b1;
-                next_layer_block16_pair(a, f, u0, u1, sC + n0, sT + n0, fsx0, fsx1, ok2[0], ok2[1],
-                                        obase2[0] + (int64_t)n0 * ostride, obase2[1] + (int64_t)n0 * ostride, ostride, want,
-                                        a0, b0, a1, b1);
-                nz0 |= a0 << (16 * hb); sg0 |= b0 << (16 * hb);
-                nz1 |= a1 << (16 * hb); sg1 |= b1 << (16 * hb);
+        const int nb = nblk16 / nparts;                              // 16-channel blocks of this warp: 1, 2 or 4
+        uint32_t nz0 = 0, sg0 = 0, nz1 = 0, sg1 = 0;
+        #pragma unroll 1
+        for (int k = part * nb; k < (part + 1) * nb; ++k) {
+            const int n0 = k * 16;
+            uint32_t u0[16], u1[16];
+            tc::tmem_ld16(trow2[0] + (uint32_t)n0, u0);
+            tc::tmem_ld16(trow2[1] + (uint32_t)n0, u1);
+            tc::tmem_ld_wait();
+            uint32_t a0, b0, a1, b1;
+            next_layer_block16_pair(a, f, u0, u1, sC + n0, sT + n0, fsx0, fsx1, ok2[0], ok2[1],
+                                    obase2[0] + (int64_t)n0 * ostride, obase2[1] + (int64_t)n0 * ostride, ostride, want,
+                                    a0, b0, a1, b1);
+            const int off = (k >> 3) * kBlockBytes + ((k >> 1) & 3) * 4;      // the block's word in the packed row
+            if (nb == 1) {
+                // a lone block is half a word: 16-bit stores
+                if (row2[0] != nullptr) {
+                    *reinterpret_cast<uint16_t*>(row2[0] + off + 2 * (k & 1)) = (uint16_t)a0;
+                    *reinterpret_cast<uint16_t*>(row2[0] + off + 16 + 2 * (k & 1)) = (uint16_t)b0;
+                }
+                if (row2[1] != nullptr) {
+                    *reinterpret_cast<uint16_t*>(row2[1] + off + 2 * (k & 1)) = (uint16_t)a1;
+                    *reinterpret_cast<uint16_t*>(row2[1] + off + 16 + 2 * (k & 1)) = (uint16_t)b1;
+                }
+                continue;
             }
-            const int off = (w >> 2) * kBlockBytes + (w & 3) * 4;
-            if (row2[0] != nullptr) {
-                *reinterpret_cast<uint32_t*>(row2[0] + off) = nz0;
-                *reinterpret_cast<uint32_t*>(row2[0] + off + 16) = sg0;
-            }
-            if (row2[1] != nullptr) {
-                *reinterpret_cast<uint32_t*>(row2[1] + off) = nz1;
-                *reinterpret_cast<uint32_t*>(row2[1] + off + 16) = sg1;
+            // (nb is even and the warp's first block is even: blocks come in whole words)
+            nz0 |= a0 << (16 * (k & 1)); sg0 |= b0 << (16 * (k & 1));
+            nz1 |= a1 << (16 * (k & 1)); sg1 |= b1 << (16 * (k & 1));
+            if (k & 1) {
+                if (row2[0] != nullptr) {
+                    *reinterpret_cast<uint32_t*>(row2[0] + off) = nz0;
+                    *reinterpret_cast<uint32_t*>(row2[0] + off + 16) = sg0;
+                }
+                if (row2[1] != nullptr) {
+                    *reinterpret_cast<uint32_t*>(row2[1] + off) = nz1;
+                    *reinterpret_cast<uint32_t*>(row2[1] + off + 16) = sg1;
+                }
+                nz0 = sg0 = nz1 = sg1 = 0;
             }
         }
-        for (int w = nwords + half; w < ncb * 4; w += 2) {          // zero fill past N
+        for (int w = nwords + part; w < ncb * 4; w += nparts) {          // zero fill past N
             const int off = (w >> 2) * kBlockBytes + (w & 3) * 4;
             #pragma unroll
             for (int t = 0; t < 2; ++t)
@@ -350,7 +368,7 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
         bool sx_ready = false;
         float fsx = 0.f;
         for (int cb = 0; cb < ncb; ++cb) {
-            if (((tm * ncb + cb) & 1) != half) continue;
+            if ((tm * ncb + cb) % nparts != part) continue;
             uint32_t nzw[4] = {0u, 0u, 0u, 0u}, sgw[4] = {0u, 0u, 0u, 0u};
             #pragma unroll 1
             for (int k = 0; k < 8; ++k) {
@@ -409,6 +427,12 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nchunk = p.Cp / 16;
+    // Packed rows in and a full-precision stream out (a block's second layer: skip connection read, fp32 written): the
+    // converters' share of a tile is small (one table look-up per 32 codes) and the epilogue's, a chain of loads and
+    // stores per output, is the kernel's largest, so the converter warps take half of every tile's epilogue as well
+    // (four warps per TMEM lane quarter instead of two, twice the loads in flight).
+    bool helpers = false;
+    if constexpr (kNext) helpers = f.x_packed != nullptr && (f.skip != nullptr || a.out != nullptr);
     // this CTA's strip of padded rows
     const int s0 = (int)((int64_t)blockIdx.x * p.total_rows / p.grid);
     const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
@@ -425,8 +449,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         tc::mbar_init(&a_empty[1], 1);
         tc::mbar_init(&acc_full[0], 1);
         tc::mbar_init(&acc_full[1], 1);
-        tc::mbar_init(&acc_empty[0], kEpiThreads);
-        tc::mbar_init(&acc_empty[1], kEpiThreads);
+        tc::mbar_init(&acc_empty[0], kEpiThreads + (helpers ? kConvThreads : 0));
+        tc::mbar_init(&acc_empty[1], kEpiThreads + (helpers ? kConvThreads : 0));
         for (int i = 0; i < kMaxStages; ++i) {
             tc::mbar_init(&st_full[i], 1);
             tc::mbar_init(&st_empty[i], kConvThreads);
@@ -623,6 +647,37 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     tc::mbar_arrive(&a_full[p.strip ? it * ngroup + grp : buf * kMaxGroups + grp]);
             }
             if (tid == 0 && it < 8) RTN_TL(conv_i8, 25 + 2 * it);
+            if constexpr (kNext) {
+                // this warp's share of the previous tile's epilogue (the tile just converted feeds the tensor core
+                // meanwhile)
+                if (helpers && it > 0) {
+                    if (it == 1)        // the constants and thresholds the epilogue warps wrote at set-up
+                        asm volatile("bar.sync %0, %1;" ::"r"(kConstBarrier), "r"(kEpiThreads + kConvThreads) : "memory");
+                    const int pg = g - (it == 1 ? p.R0 : p.RT);
+                    role_wait(tid < 32, &acc_full[(it - 1) & 1], ((it - 1) >> 1) & 1, a.status, dead, kConvBarrier, kConvThreads);
+                    const bool alive = !*dead;
+                    tc::tc_fence_after_sync();
+                    next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, (it - 1) & 1, pg,
+                                       it == 1 ? p.R0 : p.RT, alive, warp & 3, lane, 2 + (tid >> 7), 4);
+                    tc::tc_fence_before_sync();
+                    tc::mbar_arrive(&acc_empty[(it - 1) & 1]);
+                }
+            }
+        }
+        if constexpr (kNext) {
+            if (helpers && it > 0) {                 // the strip's last tile
+                const int last = it - 1;
+                if (last == 0)
+                    asm volatile("bar.sync %0, %1;" ::"r"(kConstBarrier), "r"(kEpiThreads + kConvThreads) : "memory");
+                const int lg = s0 + (last == 0 ? 0 : p.R0 + (last - 1) * p.RT);
+                role_wait(tid < 32, &acc_full[last & 1], (last >> 1) & 1, a.status, dead, kConvBarrier, kConvThreads);
+                const bool alive = !*dead;
+                tc::tc_fence_after_sync();
+                next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, last & 1, lg,
+                                   min(last == 0 ? p.R0 : p.RT, s1 - lg), alive, warp & 3, lane, 2 + (tid >> 7), 4);
+                tc::tc_fence_before_sync();
+                tc::mbar_arrive(&acc_empty[last & 1]);
+            }
         }
     } else if (warp == kProdWarp) {
         // ------------------------------------------------------------ producer
@@ -812,6 +867,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             }
         }
         asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible
+        if (helpers) asm volatile("bar.arrive %0, %1;" ::"r"(kConstBarrier), "r"(kEpiThreads + kConvThreads) : "memory");
         tc::pdl_wait();                             // out may still be read by the previous kernel
         if (etid == 0) RTN_TL(conv_i8, 3);
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;      // kEpiWarp0 is a multiple of 4
@@ -848,7 +904,7 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             if (etid == 0 && it < 8) RTN_TL(conv_i8, 56 + 2 * it);
             if constexpr (kNext) {
                 next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, buf, g, nrows,
-                                   alive, q, lane, half);
+                                   alive, q, lane, half, helpers ? 4 : 2);
             } else if (p.const_tmem && a.dbg_acc == nullptr && ntm == 2 && a.pad_mode == RTN_PAD_CODE_ZERO) {
                 // Full tile, constants in tensor memory, no border classes: the thread's pixels of both
                 // sub-tiles go through the channel blocks together, so that one fetch of a block's
