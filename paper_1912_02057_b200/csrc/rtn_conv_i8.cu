@@ -71,7 +71,6 @@ constexpr int kTileM = 128;                            // pixels per MMA (TMEM l
 constexpr size_t kSmemLimit = 220 * 1024;
 constexpr int kConvBarrier = 1;                        // named barrier of the converter warps
 constexpr int kEpiBarrier = 2;                         // named barrier of the epilogue warps
-constexpr int kConstBarrier = 3;                       // epilogue warps arrive (constants written), helper warps wait
 
 struct ConvI8Plan {
     int PW, PH;            // padded image extent
@@ -427,12 +426,6 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nchunk = p.Cp / 16;
-    // Packed rows in and a full-precision stream out (a block's second layer: skip connection read, fp32 written): the
-    // converters' share of a tile is small (one table look-up per 32 codes) and the epilogue's, a chain of loads and
-    // stores per output, is the kernel's largest, so the converter warps take half of every tile's epilogue as well
-    // (four warps per TMEM lane quarter instead of two, twice the loads in flight).
-    bool helpers = false;
-    if constexpr (kNext) helpers = f.x_packed != nullptr && (f.skip != nullptr || a.out != nullptr);
     // this CTA's strip of padded rows
     const int s0 = (int)((int64_t)blockIdx.x * p.total_rows / p.grid);
     const int s1 = (int)((int64_t)(blockIdx.x + 1) * p.total_rows / p.grid);
@@ -449,8 +442,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         tc::mbar_init(&a_empty[1], 1);
         tc::mbar_init(&acc_full[0], 1);
         tc::mbar_init(&acc_full[1], 1);
-        tc::mbar_init(&acc_empty[0], kEpiThreads + (helpers ? kConvThreads : 0));
-        tc::mbar_init(&acc_empty[1], kEpiThreads + (helpers ? kConvThreads : 0));
+        tc::mbar_init(&acc_empty[0], kEpiThreads);
+        tc::mbar_init(&acc_empty[1], kEpiThreads);
         for (int i = 0; i < kMaxStages; ++i) {
             tc::mbar_init(&st_full[i], 1);
             tc::mbar_init(&st_empty[i], kConvThreads);
@@ -647,37 +640,6 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     tc::mbar_arrive(&a_full[p.strip ? it * ngroup + grp : buf * kMaxGroups + grp]);
             }
             if (tid == 0 && it < 8) RTN_TL(conv_i8, 25 + 2 * it);
-            if constexpr (kNext) {
-                // this warp's share of the previous tile's epilogue (the tile just converted feeds the tensor core
-                // meanwhile)
-                if (helpers && it > 0) {
-                    if (it == 1)        // the constants and thresholds the epilogue warps wrote at set-up
-                        asm volatile("bar.sync %0, %1;" ::"r"(kConstBarrier), "r"(kEpiThreads + kConvThreads) : "memory");
-                    const int pg = g - (it == 1 ? p.R0 : p.RT);
-                    role_wait(tid < 32, &acc_full[(it - 1) & 1], ((it - 1) >> 1) & 1, a.status, dead, kConvBarrier, kConvThreads);
-                    const bool alive = !*dead;
-                    tc::tc_fence_after_sync();
-                    next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, (it - 1) & 1, pg,
-                                       it == 1 ? p.R0 : p.RT, alive, warp & 3, lane, 2 + (tid >> 7), 4);
-                    tc::tc_fence_before_sync();
-                    tc::mbar_arrive(&acc_empty[(it - 1) & 1]);
-                }
-            }
-        }
-        if constexpr (kNext) {
-            if (helpers && it > 0) {                 // the strip's last tile
-                const int last = it - 1;
-                if (last == 0)
-                    asm volatile("bar.sync %0, %1;" ::"r"(kConstBarrier), "r"(kEpiThreads + kConvThreads) : "memory");
-                const int lg = s0 + (last == 0 ? 0 : p.R0 + (last - 1) * p.RT);
-                role_wait(tid < 32, &acc_full[last & 1], (last >> 1) & 1, a.status, dead, kConvBarrier, kConvThreads);
-                const bool alive = !*dead;
-                tc::tc_fence_after_sync();
-                next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, last & 1, lg,
-                                   min(last == 0 ? p.R0 : p.RT, s1 - lg), alive, warp & 3, lane, 2 + (tid >> 7), 4);
-                tc::tc_fence_before_sync();
-                tc::mbar_arrive(&acc_empty[last & 1]);
-            }
         }
     } else if (warp == kProdWarp) {
         // ------------------------------------------------------------ producer
@@ -867,7 +829,6 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             }
         }
         asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");     // constants visible
-        if (helpers) asm volatile("bar.arrive %0, %1;" ::"r"(kConstBarrier), "r"(kEpiThreads + kConvThreads) : "memory");
         tc::pdl_wait();                             // out may still be read by the previous kernel
         if (etid == 0) RTN_TL(conv_i8, 3);
         const int q = warp & 3, half = (warp - kEpiWarp0) >> 2;      // kEpiWarp0 is a multiple of 4
@@ -904,10 +865,11 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             if (etid == 0 && it < 8) RTN_TL(conv_i8, 56 + 2 * it);
             if constexpr (kNext) {
                 next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, buf, g, nrows,
-                                   alive, q, lane, half, helpers ? 4 : 2);
-            } else if (p.const_tmem && a.dbg_acc == nullptr && ntm == 2 && a.pad_mode == RTN_PAD_CODE_ZERO) {
-                // Full tile, constants in tensor memory, no border classes: the thread's pixels of both
-                // sub-tiles go through the channel blocks together, so that one fetch of a block's
+                                   alive, q, lane, half, 2);
+            } else if (p.const_tmem && a.dbg_acc == nullptr && a.pad_mode == RTN_PAD_CODE_ZERO) {
+                // Constants in tensor memory, no border classes: the thread's pixels of both sub-tiles (where the
+                // tile has one sub-tile, the second pixel does not exist and nothing is stored for it) go
+                // through the channel blocks together, so that one fetch of a block's
                 // constants serves two pixels and the epilogue waits for tensor memory half as often
                 // (the wait for a tcgen05.ld, several hundred cycles while the tensor core works on the next
                 // tile, is what this epilogue's time is made of).
@@ -922,8 +884,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     const uint32_t G = (uint32_t)g + row;
                     const uint32_t b = fdiv(G, p.div_ph);
                     const int ho = (int)(G - b * (uint32_t)p.PH);
-                    ok2[t] = alive && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
-                    trow2[t] = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + t) * p.Np);
+                    ok2[t] = alive && t < ntm && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
+                    trow2[t] = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + (t < ntm ? t : 0)) * p.Np);
                     optr2[t] = a.out + (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
                     asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
                                  : "=r"(sx2[t]) : "r"(trow2[t] + (uint32_t)a.N) : "memory");
