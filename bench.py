@@ -540,6 +540,14 @@ def run_peaks(ctx):
             entry["source"] = ("measured: rtn_probe_peak_popc, AND + XOR-AND + 2 popcounts + 2 adds per 32 code pairs "
                                "on registers, 1024 threads per SM, event-timed")
         out[name] = entry
+    # what one tensor-core instruction of a narrower accumulator costs with nothing else in the way (cycles per
+    # instruction from the in-kernel counts): the floor under the conv kernels' 64- to 128-column instructions
+    widths = {}
+    for n_cols in (32, 64, 80, 128, 256):
+        cyc, _ = rtn.rtn_probe_i8_rate(n_cols, 4096)
+        torch.cuda.synchronize()
+        widths[str(n_cols)] = float(np.median(cyc.cpu().numpy())) / 4096.0
+    out["i8"]["cycles_per_mma_by_columns"] = widths
     if rtn.rtn_last_device_status() != 0:
         raise RuntimeError("device status after the peak probes")
     # what a plain copy reaches at the size of the HBM-bound conv configurations (25.7 MB in, 25.7 MB out):

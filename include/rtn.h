@@ -269,6 +269,9 @@ rtn_status rtn_selftest_wait_timeout(int64_t polls, int32_t* gave_up, void* stre
  *   rtn_probe_peak_i8   n_mma (1..2^22) tcgen05.mma kind::i8 of M = 128, N = 256, K = 32 per CTA, operands in
  *                       shared memory, one accumulator; rtn_probe_i8_ops_per_mma() = 2*128*256*32 operations each.
  *                       The final wait is bounded like every other (rtn_last_device_status reports a time-out).
+ *   rtn_probe_i8_rate   the same loop with accumulators of n_cols columns (a multiple of 16 in 16..256): what one
+ *                       instruction of that width costs when nothing else is in the way (narrow instructions do not
+ *                       get cheaper in proportion); 2*128*n_cols*32 operations each.
  *   rtn_probe_peak_popc rounds (1..2^24) rounds per thread of 64 word pairs, 1024 threads per CTA, registers
  *                       only; rtn_probe_popc_ops_per_round() operations (2 per code pair) per CTA and round.
  *                       `sink`: device int32 the kernel never writes in practice (keeps the loop alive).
@@ -280,6 +283,7 @@ int64_t rtn_probe_ctas(void);
 int64_t rtn_probe_i8_ops_per_mma(void);
 int64_t rtn_probe_popc_ops_per_round(void);
 rtn_status rtn_probe_peak_i8(int64_t n_mma, int64_t* cycles, void* stream);
+rtn_status rtn_probe_i8_rate(int64_t n_cols, int64_t n_mma, int64_t* cycles, void* stream);
 rtn_status rtn_probe_peak_popc(int64_t rounds, int64_t* cycles, int32_t* sink, void* stream);
 rtn_status rtn_probe_copy(const void* src, void* dst, int64_t bytes, void* stream);
 

@@ -105,6 +105,8 @@ def lib():
         L.rtn_probe_popc_ops_per_round.argtypes = []
         L.rtn_probe_peak_i8.restype = _int
         L.rtn_probe_peak_i8.argtypes = [_i64, _vp, _vp]
+        L.rtn_probe_i8_rate.restype = _int
+        L.rtn_probe_i8_rate.argtypes = [_i64, _i64, _vp, _vp]
         L.rtn_probe_peak_popc.restype = _int
         L.rtn_probe_peak_popc.argtypes = [_i64, _vp, _vp, _vp]
         L.rtn_probe_copy.restype = _int
@@ -334,6 +336,15 @@ def rtn_probe_peak_i8(n_mma, stream=None):
     cycles = torch.zeros((ctas,), dtype=torch.int64, device="cuda")
     _check(lib().rtn_probe_peak_i8(int(n_mma), _ptr(cycles, torch.int64), _stream(stream)), "rtn_probe_peak_i8")
     return cycles, int(n_mma) * int(lib().rtn_probe_i8_ops_per_mma())
+
+
+def rtn_probe_i8_rate(n_cols, n_mma, stream=None):
+    """The tensor-pipe probe with accumulators of n_cols columns; returns (cycles int64 [CTAs] on the device,
+    operations per CTA)."""
+    ctas = int(lib().rtn_probe_ctas())
+    cycles = torch.zeros((ctas,), dtype=torch.int64, device="cuda")
+    _check(lib().rtn_probe_i8_rate(int(n_cols), int(n_mma), _ptr(cycles, torch.int64), _stream(stream)), "rtn_probe_i8_rate")
+    return cycles, int(n_mma) * 2 * 128 * int(n_cols) * 32
 
 
 def rtn_probe_peak_popc(rounds, stream=None):

@@ -1,6 +1,7 @@
 // Peak probes: the two non-memory ceilings the contraction kernels are measured against, as committed code.
-//   probe_i8_kernel    one CTA per SM issues tcgen05.mma kind::i8 (M = 128, N = 256, K = 32) back to back on
-//                      operands that stay in shared memory: int8 tensor-pipe rate, nothing else in the way.
+//   probe_i8_kernel    one CTA per SM issues tcgen05.mma kind::i8 (M = 128, N = 256 or a given column count,
+//                      K = 32) back to back on operands that stay in shared memory: int8 tensor-pipe rate, nothing
+//                      else in the way.
 //   probe_popc_kernel  every thread runs the inner product of Eq. 9 (AND, XOR-AND, two popcounts, two adds per
 //                      32 code pairs) on registers only: issue rate of the bit-plane kernels' instruction mix.
 // Both write the SM-clock cycles each CTA spent in its loop; the caller times the launch with events as well.
@@ -23,7 +24,7 @@ __device__ __forceinline__ uint32_t mix(uint32_t v)
 }
 
 __global__ void __launch_bounds__(kProbeThreads, 1)
-probe_i8_kernel(uint32_t n_mma, long long* cycles, unsigned* status)
+probe_i8_kernel(uint32_t n_cols, uint32_t n_mma, long long* cycles, unsigned* status)
 {
     // [K chunk of 16 B][row][16 B]: the K-major no-swizzle operand layout of the contraction kernels
     __shared__ __align__(128) uint8_t sA[2 * kProbeM * 16];
@@ -40,7 +41,7 @@ probe_i8_kernel(uint32_t n_mma, long long* cycles, unsigned* status)
         const uint32_t r = mix(i * 2246822519u + 77u * blockIdx.x);
         reinterpret_cast<uint32_t*>(sB)[i] = __byte_perm(0x0100FF00u, 0u, r & 0x3333u);
     }
-    if (warp == 0) tc::tmem_alloc(&slot, kProbeN);
+    if (warp == 0) tc::tmem_alloc(&slot, kProbeN);            // (the largest column count)
     if (threadIdx.x == 32) {
         tc::mbar_init(&done, 1);
         tc::mbar_init_fence();
@@ -52,8 +53,8 @@ probe_i8_kernel(uint32_t n_mma, long long* cycles, unsigned* status)
     const uint32_t tmem = slot;
     if (threadIdx.x == 0) {
         const uint64_t a_desc = tc::smem_desc_kmajor(tc::smem_addr(sA), kProbeM * 16, 128);
-        const uint64_t b_desc = tc::smem_desc_kmajor(tc::smem_addr(sB), kProbeN * 16, 128);
-        const uint32_t idesc = tc::idesc_i8(kProbeM, kProbeN);
+        const uint64_t b_desc = tc::smem_desc_kmajor(tc::smem_addr(sB), n_cols * 16, 128);
+        const uint32_t idesc = tc::idesc_i8(kProbeM, n_cols);
         const long long t0 = clock64();
         tc::mma_i8_ss(tmem, a_desc, b_desc, idesc, false);
         for (uint32_t i = 1; i < n_mma; ++i) tc::mma_i8_ss_acc(tmem, a_desc, b_desc, idesc);
@@ -125,13 +126,19 @@ int64_t rtn_probe_popc_ops_per_round(void)
 
 rtn_status rtn_probe_peak_i8(int64_t n_mma, int64_t* cycles, void* stream)
 {
+    return rtn_probe_i8_rate(rtn::kProbeN, n_mma, cycles, stream);
+}
+
+rtn_status rtn_probe_i8_rate(int64_t n_cols, int64_t n_mma, int64_t* cycles, void* stream)
+{
     if (cycles == nullptr) return RTN_ERR_NULL;
     if (n_mma < 1 || n_mma > (1 << 22)) return RTN_ERR_SHAPE;
+    if (n_cols < 16 || n_cols > rtn::kProbeN || n_cols % 16 != 0) return RTN_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(cycles) % 8 != 0) return RTN_ERR_ALIGN;
     unsigned* word = rtn::device_status_word();      // receives a time-out of the final (bounded) wait
     if (word == nullptr) return RTN_ERR_CUDA;
     rtn::probe_i8_kernel<<<(unsigned)rtn::device_sm_count(), rtn::kProbeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        (uint32_t)n_mma, reinterpret_cast<long long*>(cycles), word);
+        (uint32_t)n_cols, (uint32_t)n_mma, reinterpret_cast<long long*>(cycles), word);
     return cudaGetLastError() == cudaSuccess ? RTN_OK : RTN_ERR_CUDA;
 }
 

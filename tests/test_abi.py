@@ -89,3 +89,26 @@ def test_gemm_kernel_launches_follow_the_operand_expansion():
     if rtn.rtn_choose_gemm_variant(4096, 4096, 4096) == rtn.VARIANT_I8:
         assert rtn.rtn_gemm_kernel_launches(4096, 4096, 4096) == 2    # operands expanded ahead, then the contraction
         assert rtn.rtn_gemm_kernel_launches(128, 4096, 4096) == 1     # one row tile: everything inside the kernel
+
+
+def test_probe_argument_errors_without_a_gpu():
+    # RTN_ERR_NULL = 1, RTN_ERR_SHAPE = 2, RTN_ERR_ALIGN = 3 (rtn.h)
+    L = ctypes.CDLL(rtn.lib_path())
+    for f in (L.rtn_probe_peak_i8, L.rtn_probe_i8_rate, L.rtn_probe_peak_popc, L.rtn_probe_copy):
+        f.restype = ctypes.c_int
+    buf = ctypes.create_string_buffer(64)
+    ok = ctypes.cast(buf, ctypes.c_void_p)
+    odd = ctypes.c_void_p(ok.value + 4)
+    i64, vp = ctypes.c_int64, ctypes.c_void_p
+    assert L.rtn_probe_peak_i8(i64(8), vp(None), vp(None)) == 1
+    assert L.rtn_probe_peak_i8(i64(0), ok, vp(None)) == 2
+    assert L.rtn_probe_i8_rate(i64(64), i64(8), vp(None), vp(None)) == 1
+    for bad_cols in (0, 8, 24, 272):
+        assert L.rtn_probe_i8_rate(i64(bad_cols), i64(8), ok, vp(None)) == 2
+    assert L.rtn_probe_i8_rate(i64(64), i64(8), odd, vp(None)) == 3
+    assert L.rtn_probe_peak_popc(i64(8), vp(None), ok, vp(None)) == 1
+    assert L.rtn_probe_peak_popc(i64(0), ok, ok, vp(None)) == 2
+    assert L.rtn_probe_copy(vp(None), ok, i64(16), vp(None)) == 1
+    assert L.rtn_probe_copy(ok, ok, i64(24), vp(None)) == 2
+    assert L.rtn_probe_copy(odd, ok, i64(16), vp(None)) == 3
+    assert L.rtn_probe_i8_ops_per_mma() == 2 * 128 * 256 * 32
