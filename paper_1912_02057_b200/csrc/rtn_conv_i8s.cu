@@ -254,37 +254,38 @@ __device__ __forceinline__ void role_wait(bool leader, uint64_t* bar, uint32_t p
 }
 
 // The filter bank expanded once: wexp[pass][stage][16-byte k chunk (8)][filter row of the pass][16 B], the bytes a ring
-// stage holds, in the slice order of the plan (32-channel group outer, tap inner).  Thread = (stage, filter row).
+// stage holds, in the slice order of the plan (32-channel group outer, tap inner).  Thread = (stage, slice of the
+// stage, filter row): one word of each bit plane in, 32 bytes out (the kernel is a launch and one round trip to
+// memory long, so the work is spread thin).
 __global__ void __launch_bounds__(256)
 conv_expand_filters_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, uint4* __restrict__ wexp)
 {
     tc::pdl_trigger();          // the contraction kernel may start its set-up (it reads no expanded filters there)
     const int nstages = p.nK / kSlices;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= (int64_t)p.npass * nstages * p.NpP) return;
-    const int st = (int)(i / p.NpP);                        // pass * nstages + stage of the pass
-    const int row = (int)(i % p.NpP) + (st / nstages) * p.NpP;      // filter
+    if (i >= (int64_t)p.npass * nstages * kSlices * p.NpP) return;
+    const int r = (int)(i % p.NpP);
+    const int sj = (int)(i / p.NpP);                         // (pass * nstages + stage of the pass) * kSlices + slice
+    const int j = sj % kSlices, st = sj / kSlices;
+    const int row = r + (st / nstages) * p.NpP;             // filter
     const int stage_of_pass = st % nstages;
     const int cwords = p.Cp / 32, nwords = p.T * cwords;
     const int64_t row_blocks = ((int64_t)p.T * cwords + 3) / 4;
-    const uint32_t* Wrow = reinterpret_cast<const uint32_t*>(a.w_packed) + (int64_t)row * row_blocks * 8;
-    uint4* dst = wexp + (int64_t)st * kSlices * 2 * p.NpP + (i % p.NpP);
-    #pragma unroll
-    for (int j = 0; j < kSlices; ++j) {
-        // slice stage*4 + j of the stream = (32-channel group h, tap t) = word t*cwords + h of the packed row
-        const int s = stage_of_pass * kSlices + j;
-        uint32_t nz = 0, sg = 0;
-        if (s < nwords && row < a.N) {
-            const int h = s / p.T, t = s - h * p.T;
-            const int word = t * cwords + h;
-            nz = __ldg(Wrow + (word >> 2) * 8 + (word & 3));
-            sg = __ldg(Wrow + (word >> 2) * 8 + 4 + (word & 3));
-        }
-        uint32_t o[8];
-        tc::unpack32(nz, sg, o);
-        dst[(2 * j) * p.NpP] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[(2 * j + 1) * p.NpP] = make_uint4(o[4], o[5], o[6], o[7]);
+    // slice stage*4 + j of the stream = (32-channel group h, tap t) = word t*cwords + h of the packed row
+    const int sl = stage_of_pass * kSlices + j;
+    uint32_t nz = 0, sg = 0;
+    if (sl < nwords && row < a.N) {
+        const uint32_t* Wrow = reinterpret_cast<const uint32_t*>(a.w_packed) + (int64_t)row * row_blocks * 8;
+        const int h = sl / p.T, t = sl - h * p.T;
+        const int word = t * cwords + h;
+        nz = __ldg(Wrow + (word >> 2) * 8 + (word & 3));
+        sg = __ldg(Wrow + (word >> 2) * 8 + 4 + (word & 3));
     }
+    uint32_t o[8];
+    tc::unpack32(nz, sg, o);
+    uint4* dst = wexp + ((int64_t)st * kSlices + j) * 2 * p.NpP + r;
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[p.NpP] = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
 // kPre: the filter stages come from the scratch buffer conv_expand_filters_kernel wrote (bulk copies by
@@ -845,7 +846,7 @@ static cudaError_t launch_i8s_mode(const ConvArgs& c, const NextLayerArgs& f, cu
     void* scratch = nullptr;
     cudaError_t e = cudaMallocAsync(&scratch, bytes, s);
     if (e != cudaSuccess) return e;
-    const int64_t items = (int64_t)p.npass * nstages * p.NpP;
+    const int64_t items = (int64_t)p.npass * nstages * kSlices * p.NpP;
     conv_expand_filters_kernel<<<(unsigned)((items + 255) / 256), 256, 0, s>>>(c, p, reinterpret_cast<uint4*>(scratch));
     e = cudaGetLastError();
     if (e == cudaSuccess)
