@@ -1010,11 +1010,16 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                     if (!sx_ready) { fsx = (float)(int)sx_raw; sx_ready = true; }
                     if (ok) {
                         if (!border && dptr == nullptr && n0 + 16 <= a.N) {
+                            // results first, stores after (a load of the next constants may not pass a global store)
+                            float r[16];
                             #pragma unroll
                             for (int j = 0; j < 16; ++j) {
                                 const float4 c = sC[n0 + j];
-                                optr[(int64_t)(n0 + j) * ostride] = fmaf(c.x, (float)(int)u[j], fmaf(c.y, fsx, c.z));
+                                r[j] = fmaf(c.x, (float)(int)u[j], fmaf(c.y, fsx, c.z));
                             }
+                            float* o = optr + (int64_t)n0 * ostride;
+                            #pragma unroll
+                            for (int j = 0; j < 16; ++j, o += ostride) *o = r[j];
                         } else {
                             #pragma unroll
                             for (int j = 0; j < 16; ++j) {

@@ -547,11 +547,16 @@ conv_i8r_kernel(const ConvArgs a, const __grid_constant__ ConvI8RPlan p, const u
                 }
                 float* optr = a.out + obase + (int64_t)n0 * ostride;
                 if (!border && a.dbg_acc == nullptr && n0 + 16 <= a.N) {
+                    // results first, stores after: a shared-memory load may not be moved above a global store the
+                    // compiler cannot tell apart from it, and alternating the two made every column wait for the last
+                    float r[16];
                     #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const float4 c = sC[r0 + j];
-                        optr[(int64_t)j * ostride] = fmaf(c.x, (float)(int)v[j], fmaf(c.y, fsx, c.z));
+                        r[j] = fmaf(c.x, (float)(int)v[j], fmaf(c.y, fsx, c.z));
                     }
+                    #pragma unroll
+                    for (int j = 0; j < 16; ++j, optr += ostride) *optr = r[j];
                 } else {
                     #pragma unroll
                     for (int j = 0; j < 16; ++j) {

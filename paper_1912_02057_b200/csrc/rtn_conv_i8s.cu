@@ -557,11 +557,18 @@ conv_i8s_kernel(const ConvArgs a, const __grid_constant__ ConvI8SPlan p, const u
                         continue;
                     }
                     if (!border && dptr == nullptr && n0 + 16 <= a.N) {
+                        // all sixteen results first, then the stores: a shared-memory load of the next column's
+                        // constants may not be moved above a global store the compiler cannot tell apart from it, so
+                        // with load and store alternating every column waited for the one before
+                        float r[16];
                         #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const float4 c = sC[n0 + j];
-                            optr[(int64_t)(n0 + j) * ostride] = fmaf(c.x, (float)(int)v[j], fmaf(c.y, fsx, c.z));
+                            r[j] = fmaf(c.x, (float)(int)v[j], fmaf(c.y, fsx, c.z));
                         }
+                        float* o = optr + (int64_t)n0 * ostride;
+                        #pragma unroll
+                        for (int j = 0; j < 16; ++j, o += ostride) *o = r[j];
                     } else {
                         #pragma unroll
                         for (int j = 0; j < 16; ++j) {
