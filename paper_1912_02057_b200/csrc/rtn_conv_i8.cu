@@ -96,6 +96,9 @@ struct ConvI8Plan {
     uint32_t box_bytes;    // one TMA box: 32 channels x one image row of fp32
     int nslots;            // row slots of the TMA ring
     uint32_t off_stage;
+    int sk_stage;          // the skip connection's values of a tile are staged in shared memory by TMA (set by the launcher)
+    int sk_groups;         // 32-channel groups of the output (boxes per row)
+    uint32_t off_skip, sk_box;     // two buffers of RT rows x sk_groups boxes of sk_box bytes (32 channels x one output row)
     uint32_t off_a[2], off_w, off_lo, off_hi, off_c, off_t, off_rows, off_bar, off_misc;
     size_t smem_bytes;
     // Per MMA of a sub-tile (tap t, channel group h), in 16-byte units: start of the A window
@@ -179,6 +182,7 @@ bool make_plan(const ConvArgs& c, ConvI8Plan& p, int sms, bool next = false)
     if (o > kSmemLimit) return false;
     // staging ring for TMA
     p.use_tma = 0; p.stages = 0; p.nslots = 0; p.off_stage = o;
+    p.sk_stage = 0; p.sk_groups = 0; p.off_skip = 0; p.sk_box = 0;
     p.box_bytes = 32u * (uint32_t)c.W * 4u;
     const bool tma_ok = (c.W % 4 == 0) && (reinterpret_cast<uintptr_t>(c.x) % 16 == 0);
     if (tma_ok) {
@@ -247,9 +251,11 @@ __device__ __forceinline__ void issue_mmas(const ConvI8Plan& p, int i0, uint32_t
 // block of 128 output channels), dealt to those warps in turn: a thread then holds all 128 codes of its pixel and
 // writes each bit plane of the packed row with one 16-byte store.  Constants and the next layer's thresholds come
 // from shared memory.
+template <bool kSk>
 __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const ConvI8Plan& p, const NextLayerArgs& f,
                                                    const float4* sC, const float2* sT, uint32_t tmem, int buf, int g,
-                                                   int nrows, bool alive, int q, int lane, int part, int nparts)
+                                                   int nrows, bool alive, int q, int lane, int part, int nparts,
+                                                   const float* sk_buf)
 {
     const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
     const int64_t ostride = (int64_t)a.Ho * a.Wo;
@@ -267,6 +273,7 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
         int64_t obase2[2];
         uint8_t* row2[2];
         uint32_t sx2[2];
+        const float* sk2[2];                        // the pixel's staged skip values: channel n at sk2[t][skip_index(n)]
         #pragma unroll
         for (int t = 0; t < 2; ++t) {
             const uint32_t pl = (uint32_t)(t * kTileM + q * 32 + lane);
@@ -278,6 +285,8 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
             ok2[t] = alive && t < ntm && (int)row < nrows && b < (uint32_t)a.B && ho < a.Ho && wo < a.Wo;
             trow2[t] = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * p.TM + (t < ntm ? t : 0)) * p.Np);
             obase2[t] = (((int64_t)b * a.N) * a.Ho + ho) * a.Wo + wo;
+            // staged as [row of the tile][32-channel group][channel][Wo]
+            sk2[t] = kSk ? sk_buf + (size_t)row * p.sk_groups * (p.sk_box / 4) + wo : nullptr;
             row2[t] = (ok2[t] && f.out_packed != nullptr)
                           ? f.out_packed + (((int64_t)b * a.Ho + ho) * a.Wo + wo) * (int64_t)(ncb * kBlockBytes) : nullptr;
             asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
@@ -296,9 +305,12 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
             tc::tmem_ld16(trow2[1] + (uint32_t)n0, u1);
             tc::tmem_ld_wait();
             uint32_t a0, b0, a1, b1;
-            next_layer_block16_pair(a, f, u0, u1, sC + n0, sT + n0, fsx0, fsx1, ok2[0], ok2[1],
-                                    obase2[0] + (int64_t)n0 * ostride, obase2[1] + (int64_t)n0 * ostride, ostride, want,
-                                    a0, b0, a1, b1);
+            // (channel n0 + j of the staging buffer: group n0 / 32, channel n0 % 32 + j of the group, a.Wo floats apart)
+            const int sk_off = ((n0 >> 5) * 32 + (n0 & 31)) * a.Wo;
+            next_layer_block16_pair<kSk>(a, f, u0, u1, sC + n0, sT + n0, fsx0, fsx1, ok2[0], ok2[1],
+                                         obase2[0] + (int64_t)n0 * ostride, obase2[1] + (int64_t)n0 * ostride, ostride, want,
+                                         a0, b0, a1, b1, kSk ? sk2[0] + sk_off : nullptr, kSk ? sk2[1] + sk_off : nullptr,
+                                         a.Wo);
             const int off = (k >> 3) * kBlockBytes + ((k >> 1) & 3) * 4;      // the block's word in the packed row
             if (nb == 1) {
                 // a lone block is half a word: 16-bit stores
@@ -402,7 +414,9 @@ __device__ __forceinline__ void next_epilogue_tile(const ConvArgs& a, const Conv
 // kNext: the layer hands its result to the next one (NextLayerArgs): the input may come as packed pixel
 // rows (the converters then expand bit planes instead of ternarizing fp32), and the epilogue applies
 // phi, adds the skip connection and writes fp32 and / or packed Eq. 3 codes.
-template <bool kNext>
+// kSk (only with kNext, packed input and a skip connection): the producer warp stages each tile's skip values in
+// shared memory by TMA (ConvI8Plan::sk_stage), and the epilogue reads them from there.
+template <bool kNext, bool kSk = false>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __grid_constant__ CUtensorMap tmap,
                const NextLayerArgs f)
@@ -446,7 +460,8 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
         tc::mbar_init(&acc_empty[1], kEpiThreads);
         for (int i = 0; i < kMaxStages; ++i) {
             tc::mbar_init(&st_full[i], 1);
-            tc::mbar_init(&st_empty[i], kConvThreads);
+            // (staged skip values: slots 0, 1 = the two tile buffers, released by the epilogue's threads)
+            tc::mbar_init(&st_empty[i], kSk ? kEpiThreads : kConvThreads);
         }
         tc::mbar_init_fence();
         *dead = 0;
@@ -712,6 +727,44 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
                 if (lane == 0 && it < 8) RTN_TL(conv_i8, 9 + 2 * it);
             }
         }
+        if constexpr (kNext && kSk) {
+            {
+                // The skip connection's values of tile it go to buffer it & 1, one box (32 channels x one output row)
+                // per row and channel group, a tile ahead of the epilogue that reads them.
+                tc::pdl_wait();                         // the skip tensor may be the previous kernel's output
+                const uint32_t stage0 = tc::smem_addr(smem + p.off_skip);
+                bool alive = true;
+                int it = 0;
+                for (int g = s0; g < s1 && alive; g += it == 0 ? p.R0 : p.RT, ++it) {
+                    const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
+                    const int buf = it & 1;
+                    uint32_t info = 0xFFFFFFFFu;        // lane j: output row of the tile's row j, if it is one
+                    if (lane < nrows) {
+                        const uint32_t G = (uint32_t)(g + lane);
+                        const uint32_t b = fdiv(G, p.div_ph);
+                        const int ho = (int)(G - b * (uint32_t)p.PH);
+                        if (b < (uint32_t)a.B && ho < a.Ho) info = (b << 11) | (uint32_t)ho;
+                    }
+                    const uint32_t mask = __ballot_sync(0xffffffffu, info != 0xFFFFFFFFu);
+                    bool ok = true;
+                    if (lane == 0) ok = wait_or_die(&st_empty[buf], ((it >> 1) & 1) ^ 1, a.status, dead);
+                    if (!__shfl_sync(0xffffffffu, ok ? 1 : 0, 0)) { alive = false; break; }
+                    if (lane == 0) {
+                        if (mask == 0) tc::mbar_arrive(&st_full[buf]);
+                        else mbar_expect_tx(&st_full[buf], (uint32_t)__popc(mask) * (uint32_t)p.sk_groups * p.sk_box);
+                    }
+                    __syncwarp();
+                    // lane j issues the boxes of row j
+                    if (info != 0xFFFFFFFFu) {
+                        const uint32_t bar = tc::smem_addr(&st_full[buf]);
+                        for (int gq = 0; gq < p.sk_groups; ++gq)
+                            tma_load_row(stage0 + (uint32_t)(((buf * p.RT + lane) * p.sk_groups + gq)) * p.sk_box, &tmap,
+                                         (int)(info & 0x7FFu), gq * 32, (int)(info >> 11), bar);
+                    }
+                    __syncwarp();
+                }
+            }
+        }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------ MMA issue (one thread)
         if (lane == 0) {
@@ -859,13 +912,20 @@ conv_i8_kernel(const ConvArgs a, const __grid_constant__ ConvI8Plan p, const __g
             const int buf = it & 1;
             const int nrows = min(it == 0 ? p.R0 : p.RT, s1 - g);
             const int ntm = (nrows * p.PW + kTileM - 1) / kTileM;
-            role_wait(warp == kEpiWarp0, &acc_full[buf], (it >> 1) & 1, a.status, dead, kEpiBarrier, kEpiThreads);
+            if (warp == kEpiWarp0) {
+                wait_or_die(&acc_full[buf], (it >> 1) & 1, a.status, dead);
+                if constexpr (kSk) wait_or_die(&st_full[buf], (it >> 1) & 1, a.status, dead);     // the tile's skip values
+            }
+            asm volatile("bar.sync %0, %1;" ::"r"(kEpiBarrier), "r"(kEpiThreads) : "memory");
             const bool alive = !*dead;
             tc::tc_fence_after_sync();
             if (etid == 0 && it < 8) RTN_TL(conv_i8, 56 + 2 * it);
             if constexpr (kNext) {
-                next_epilogue_tile(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, buf, g, nrows,
-                                   alive, q, lane, half, 2);
+                const float* sk_buf = kSk ? reinterpret_cast<const float*>(smem + p.off_skip) +
+                                                (size_t)buf * p.RT * p.sk_groups * (p.sk_box / 4) : nullptr;
+                next_epilogue_tile<kSk>(a, p, f, sC, reinterpret_cast<const float2*>(smem + p.off_t), tmem, buf, g, nrows,
+                                        alive, q, lane, half, 2, sk_buf);
+                if constexpr (kSk) tc::mbar_arrive(&st_empty[buf]);    // this thread has read its skip values
             } else if (p.const_tmem && a.dbg_acc == nullptr && a.pad_mode == RTN_PAD_CODE_ZERO) {
                 // Constants in tensor memory, no border classes: the thread's pixels of both sub-tiles (where the
                 // tile has one sub-tile, the second pixel does not exist and nothing is stored for it) go
@@ -1083,6 +1143,30 @@ static cudaError_t launch_conv_i8_any_mode(const ConvArgs& c, const NextLayerArg
         // packed pixel rows are read with plain loads by the converters: no staging ring
         p.use_tma = 0;
         p.smem_bytes = p.off_stage;
+        // The skip connection of a block's second layer: with no input ring to fill, the producer warp stages each
+        // tile's skip values in shared memory by TMA a tile ahead (boxes of 32 channels x one output row), and the
+        // epilogue reads them from there: as global loads they were a dependent trip to memory per half block, half of
+        // such a layer's time.  Two tile buffers must fit; the channel-split epilogue is the one that reads them.
+        const uint32_t base = (p.off_stage + 127) / 128 * 128;
+        const uint32_t sk_box = 32u * (uint32_t)c.Wo * 4u;
+        const int groups = (int)(c.N / 32);
+        if (f->skip != nullptr && (c.N == 64 || c.N == 128) && c.pad_mode == RTN_PAD_CODE_ZERO && c.Wo % 4 == 0 &&
+            reinterpret_cast<uintptr_t>(f->skip) % 16 == 0 &&
+            base + (uint64_t)2 * p.RT * groups * sk_box <= kSmemLimit) {
+            EncodeTiledFn enc = encode_tiled_fn();
+            const cuuint64_t dims[4] = {(cuuint64_t)c.Wo, (cuuint64_t)c.Ho, (cuuint64_t)c.N, (cuuint64_t)c.B};
+            const cuuint64_t strides[3] = {(cuuint64_t)c.Wo * 4, (cuuint64_t)c.Wo * c.Ho * 4,
+                                           (cuuint64_t)c.Wo * c.Ho * c.N * 4};
+            const cuuint32_t box[4] = {(cuuint32_t)c.Wo, 1, 32, 1};
+            const cuuint32_t estr[4] = {1, 1, 1, 1};
+            if (enc != nullptr &&
+                enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(f->skip), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS) {
+                p.sk_stage = 1; p.sk_groups = groups; p.off_skip = base; p.sk_box = sk_box;
+                p.smem_bytes = base + (size_t)2 * p.RT * groups * sk_box;
+            }
+        }
     }
     if (p.use_tma) {
         EncodeTiledFn enc = encode_tiled_fn();
@@ -1101,6 +1185,12 @@ static cudaError_t launch_conv_i8_any_mode(const ConvArgs& c, const NextLayerArg
         }
     }
     if (f != nullptr) {
+        if (p.sk_stage) {
+            cudaError_t e = cudaFuncSetAttribute(conv_i8_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)p.smem_bytes);
+            if (e != cudaSuccess) return e;
+            return launch_pdl(conv_i8_kernel<true, true>, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, s, c, p, tmap, *f);
+        }
         cudaError_t e = cudaFuncSetAttribute(conv_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)p.smem_bytes);
         if (e != cudaSuccess) return e;

@@ -249,14 +249,18 @@ __device__ __forceinline__ void next_layer_block16(const ConvArgs& a, const Next
 // The hand-over step for TWO pixels of a thread and one block of 16 output channels, all of which exist (layers
 // without border classes): every constant and threshold pair is fetched once and serves both pixels, and the two
 // pixels' arithmetic interleaves, which is what an epilogue bound by the round trips of its loads needs.
-// v0, v1: the block's accumulators of the two pixels; o0_0, o0_1: offsets of (b, n0, ho, wo) of each pixel;
+// v0, v1: the block's accumulators of the two pixels; o0_0, o0_1: offsets of (b, n0, ho, wo) of each pixel; sk0, sk1: when
+// not null, where channel n0 of each pixel's skip value sits in shared memory (channel n0 + j is j * sk_stride floats on);
 // ok0, ok1: the pixel exists (nothing is read or written for one that does not).
+template <bool kSk = false>
 __device__ __forceinline__ void next_layer_block16_pair(const ConvArgs& a, const NextLayerArgs& f,
                                                         const uint32_t (&v0)[16], const uint32_t (&v1)[16],
                                                         const float4* sC, const float2* sT, float fsx0, float fsx1,
                                                         bool ok0, bool ok1, int64_t o0_0, int64_t o0_1, int64_t ostride,
                                                         bool want_codes, uint32_t& nzb0, uint32_t& sgb0,
-                                                        uint32_t& nzb1, uint32_t& sgb1)
+                                                        uint32_t& nzb1, uint32_t& sgb1,
+                                                        const float* sk0 = nullptr, const float* sk1 = nullptr,
+                                                        int sk_stride = 0)
 {
     nzb0 = sgb0 = nzb1 = sgb1 = 0;
     #pragma unroll
@@ -275,9 +279,19 @@ __device__ __forceinline__ void next_layer_block16_pair(const ConvArgs& a, const
         if (f.skip != nullptr) {
             float s0[8], s1[8];
             #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                s0[j] = ok0 ? __ldg(f.skip + o0_0 + (int64_t)(h + j) * ostride) : 0.f;
-                s1[j] = ok1 ? __ldg(f.skip + o0_1 + (int64_t)(h + j) * ostride) : 0.f;
+            if constexpr (kSk) {
+                // staged in shared memory by the kernel's producer warp (sk_stride floats between channels)
+                #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    s0[j] = ok0 ? sk0[(h + j) * sk_stride] : 0.f;
+                    s1[j] = ok1 ? sk1[(h + j) * sk_stride] : 0.f;
+                }
+            } else {
+                #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    s0[j] = ok0 ? __ldg(f.skip + o0_0 + (int64_t)(h + j) * ostride) : 0.f;
+                    s1[j] = ok1 ? __ldg(f.skip + o0_1 + (int64_t)(h + j) * ostride) : 0.f;
+                }
             }
             #pragma unroll
             for (int j = 0; j < 8; ++j) { y0[j] += s0[j]; y1[j] += s1[j]; }
