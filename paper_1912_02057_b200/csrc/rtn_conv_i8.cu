@@ -29,7 +29,9 @@
 //   warps 4..11   epilogue: tcgen05.ld the accumulators of tile i-1, affine form, store fp32
 //   warps 2, 3, 12..17  converters: read a stage, ternarize, write the code array of tile i
 // When the input cannot be described to TMA (W not a multiple of 4, unaligned base) the converters
-// load the fp32 values themselves.
+// load the fp32 values themselves.  With packed pixel rows as input (hand-over from the layer before) there is
+// no stage ring; in a layer that also adds a skip connection the producer warp then stages each tile's skip
+// values in shared memory by TMA, a tile ahead of the epilogue that adds them (conv_i8_kernel<true, true>).
 #include "rtn_internal.cuh"
 #include "rtn_tcgen05.cuh"
 #include "rtn_conv_i8_common.cuh"
